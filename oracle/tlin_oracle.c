@@ -1,0 +1,201 @@
+/*
+ * CPU oracle for the TLinFormer attention hot path.  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, fp64 statement of what the GPU library must compute.  It is
+ * used by the tests, by the smoke check and by the benchmark's CPU-baseline
+ * leg, never by the product path, and it shares no code, header, table or
+ * helper with the CUDA sources.
+ *
+ * What it follows (paper: "Rethinking Transformer Connectivity: TLinFormer"):
+ *   - Section 3, the attention formula  softmax(Q K^T / sqrt(d_k)) V.  The
+ *     method is exact (no approximation), so the oracle is that definition
+ *     written out: every row's scores are materialised, the maximum is taken,
+ *     the exponentials are summed, and the values are averaged.  Two passes, no
+ *     tiling, no running maximum.
+ *   - Section 3, "Causal Attention": query i may use keys j <= i.  When the W
+ *     queries are the last W positions of an N-long sequence (history followed
+ *     by the generation window, Fig. "ideal connection"), query i sits at
+ *     absolute position N-W+i, hence the rule j <= N-W+i.
+ *   - Section 3, "Focused Attention" / "Cross Attention": a few queries over all
+ *     keys, unmasked (causal_window = 0).
+ *   - Appendix A, "Cache Hit": in a cached step only the newest token takes
+ *     part; it attends to every cached row including its own.
+ *
+ * Every function is pinned by tests that do not call it to produce their
+ * expectation (closed forms, brute force with an explicit probability matrix,
+ * a textbook library routine, invariants); no function here is "parity
+ * unpinned".
+ *
+ * Element types: 0 = bfloat16 bit patterns (uint16_t), 1 = IEEE float.
+ * Inputs are widened exactly to double.  Outputs are double.
+ * Threads: rows are independent; an OpenMP parallel-for hands them out.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { TLIN_REF_BF16 = 0, TLIN_REF_F32 = 1 };
+
+static double widen(const void *base, int elem_type, int64_t idx)
+{
+    if (elem_type == TLIN_REF_BF16) {
+        uint32_t bits = ((uint32_t)((const uint16_t *)base)[idx]) << 16;
+        float f;
+        memcpy(&f, &bits, sizeof f);
+        return (double)f;
+    }
+    return (double)((const float *)base)[idx];
+}
+
+int tlin_ref_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* Mask predicate (Section 3, causal rule, aligned to the end of the sequence). */
+int tlin_ref_allowed(int64_t i, int64_t j, int64_t N, int64_t W, int causal_window)
+{
+    if (j < 0 || j >= N) return 0;
+    if (causal_window) return j <= (N - W) + i;
+    return 1;
+}
+
+/*
+ * One query row against key/value rows [0, N): the attention formula of
+ * Section 3 with the mask above.  scores is caller scratch of N doubles.
+ */
+static void attend_row(const void *q, const void *k, const void *v, int elem_type,
+                       int64_t qoff, int64_t kvoff, int64_t i, int64_t N, int64_t W, int d,
+                       int causal_window, double *scores, double *out_row, double *lse_out)
+{
+    const double inv_sqrt_d = 1.0 / sqrt((double)d);
+    double m = -INFINITY;
+    for (int64_t j = 0; j < N; ++j) {
+        if (!tlin_ref_allowed(i, j, N, W, causal_window)) { scores[j] = -INFINITY; continue; }
+        double s = 0.0;
+        for (int c = 0; c < d; ++c)
+            s += widen(q, elem_type, qoff + c) * widen(k, elem_type, kvoff + j * d + c);
+        s *= inv_sqrt_d;
+        scores[j] = s;
+        if (s > m) m = s;
+    }
+    double l = 0.0;
+    for (int c = 0; c < d; ++c) out_row[c] = 0.0;
+    for (int64_t j = 0; j < N; ++j) {
+        if (scores[j] == -INFINITY) continue;
+        double p = exp(scores[j] - m);
+        l += p;
+        for (int c = 0; c < d; ++c) out_row[c] += p * widen(v, elem_type, kvoff + j * d + c);
+    }
+    for (int c = 0; c < d; ++c) out_row[c] /= l;
+    *lse_out = m + log(l);
+}
+
+/*
+ * q:[B,H,W,d]  k,v:[B,H,N,d]  ->  out:[B,H,W,d] (double)  lse:[B,H,W] (double)
+ * causal_window = 0: every query sees all N keys.
+ * causal_window = 1: query i sees key j iff j <= N-W+i; requires N >= W.
+ * Returns 0, or -1 on a bad argument.
+ */
+int tlin_ref_attn_forward(const void *q, const void *k, const void *v, int elem_type,
+                          double *out, double *lse,
+                          int B, int H, int64_t N, int64_t W, int d, int causal_window)
+{
+    if (!q || !k || !v || !out || !lse) return -1;
+    if (B <= 0 || H <= 0 || N <= 0 || W <= 0 || d <= 0) return -1;
+    if (causal_window && N < W) return -1;
+    if (elem_type != TLIN_REF_BF16 && elem_type != TLIN_REF_F32) return -1;
+    const int64_t rows = (int64_t)B * H * W;
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *scores = (double *)malloc((size_t)N * sizeof(double));
+        if (!scores) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp for schedule(dynamic, 4)
+        for (int64_t r = 0; r < rows; ++r) {
+            if (!scores) continue;
+            const int64_t bh = r / W, i = r % W;
+            attend_row(q, k, v, elem_type, (bh * W + i) * d, bh * N * d, i, N, W, d,
+                       causal_window, scores, out + r * d, lse + r);
+        }
+        free(scores);
+    }
+    return failed ? -2 : 0;
+}
+
+/*
+ * One cached decode step (Appendix A, "Cache Hit"; Section 5.2, static history
+ * cache).  k_cache,v_cache:[B,H,Ncap,d] hold `pos` valid rows.  The new key and
+ * value ([B,H,1,d]) are copied verbatim into row `pos`, then the new query
+ * attends to rows [0, pos] (its own row included, causal rule j <= i).
+ * The caches are modified in place.  out:[B,H,1,d], lse:[B,H].
+ */
+int tlin_ref_decode_step(const void *q_new, const void *k_new, const void *v_new,
+                         void *k_cache, void *v_cache, int elem_type,
+                         double *out, double *lse,
+                         int B, int H, int64_t Ncap, int64_t pos, int d)
+{
+    if (!q_new || !k_new || !v_new || !k_cache || !v_cache || !out || !lse) return -1;
+    if (B <= 0 || H <= 0 || d <= 0 || Ncap <= 0 || pos < 0 || pos >= Ncap) return -1;
+    if (elem_type != TLIN_REF_BF16 && elem_type != TLIN_REF_F32) return -1;
+    const size_t esz = elem_type == TLIN_REF_BF16 ? 2 : 4;
+    const int64_t L = pos + 1;
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *scores = (double *)malloc((size_t)L * sizeof(double));
+        if (!scores) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t bh = 0; bh < (int64_t)B * H; ++bh) {
+            if (!scores) continue;
+            char *kc = (char *)k_cache + (size_t)(bh * Ncap) * d * esz;
+            char *vc = (char *)v_cache + (size_t)(bh * Ncap) * d * esz;
+            memcpy(kc + (size_t)pos * d * esz, (const char *)k_new + (size_t)bh * d * esz, (size_t)d * esz);
+            memcpy(vc + (size_t)pos * d * esz, (const char *)v_new + (size_t)bh * d * esz, (size_t)d * esz);
+            /* a single unmasked query over the L rows now valid */
+            attend_row(q_new, kc, vc, elem_type, bh * d, 0, 0, L, 1, d, 0, scores, out + bh * d, lse + bh);
+        }
+        free(scores);
+    }
+    return failed ? -2 : 0;
+}
+
+/*
+ * Exact combination of two attention results over disjoint key sets A and B for
+ * the same queries: with z = exp(lse), softmax over A u B weights each side by
+ * z_a/(z_a+z_b) and z_b/(z_a+z_b).  lse = -inf marks an empty side.
+ * out_a,out_b,out:[rows,d]  lse_a,lse_b,lse:[rows], all double.
+ */
+int tlin_ref_merge_lse(const double *out_a, const double *lse_a, const double *out_b, const double *lse_b,
+                       double *out, double *lse, int64_t rows, int d)
+{
+    if (!out_a || !lse_a || !out_b || !lse_b || !out || !lse || rows < 0 || d <= 0) return -1;
+    for (int64_t r = 0; r < rows; ++r) {
+        const double la = lse_a[r], lb = lse_b[r];
+        const double m = la > lb ? la : lb;
+        if (m == -INFINITY) {
+            lse[r] = -INFINITY;
+            for (int c = 0; c < d; ++c) out[r * d + c] = 0.0;
+            continue;
+        }
+        const double wa = exp(la - m), wb = exp(lb - m);
+        const double z = wa + wb;
+        lse[r] = m + log(z);
+        for (int c = 0; c < d; ++c) out[r * d + c] = (wa * out_a[r * d + c] + wb * out_b[r * d + c]) / z;
+    }
+    return 0;
+}

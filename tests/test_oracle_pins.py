@@ -1,0 +1,363 @@
+"""Pins for the CPU oracle: every expectation here comes from the paper's formula
+worked by other means (explicit probability matrices, closed forms, invariants,
+a textbook library routine, hand-derived fixtures), never from the oracle itself."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import cost_model
+from paper_2508_20407_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+rng = np.random.default_rng(1234)
+
+
+def brute_force(q, k, v, causal_window):
+    """Explicit-matrix attention, written independently of the oracle: returns (out, lse, P)."""
+    q, k, v = (np.asarray(a, dtype=np.float64) for a in (q, k, v))
+    B, H, W, d = q.shape
+    N = k.shape[2]
+    S = np.einsum("bhid,bhjd->bhij", q, k) / math.sqrt(d)
+    if causal_window:
+        i = np.arange(W)[:, None]
+        j = np.arange(N)[None, :]
+        S = np.where(j <= (N - W) + i, S, -np.inf)
+    E = np.exp(S - S.max(axis=-1, keepdims=True))
+    P = E / E.sum(axis=-1, keepdims=True)
+    lse = np.log(np.exp(S).sum(axis=-1))
+    return np.einsum("bhij,bhjd->bhid", P, v), lse, P
+
+
+def rand(*shape):
+    return rng.standard_normal(shape).astype(np.float32)
+
+
+# ---------------------------------------------------------------- brute force / library
+@pytest.mark.parametrize("B,H,N,W,d,causal", [
+    (1, 1, 8, 4, 4, 1), (1, 1, 8, 4, 4, 0), (2, 3, 7, 7, 3, 1), (1, 2, 5, 1, 2, 1),
+    (1, 1, 1, 1, 1, 1), (2, 2, 33, 9, 8, 1), (1, 2, 33, 40, 8, 0), (1, 1, 6, 6, 5, 0),
+])
+def test_brute_force_tiny(B, H, N, W, d, causal):
+    q, k, v = rand(B, H, W, d), rand(B, H, N, d), rand(B, H, N, d)
+    out, lse = oracle.attn_forward(q, k, v, causal)
+    ref, ref_lse, P = brute_force(q, k, v, causal)
+    assert np.abs(P.sum(-1) - 1).max() < 1e-14
+    assert np.abs(out - ref).max() < 1e-13
+    assert np.abs(lse - ref_lse).max() < 1e-13
+
+
+def test_hand_derived_fixture():
+    vals = {}
+    consts = {"LN3": math.log(3.0), "LN4": math.log(4.0), "LN8": math.log(8.0)}
+    for line in open(os.path.join(GOLDEN, "attention_two_keys.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        name, *nums = line.split()
+        vals[name] = np.array([consts[x] if x in consts else float(x) for x in nums])
+    q = vals["q"].astype(np.float32).reshape(1, 1, 1, 4)
+    for nk, o_name, l_name in ((2, "out2", "lse2"), (3, "out3", "lse3")):
+        k = np.stack([vals[f"k{j}"] for j in range(nk)]).astype(np.float32).reshape(1, 1, nk, 4)
+        v = np.stack([vals[f"v{j}"] for j in range(nk)]).astype(np.float32).reshape(1, 1, nk, 4)
+        out, lse = oracle.attn_forward(q, k, v, 0)
+        assert np.abs(out.ravel() - vals[o_name]).max() < 2e-6
+        assert abs(lse.item() - vals[l_name].item()) < 1e-6
+
+
+def test_reduces_to_textbook_causal_when_history_empty():
+    # First training chunk has an empty history (Section 5.1): N == W, plain causal attention.
+    q, k, v = rand(2, 2, 17, 8), rand(2, 2, 17, 8), rand(2, 2, 17, 8)
+    out, _ = oracle.attn_forward(q, k, v, 1)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q).double(), torch.from_numpy(k).double(), torch.from_numpy(v).double(), is_causal=True)
+    assert np.abs(out - ref.numpy()).max() < 1e-13
+
+
+def test_reduces_to_textbook_self_attention():
+    # Self attention (Section 3): Q = K = V = X, unmasked.
+    x = rand(1, 3, 19, 8)
+    out, _ = oracle.attn_forward(x, x, x, 0)
+    xt = torch.from_numpy(x).double()
+    ref = torch.nn.functional.scaled_dot_product_attention(xt, xt, xt)
+    assert np.abs(out - ref.numpy()).max() < 1e-13
+
+
+def test_window_rows_equal_last_rows_of_full_causal_attention():
+    # One softmax over history + window == the last W rows of causal attention over the whole sequence.
+    N, W, d = 40, 12, 8
+    x_q, k, v = rand(1, 2, N, d), rand(1, 2, N, d), rand(1, 2, N, d)
+    full = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(x_q).double(), torch.from_numpy(k).double(), torch.from_numpy(v).double(), is_causal=True)
+    out, _ = oracle.attn_forward(x_q[:, :, N - W:], k, v, 1)
+    assert np.abs(out - full.numpy()[:, :, N - W:]).max() < 1e-13
+
+
+# ---------------------------------------------------------------- closed forms
+def test_constant_values_give_constant_output():
+    q, k = rand(1, 2, 5, 4), rand(1, 2, 11, 4)
+    v = np.ones((1, 2, 11, 4), dtype=np.float32)
+    for causal in (0, 1):
+        out, _ = oracle.attn_forward(q, k, v, causal)
+        assert np.abs(out - 1.0).max() < 1e-15
+
+
+@pytest.mark.parametrize("N,W", [(11, 5), (6, 6), (9, 1)])
+def test_zero_query_gives_mean_and_log_count(N, W):
+    q = np.zeros((1, 1, W, 4), dtype=np.float32)
+    k, v = rand(1, 1, N, 4), rand(1, 1, N, 4)
+    out, lse = oracle.attn_forward(q, k, v, 1)
+    for i in range(W):
+        cnt = N - W + i + 1
+        assert abs(lse[0, 0, i] - math.log(cnt)) < 1e-14
+        assert np.abs(out[0, 0, i] - v[0, 0, :cnt].astype(np.float64).mean(0)).max() < 1e-14
+    out, lse = oracle.attn_forward(q, k, v, 0)
+    assert np.abs(lse - math.log(N)).max() < 1e-14
+    assert np.abs(out - v.astype(np.float64).mean(2, keepdims=True)).max() < 1e-14
+
+
+def test_identical_keys_shift_lse_only():
+    d, N, W = 4, 9, 3
+    q, v = rand(1, 1, W, d), rand(1, 1, N, d)
+    k0 = rand(d)
+    k = np.broadcast_to(k0, (1, 1, N, d)).copy()
+    out, lse = oracle.attn_forward(q, k, v, 0)
+    s = (q[0, 0].astype(np.float64) @ k0.astype(np.float64)) / math.sqrt(d)
+    assert np.abs(lse[0, 0] - (s + math.log(N))).max() < 1e-13
+    assert np.abs(out[0, 0] - v[0, 0].astype(np.float64).mean(0)).max() < 1e-13
+
+
+def test_dominant_key_selects_its_value():
+    d, N = 4, 12
+    q, k, v = rand(1, 1, 1, d), 0.01 * rand(1, 1, N, d), rand(1, 1, N, d)
+    k[0, 0, 7] = 200.0 * q[0, 0, 0] / np.linalg.norm(q[0, 0, 0])
+    out, _ = oracle.attn_forward(q, k, v, 0)
+    assert np.abs(out[0, 0, 0] - v[0, 0, 7]).max() < 1e-12
+
+
+def test_key_shift_moves_lse_by_q_dot_c():
+    d, N, W = 8, 10, 4
+    # dyadic values keep k + c exact in fp32
+    q = np.round(rand(1, 1, W, d) * 8) / 8
+    k = np.round(rand(1, 1, N, d) * 8) / 8
+    v = rand(1, 1, N, d)
+    c = (np.round(rand(d) * 8) / 8).astype(np.float32)
+    out0, lse0 = oracle.attn_forward(q.astype(np.float32), k.astype(np.float32), v, 1)
+    out1, lse1 = oracle.attn_forward(q.astype(np.float32), (k + c).astype(np.float32), v, 1)
+    shift = (q[0, 0].astype(np.float64) @ c.astype(np.float64)) / math.sqrt(d)
+    assert np.abs(out1 - out0).max() < 1e-12
+    assert np.abs((lse1 - lse0)[0, 0] - shift).max() < 1e-12
+
+
+def test_key_permutation_invariance_without_mask():
+    q, k, v = rand(1, 2, 3, 4), rand(1, 2, 13, 4), rand(1, 2, 13, 4)
+    perm = rng.permutation(13)
+    out0, lse0 = oracle.attn_forward(q, k, v, 0)
+    out1, lse1 = oracle.attn_forward(q, k[:, :, perm].copy(), v[:, :, perm].copy(), 0)
+    assert np.abs(out1 - out0).max() < 1e-13 and np.abs(lse1 - lse0).max() < 1e-13
+
+
+def test_scale_is_inverse_sqrt_of_head_dim():
+    # single key pair: lse difference between two keys' scores isolates the 1/sqrt(d) factor
+    d = 16
+    q = np.zeros((1, 1, 1, d), np.float32); q[..., 0] = 4.0
+    k = np.zeros((1, 1, 1, d), np.float32); k[..., 0] = 3.0
+    v = rand(1, 1, 1, d)
+    _, lse = oracle.attn_forward(q, k, v, 0)
+    assert abs(lse.item() - 12.0 / 4.0) < 1e-14
+
+
+# ---------------------------------------------------------------- mask and causality
+def test_mask_predicate_exhaustive_small():
+    for N in range(1, 9):
+        for W in range(1, N + 1):
+            cnt = 0
+            for i in range(W):
+                for j in range(-1, N + 1):
+                    exp = (0 <= j < N) and (j <= N - W + i)
+                    assert oracle.allowed(i, j, N, W, 1) == exp
+                    cnt += exp
+                    assert oracle.allowed(i, j, N, W, 0) == (0 <= j < N)
+            assert cnt == cost_model.allowed_pairs(N, W, 1) == W * (N - W) + W * (W + 1) // 2
+
+
+def test_future_tokens_do_not_change_earlier_rows_bitwise():
+    N, W, d = 24, 10, 8
+    q, k, v = rand(1, 2, W, d), rand(1, 2, N, d), rand(1, 2, N, d)
+    out0, lse0 = oracle.attn_forward(q, k, v, 1)
+    for i in (0, 3, 8):
+        k2, v2 = k.copy(), v.copy()
+        k2[:, :, N - W + i + 1:] += 5.0
+        v2[:, :, N - W + i + 1:] -= 3.0
+        out1, lse1 = oracle.attn_forward(q, k2, v2, 1)
+        assert np.array_equal(out1[:, :, :i + 1], out0[:, :, :i + 1])
+        assert np.array_equal(lse1[:, :, :i + 1], lse0[:, :, :i + 1])
+        if i + 1 < W:
+            assert not np.array_equal(out1[:, :, i + 1:], out0[:, :, i + 1:])
+
+
+def test_rejects_window_longer_than_sequence():
+    with pytest.raises(ValueError):
+        oracle.attn_forward(rand(1, 1, 5, 4), rand(1, 1, 4, 4), rand(1, 1, 4, 4), 1)
+
+
+# ---------------------------------------------------------------- element types
+def test_bf16_inputs_are_widened_exactly():
+    q = torch.randn(1, 2, 5, 8, generator=torch.Generator().manual_seed(3)).bfloat16()
+    k = torch.randn(1, 2, 9, 8, generator=torch.Generator().manual_seed(4)).bfloat16()
+    v = torch.randn(1, 2, 9, 8, generator=torch.Generator().manual_seed(5)).bfloat16()
+    out_b, lse_b = oracle.attn_forward(q, k, v, 1)
+    ref, ref_lse, _ = brute_force(q.float().numpy(), k.float().numpy(), v.float().numpy(), 1)
+    assert np.abs(out_b - ref).max() < 1e-13 and np.abs(lse_b - ref_lse).max() < 1e-13
+    bits = k.view(torch.int16).numpy().view(np.uint16)
+    out_u, _ = oracle.attn_forward(q.view(torch.int16).numpy().view(np.uint16), bits,
+                                   v.view(torch.int16).numpy().view(np.uint16), 1)
+    assert np.array_equal(out_u, out_b)
+
+
+# ---------------------------------------------------------------- split / merge
+def merge_by_definition(oa, la, ob, lb):
+    za, zb = np.exp(la), np.exp(lb)
+    return (za[..., None] * oa + zb[..., None] * ob) / (za + zb)[..., None], np.log(za + zb)
+
+
+@pytest.mark.parametrize("split", [1, 5, 12])
+def test_attention_over_union_equals_merge_of_parts(split):
+    N, W, d = 13, 4, 8
+    q, k, v = rand(1, 2, W, d), rand(1, 2, N, d), rand(1, 2, N, d)
+    full, full_lse, _ = brute_force(q, k, v, 0)
+    oa, la, _ = brute_force(q, k[:, :, :split], v[:, :, :split], 0)
+    ob, lb, _ = brute_force(q, k[:, :, split:], v[:, :, split:], 0)
+    out, lse = oracle.merge_lse(oa, la, ob, lb)
+    assert np.abs(out - full).max() < 1e-12 and np.abs(lse - full_lse).max() < 1e-12
+    out_d, lse_d = merge_by_definition(oa, la, ob, lb)
+    assert np.abs(out - out_d).max() < 1e-12 and np.abs(lse - lse_d).max() < 1e-12
+
+
+def test_merge_with_empty_side_and_large_lse():
+    oa, ob = rng.standard_normal((3, 4)), rng.standard_normal((3, 4))
+    la = np.array([0.3, -np.inf, 900.0])
+    lb = np.array([-np.inf, -np.inf, 899.0])
+    out, lse = oracle.merge_lse(oa, la, ob, lb)
+    assert np.array_equal(out[0], oa[0]) and lse[0] == 0.3
+    assert lse[1] == -np.inf and np.array_equal(out[1], np.zeros(4))
+    w = 1.0 / (1.0 + math.exp(-1.0))
+    assert np.abs(out[2] - (w * oa[2] + (1 - w) * ob[2])).max() < 1e-14
+    assert abs(lse[2] - (900.0 + math.log1p(math.exp(-1.0)))) < 1e-12
+
+
+def test_history_plus_window_decomposition_matches_single_softmax():
+    # "combined" read as one softmax over history (unmasked) and window (causal): equals the
+    # merge of a focused call on the history and a plain causal call on the window.
+    N, W, d = 29, 7, 8
+    q, k, v = rand(1, 2, W, d), rand(1, 2, N, d), rand(1, 2, N, d)
+    joint, joint_lse = oracle.attn_forward(q, k, v, 1)
+    oh, lh = oracle.attn_forward(q, k[:, :, :N - W].copy(), v[:, :, :N - W].copy(), 0)
+    ow, lw = oracle.attn_forward(q, k[:, :, N - W:].copy(), v[:, :, N - W:].copy(), 1)
+    out, lse = merge_by_definition(oh, lh, ow, lw)
+    assert np.abs(out - joint).max() < 1e-12 and np.abs(lse - joint_lse).max() < 1e-12
+
+
+# ---------------------------------------------------------------- decode
+def test_decode_steps_equal_rows_of_full_forward_and_cache_bookkeeping():
+    B, H, N0, T, d = 2, 2, 11, 5, 8
+    Ncap = N0 + T + 2
+    canary = np.float32(-777.0)
+    k_cache = np.full((B, H, Ncap, d), canary, dtype=np.float32)
+    v_cache = np.full((B, H, Ncap, d), canary, dtype=np.float32)
+    k_hist, v_hist = rand(B, H, N0, d), rand(B, H, N0, d)
+    k_cache[:, :, :N0], v_cache[:, :, :N0] = k_hist, v_hist
+    qn, kn, vn = rand(T, B, H, 1, d), rand(T, B, H, 1, d), rand(T, B, H, 1, d)
+    k_all = np.concatenate([k_hist] + [kn[t] for t in range(T)], axis=2)
+    v_all = np.concatenate([v_hist] + [vn[t] for t in range(T)], axis=2)
+    q_all = np.concatenate([qn[t] for t in range(T)], axis=2)
+    full, full_lse, _ = brute_force(q_all, k_all, v_all, 1)
+    for t in range(T):
+        out, lse = oracle.decode_step(qn[t], kn[t], vn[t], k_cache, v_cache, N0 + t)
+        assert np.abs(out[:, :, 0] - full[:, :, t]).max() < 1e-13
+        assert np.abs(lse - full_lse[:, :, t]).max() < 1e-13
+        assert np.array_equal(k_cache[:, :, :N0 + t + 1], k_all[:, :, :N0 + t + 1])
+        assert np.array_equal(v_cache[:, :, :N0 + t + 1], v_all[:, :, :N0 + t + 1])
+        assert (k_cache[:, :, N0 + t + 1:] == canary).all() and (v_cache[:, :, N0 + t + 1:] == canary).all()
+
+
+def test_decode_matches_forward_oracle_rows_bf16():
+    wl = synth.Workload("t", 1, 2, 16, 37, 4, seed=9, decode=True)
+    (kc, vc), (qn, kn, vn) = synth.decode_inputs(wl)
+    k_all = torch.cat([kc[:, :, :wl.N]] + [kn[t] for t in range(wl.W)], dim=2)
+    v_all = torch.cat([vc[:, :, :wl.N]] + [vn[t] for t in range(wl.W)], dim=2)
+    q_all = torch.cat([qn[t] for t in range(wl.W)], dim=2)
+    full, full_lse = oracle.attn_forward(q_all, k_all, v_all, 1)
+    for t in range(wl.W):
+        out, lse = oracle.decode_step(qn[t], kn[t], vn[t], kc, vc, wl.N + t)
+        assert np.abs(out[:, :, 0] - full[:, :, t]).max() < 1e-13
+        assert np.abs(lse - full_lse[:, :, t]).max() < 1e-13
+    assert torch.equal(kc, k_all) and torch.equal(vc, v_all)
+
+
+def test_decode_rejects_bad_position():
+    z = np.zeros((1, 1, 1, 4), np.float32)
+    c = np.zeros((1, 1, 3, 4), np.float32)
+    for pos in (-1, 3):
+        with pytest.raises(ValueError):
+            oracle.decode_step(z, z, z, c, c.copy(), pos)
+
+
+# ---------------------------------------------------------------- the paper's cost model
+def test_cost_model_closed_forms_are_identities():
+    r = np.random.default_rng(7)
+    for _ in range(200):
+        W_oh, W_og, Hd, D = (int(r.integers(1, 300)), int(r.integers(1, 300)), int(r.integers(0, 9)), int(r.integers(1, 600)))
+        N = W_og + int(r.integers(1, 5000))
+        assert D * cost_model.pairs(cost_model.miss_layers(N, W_oh, W_og, Hd)) == cost_model.miss_closed_form(N, W_oh, W_og, Hd, D)
+        hit = cost_model.hit_layers(N, W_oh, W_og, Hd)
+        assert D * cost_model.pairs(hit) == cost_model.hit_closed_form(N, W_oh, W_og, Hd, D)
+        # slope/intercept form, Eq. (total cost = C1 N + C0)
+        c1 = D * (2 * W_oh + W_og)
+        c0 = D * (Hd * (W_oh ** 2 + W_og ** 2 + W_og * W_oh) + W_og ** 2 - W_og * W_oh)
+        assert c1 * N + c0 == cost_model.miss_closed_form(N, W_oh, W_og, Hd, D)
+
+
+def test_cost_model_hand_worked_examples():
+    for line in open(os.path.join(GOLDEN, "cost_model_examples.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        N, W_oh, W_og, Hd, D, miss, hit = (int(x) for x in line.split())
+        assert D * cost_model.pairs(cost_model.miss_layers(N, W_oh, W_og, Hd)) == miss
+        assert cost_model.miss_closed_form(N, W_oh, W_og, Hd, D) == miss
+        assert D * cost_model.pairs(cost_model.hit_layers(N, W_oh, W_og, Hd)) == hit
+        assert cost_model.hit_closed_form(N, W_oh, W_og, Hd, D) == hit
+
+
+# ---------------------------------------------------------------- the comparison gates themselves
+def test_gates_reject_zero_output_and_accept_rounding_noise():
+    import parity
+    wl = synth.WORKLOADS["cfg1_tiny"]
+    q, k, v = synth.forward_inputs(wl)
+    ref, ref_lse = oracle.attn_forward(q, k, v, 1)
+    with pytest.raises(AssertionError):
+        parity.check(np.zeros_like(ref), ref_lse, ref, ref_lse, "bf16", "zero control")
+    rounded = torch.from_numpy(ref).bfloat16().double().numpy()
+    parity.check(rounded, ref_lse.astype(np.float32), ref, ref_lse, "bf16", "bf16 rounding")
+    with pytest.raises(AssertionError):
+        parity.check(rounded, ref_lse + 0.01, ref, ref_lse, "bf16", "lse control")
+
+
+def test_stored_oracle_rows_have_not_drifted():
+    wl = synth.WORKLOADS["cfg1_tiny"]
+    q, k, v = synth.forward_inputs(wl)
+    out, lse = oracle.attn_forward(q, k, v, wl.causal_window)
+    n = 0
+    for line in open(os.path.join(GOLDEN, "oracle_cfg1_rows.txt")):
+        if line.startswith("#"):
+            continue
+        parts = line.split()
+        b, h, i = (int(x) for x in parts[:3])
+        vals = np.array([float(x) for x in parts[3:]])
+        assert abs(lse[b, h, i] - vals[0]) < 1e-9
+        assert np.abs(out[b, h, i, :8] - vals[1:]).max() < 1e-9
+        n += 1
+    assert n == 4
