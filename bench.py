@@ -1,0 +1,429 @@
+#!/usr/bin/env python
+"""Benchmark of the libtlin hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload fwd128k|fwd32k|fwd8k|decode]
+    python bench.py --impl reference ...        # the CPU oracle, as it stands, on the host cores
+
+One JSON line on stdout (rank 0).  A "step" is one pass of the hot path over one batch of synthetic
+input: for a forward workload the plan, the W x N exact-softmax attention with the causal window and
+the split merge; for the decode workload one cached single-token step (append + attend + merge).
+The headline workload is the N=131072 forward; the N=32768 forward and the cached decode are timed
+in the same run and reported under "also" (skip with --only).
+
+`value` is measured with the inputs resident in HBM; `e2e` goes through the host-buffer entry
+points, host<->device copies inside the timed region.  With --gpus N > 1 (under torchrun) every rank
+runs an independent replica of the same workload on its own GPU: the path has no exchange step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2508_20407_b200 import synth  # noqa: E402
+
+WORKLOADS = {"fwd128k": "cfg4_vlong", "fwd32k": "cfg3_long", "fwd8k": "cfg2_mid", "decode": "cfg5_decode"}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons for one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    sm.append(float(parts[0]))
+                    smax.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------- timing helpers
+def dist_info():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def barrier(world):
+    if world > 1:
+        torch.distributed.barrier()
+
+
+def max_over_ranks(x: float, world: int, device) -> float:
+    if world == 1:
+        return x
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def time_steps(step_fn, steps, warmup, world, device, sampler=None):
+    """Device time of `steps` calls (CUDA events on the current stream), max over ranks, in ms."""
+    for i in range(warmup):
+        step_fn(i)
+    torch.cuda.synchronize()
+    barrier(world)
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        step_fn(warmup + i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None
+    barrier(world)
+    torch.cuda.synchronize()
+    return max_over_ranks(ms, world, device), clocks
+
+
+# ----------------------------------------------------------------------------- the oracle as a timed baseline
+def oracle_forward_sample(wl, k_head, v_head, q_head, rows):
+    """Last `rows` query rows of one head through the CPU oracle (exactly those rows of the workload)."""
+    import oracle
+    q = q_head[wl.W - rows:].contiguous().view(1, 1, rows, wl.d)
+    t0 = time.perf_counter()
+    out, lse = oracle.attn_forward(q, k_head.view(1, 1, wl.N, wl.d), v_head.view(1, 1, wl.N, wl.d), wl.causal_window)
+    return time.perf_counter() - t0, out, lse
+
+
+def cpu_baseline_forward(wl, q_head, k_head, v_head, target_s=12.0):
+    import oracle
+    cores = oracle.num_threads()
+    probe = min(wl.W, max(cores * 4, 8))
+    t_probe, _, _ = oracle_forward_sample(wl, k_head, v_head, q_head, probe)
+    rows = int(min(wl.W, max(probe, probe * target_s / max(t_probe, 1e-6))))
+    rows = max(cores * 4, rows // (cores * 4) * (cores * 4))
+    rows = min(rows, wl.W)
+    t, out, lse = oracle_forward_sample(wl, k_head, v_head, q_head, rows)
+    t_full = t * (wl.B * wl.H * wl.W) / rows
+    return dict(value=wl.B * wl.N / t_full, unit="context tokens/s", cores=cores, kind="oracle",
+                sample=f"last {rows} of {wl.W} query rows of head (b=0,h=0), all {wl.N} keys: {t:.2f} s, "
+                       f"scaled by {wl.B * wl.H * wl.W}/{rows} rows"), (rows, out, lse)
+
+
+def cpu_baseline_decode(wl, kc_heads, vc_heads, q_new, k_new, v_new, pos, n_heads):
+    """One decode step for the first n_heads (b,h) pairs through the CPU oracle."""
+    import oracle
+    cores = oracle.num_threads()
+    kc = kc_heads.clone()
+    vc = vc_heads.clone()
+    t0 = time.perf_counter()
+    out, lse = oracle.decode_step(q_new, k_new, v_new, kc, vc, pos)
+    t = time.perf_counter() - t0
+    t_full = t * (wl.B * wl.H) / n_heads
+    gb = 2.0 * wl.B * wl.H * (pos + 1) * wl.d * 2 / 1e9
+    return dict(value=gb / t_full, unit="GB/s", cores=cores, kind="oracle",
+                sample=f"one decode step at pos={pos} for {n_heads} of {wl.B * wl.H} (b,h) pairs: {t:.2f} s, "
+                       f"scaled by {wl.B * wl.H}/{n_heads}"), (out, lse)
+
+
+# ----------------------------------------------------------------------------- GPU legs
+def fwd_bytes(wl):
+    return 2 * (2 * wl.B * wl.H * wl.N * wl.d + 2 * wl.B * wl.H * wl.W * wl.d) + 4 * wl.B * wl.H * wl.W
+
+
+def run_forward(wl, args, rank, world, device, peaks, with_cpu):
+    from paper_2508_20407_b200 import binding as tl
+    q, k, v = synth.forward_inputs(wl, device=device)
+    out = torch.empty_like(q)
+    lse = torch.empty((wl.B, wl.H, wl.W), dtype=torch.float32, device=device)
+    tl.ensure_workspace(tl.workspace_bytes_forward(wl.B, wl.H, wl.N, wl.W, wl.d, wl.causal_window), device)
+    launches = []
+
+    def step(_):
+        tl.tlin_attn_forward(q, k, v, out, lse, wl.causal_window)
+        launches.append(tl.tlin_last_launch_count())
+
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    ms, clocks = time_steps(step, args.steps, args.warmup, world, device, sampler)
+    ms_step = ms / args.steps
+    flop = 4.0 * wl.B * wl.H * wl.W * wl.N * wl.d
+    tflops = flop / (ms_step * 1e-3) / 1e12
+    t_tensor = flop / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = fwd_bytes(wl) / (peaks["hbm_gbs"] * 1e9)
+    bound = "tensor" if t_tensor >= t_hbm else "hbm"
+    if bound == "tensor":
+        roof = dict(bound="tensor", achieved=tflops, peak=peaks["bf16_tflops"], unit="TFLOP/s",
+                    frac=tflops / peaks["bf16_tflops"])
+    else:
+        gbs = fwd_bytes(wl) / (ms_step * 1e-3) / 1e9
+        roof = dict(bound="hbm", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s", frac=gbs / peaks["hbm_gbs"])
+    roof.update(traffic=None, peak_source=peaks["source"] + " (burst)", kernel="forward (attention kernel + split merge)",
+                roofline_ms=max(t_tensor, t_hbm) * 1e3)
+
+    # end to end: pinned host buffers through the host entry point
+    e2e = None
+    if not args.no_e2e:
+        q_h, k_h, v_h = (t.cpu().pin_memory() for t in (q, k, v))
+        out_h = torch.empty_like(q_h).pin_memory()
+        lse_h = torch.empty((wl.B, wl.H, wl.W), dtype=torch.float32).pin_memory()
+
+        def step_e2e(_):
+            tl.tlin_attn_forward_host(q_h, k_h, v_h, out_h, lse_h, q, k, v, out, lse, wl.causal_window)
+
+        n_e2e = max(2, min(args.steps, 5))
+        ms_e, _ = time_steps(step_e2e, n_e2e, 1, world, device)
+        h2d = sum(t.numel() * t.element_size() for t in (q_h, k_h, v_h))
+        d2h = out_h.numel() * out_h.element_size() + lse_h.numel() * 4
+        e2e = dict(value=world * wl.B * wl.N / (ms_e / n_e2e * 1e-3), unit="context tokens/s",
+                   h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, ms_per_step=ms_e / n_e2e, steps=n_e2e)
+        del q_h, k_h, v_h
+
+    res = dict(workload=wl.name, ms_per_step=ms_step, tokens_per_s=world * wl.B * wl.N / (ms_step * 1e-3),
+               tflops=tflops, roofline=roof, e2e=e2e, clocks=clocks,
+               gpu_launches=int(sum(launches[args.warmup:])), launches_per_step=launches[-1] if launches else 0)
+
+    if with_cpu and rank == 0:
+        tl.tlin_attn_forward(q, k, v, out, lse, wl.causal_window)
+        torch.cuda.synchronize()
+        cpu, (rows, ref, ref_lse) = cpu_baseline_forward(wl, q[0, 0].cpu(), k[0, 0].cpu(), v[0, 0].cpu())
+        got = out[0, 0, wl.W - rows:].float().cpu().numpy()
+        err = abs(got - ref[0, 0]).max()
+        lerr = abs(lse[0, 0, wl.W - rows:].cpu().numpy() - ref_lse[0, 0]).max()
+        cpu["parity_on_sample"] = dict(max_abs_err=float(err), lse_max_abs_err=float(lerr))
+        res["cpu_baseline"] = cpu
+    return res
+
+
+def run_decode(wl, args, rank, world, device, peaks, with_cpu):
+    from paper_2508_20407_b200 import binding as tl
+    (kc, vc), (qn, kn, vn) = synth.decode_inputs(wl, device=device)
+    ncap = kc.shape[2]
+    out = torch.empty((wl.B, wl.H, 1, wl.d), dtype=torch.bfloat16, device=device)
+    lse = torch.empty((wl.B, wl.H), dtype=torch.float32, device=device)
+    tl.ensure_workspace(tl.workspace_bytes_decode(wl.B, wl.H, ncap, wl.d), device)
+    launches = []
+    steps = args.decode_steps
+
+    def step(i):
+        t = i % wl.W
+        tl.tlin_decode_step(qn[t], kn[t], vn[t], kc, vc, wl.N + t, out, lse)
+        launches.append(tl.tlin_last_launch_count())
+
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    ms, clocks = time_steps(step, steps, args.warmup, world, device, sampler)
+    ms_step = ms / steps
+    # algorithmic bytes of the steps actually timed: K and V rows [0,pos] once each, plus q/k/v_new, out, lse
+    tot = 0
+    for i in range(args.warmup, args.warmup + steps):
+        pos = wl.N + (i % wl.W)
+        tot += 2 * wl.B * wl.H * (pos + 1) * wl.d * 2 + 4 * wl.B * wl.H * wl.d * 2 + 4 * wl.B * wl.H
+    gbs = tot / (ms * 1e-3) / 1e9
+    roof = dict(bound="hbm", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s", frac=gbs / peaks["hbm_gbs"],
+                traffic=None, peak_source=peaks["source"], kernel="decode (split-K kernel + merge)",
+                roofline_ms=tot / steps / (peaks["hbm_gbs"] * 1e9) * 1e3)
+    e2e = None
+    if not args.no_e2e:
+        host = [t.cpu().pin_memory() for t in (qn, kn, vn)]
+        out_h = torch.empty((wl.B, wl.H, 1, wl.d), dtype=torch.bfloat16).pin_memory()
+        lse_h = torch.empty((wl.B, wl.H), dtype=torch.float32).pin_memory()
+        qd, kd, vd = (torch.empty_like(qn[0]) for _ in range(3))
+
+        def step_e2e(i):
+            t = i % wl.W
+            tl.tlin_decode_step_host(host[0][t], host[1][t], host[2][t], out_h, lse_h, qd, kd, vd, out, lse, kc, vc, wl.N + t)
+            torch.cuda.current_stream().synchronize()   # the caller reads the token's result every step
+
+        n_e2e = min(steps, 32)
+        ms_e, _ = time_steps(step_e2e, n_e2e, 1, world, device)
+        nb = wl.B * wl.H * wl.d * 2
+        e2e = dict(value=world * (tot / steps) / (ms_e / n_e2e * 1e-3) / 1e9, unit="GB/s", h2d_bytes_per_step=3 * nb,
+                   d2h_bytes_per_step=nb + wl.B * wl.H * 4, ms_per_step=ms_e / n_e2e, steps=n_e2e)
+    res = dict(workload=wl.name, ms_per_step=ms_step, gb_per_s=world * gbs, steps=steps,
+               decode_tokens_per_s=world * wl.B / (ms_step * 1e-3), roofline=roof, e2e=e2e, clocks=clocks,
+               gpu_launches=int(sum(launches[args.warmup:])), launches_per_step=launches[-1] if launches else 0)
+    if with_cpu and rank == 0:
+        n_heads = 8
+        t = 0
+        # re-run step 0 so that out/lse hold its result, then compare the sampled heads
+        tl.tlin_decode_step(qn[t], kn[t], vn[t], kc, vc, wl.N + t, out, lse)
+        torch.cuda.synchronize()
+        flat = lambda x: x.reshape(1, wl.B * wl.H, *x.shape[2:])[:, :n_heads].contiguous().cpu()
+        cpu, (ref, ref_lse) = cpu_baseline_decode(wl, flat(kc), flat(vc), flat(qn[t]), flat(kn[t]), flat(vn[t]), wl.N + t, n_heads)
+        got = flat(out).float().numpy()
+        cpu["parity_on_sample"] = dict(max_abs_err=float(abs(got - ref).max()),
+                                       lse_max_abs_err=float(abs(lse.reshape(1, -1)[:, :n_heads].cpu().numpy() - ref_lse).max()))
+        res["cpu_baseline"] = cpu
+    return res
+
+
+# ----------------------------------------------------------------------------- reference arm (the oracle)
+def run_reference(args, rank, world):
+    if rank != 0:
+        return None
+    import oracle
+    wl = synth.WORKLOADS[WORKLOADS[args.workload]]
+    cores = oracle.num_threads()
+    if wl.decode:
+        n_heads = max(1, min(cores, 8))
+        small = synth.Workload(wl.name, 1, n_heads, wl.d, wl.N, 1, wl.seed, decode=True)
+        (kc, vc), (qn, kn, vn) = synth.decode_inputs(small, steps=1)
+        times = []
+        for i in range(args.warmup + args.steps):
+            t0 = time.perf_counter()
+            oracle.decode_step(qn[0], kn[0], vn[0], kc, vc, wl.N)
+            times.append(time.perf_counter() - t0)
+        t = sum(times[args.warmup:]) / args.steps
+        t_full = t * (wl.B * wl.H) / n_heads
+        gb = 2.0 * wl.B * wl.H * (wl.N + 1) * wl.d * 2 / 1e9
+        value, unit, metric = gb / t_full, "GB/s", "decode_kv_GB_per_s"
+        sample = f"one decode step at pos={wl.N} for {n_heads} of {wl.B * wl.H} (b,h) pairs per step, scaled"
+    else:
+        rows = max(cores, 8)
+        q, k, v = synth.forward_inputs_head(wl, 0, 0, q_rows=slice(wl.W - rows, wl.W))
+        q, k, v = q.view(1, 1, rows, wl.d), k.view(1, 1, wl.N, wl.d), v.view(1, 1, wl.N, wl.d)
+        times = []
+        for i in range(args.warmup + args.steps):
+            t0 = time.perf_counter()
+            oracle.attn_forward(q, k, v, wl.causal_window)
+            times.append(time.perf_counter() - t0)
+        t = sum(times[args.warmup:]) / args.steps
+        t_full = t * (wl.B * wl.H * wl.W) / rows
+        value, unit, metric = wl.B * wl.N / t_full, "context tokens/s", "context_tokens_per_s"
+        sample = f"last {rows} of {wl.W} query rows of head (0,0), all {wl.N} keys per step, scaled by rows"
+    return {"impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_full * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "W": wl.W, "d": wl.d,
+                       "causal_window": wl.causal_window},
+            "cpu_baseline": {"value": value, "unit": unit, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+
+
+# ----------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="fwd128k")
+    ap.add_argument("--impl", choices=["tlin", "reference"], default="tlin")
+    ap.add_argument("--only", action="store_true", help="time only --workload (no 'also' legs)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--decode-steps", type=int, default=0, help="timed decode steps (default: max(steps, 64))")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "tlin" else args.warmup
+    if args.decode_steps <= 0:
+        args.decode_steps = max(args.steps, 64)
+    rank, world, local = dist_info()
+
+    if args.impl == "reference":
+        line = run_reference(args, rank, world)
+        if line is not None:
+            print(json.dumps(line), flush=True)
+        return 0
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=device)
+    peaks = load_peaks()
+    wl = synth.WORKLOADS[WORKLOADS[args.workload]]
+    with_cpu = (not args.no_cpu) and world == 1
+    runner = run_decode if wl.decode else run_forward
+    main_res = runner(wl, args, rank, world, device, peaks, with_cpu)
+    also = []
+    if not args.only and world == 1:
+        for name in ("fwd32k", "decode"):
+            if name == args.workload:
+                continue
+            torch.cuda.empty_cache()
+            w2 = synth.WORKLOADS[WORKLOADS[name]]
+            also.append((run_decode if w2.decode else run_forward)(w2, args, rank, world, device, peaks, False))
+
+    if rank == 0:
+        if wl.decode:
+            metric, unit, value = "decode_kv_GB_per_s", "GB/s", main_res["gb_per_s"]
+        else:
+            metric, unit, value = "context_tokens_per_s", "context tokens/s", main_res["tokens_per_s"]
+        line = {
+            "metric": metric, "value": value, "unit": unit, "n_gpus": world,
+            "steps": main_res.get("steps", args.steps), "warmup": args.warmup, "ms_per_step": main_res["ms_per_step"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "W": wl.W, "d": wl.d,
+                       "causal_window": wl.causal_window, "parallelism": f"replicas x{world}",
+                       "l2": "inputs larger than L2 (K+V %.0f MB vs 126 MB), no flush" % (4e-6 * wl.B * wl.H * wl.N * wl.d)},
+            "tflops": main_res.get("tflops"),
+            "roofline": main_res["roofline"], "e2e": main_res["e2e"], "clocks": main_res["clocks"],
+            "gpu_launches": main_res["gpu_launches"], "launches_per_step": main_res["launches_per_step"],
+            "cpu_baseline": main_res.get("cpu_baseline"), "also": also,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

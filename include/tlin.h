@@ -1,0 +1,170 @@
+/*
+ * libtlin -- exact-softmax attention of TLinFormer's connectivity for NVIDIA B200 (sm_100a).
+ *
+ * Paper: "Rethinking Transformer Connectivity: TLinFormer, A Path to Exact, Full
+ * Context-Aware Linear Attention" (arXiv 2508.20407).  The library covers the part of the
+ * method whose cost grows with the sequence length N: a bounded set of W queries attending
+ * over all N keys/values with the exact softmax (Section 3, attention formula; "Focused
+ * Attention", "Cross Attention"), causal attention inside the generation window (Section 3,
+ * "Causal Attention"), and the cached single-token step (Appendix A, "Cache Hit").
+ *
+ * Conventions for every entry point
+ *   - Plain C ABI.  Unless a parameter is marked HOST, data pointers are DEVICE pointers,
+ *     borrowed for the duration of the call; the caller owns and frees every buffer.
+ *   - Tensors are dense, row-major, innermost dimension d, and 16-byte aligned.
+ *   - Calls that take a stream are asynchronous on it.  Nothing here allocates or frees
+ *     device memory; split-K scratch comes from the buffer given to tlin_set_workspace.
+ *   - Return value: TLIN_OK (0) or a negative tlin_status.  Argument errors are found on the
+ *     host before anything is launched.  No C++ exception crosses the boundary.
+ *   - bf16 entry points: bfloat16 inputs, fp32 accumulation, bfloat16 output rounded to
+ *     nearest even, fp32 log-sum-exp.  *_f32 entry points: fp32 throughout.
+ *   - lse is the natural logarithm of the row's sum of exp(score), scores already scaled by
+ *     1/sqrt(d).  (The paper has no such output; it is what makes partial results mergeable.)
+ */
+#ifndef TLIN_H
+#define TLIN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Opaque CUDA stream handle (a cudaStream_t passed as a pointer; NULL = default stream). */
+typedef void* tlin_stream_t;
+
+typedef enum {
+    TLIN_OK = 0,
+    TLIN_ERR_INVALID_ARG = -1, /* null or misaligned pointer, non-positive size, N < W with a causal window, bad pos */
+    TLIN_ERR_UNSUPPORTED = -2, /* head dimension outside what the path supports */
+    TLIN_ERR_WORKSPACE = -3,   /* workspace missing or smaller than tlin_workspace_bytes_* says */
+    TLIN_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed; the message is printed to stderr */
+    TLIN_ERR_TIMEOUT = -5,     /* a bounded device-side wait ran out (reported by tlin_get_status) */
+    TLIN_ERR_ARCH = -6         /* the current device is not compute capability 10.x */
+} tlin_status;
+
+/* ------------------------------------------------------------------------------------------
+ * Forward pass ("cache miss", Section 4.1): out = softmax(q k^T / sqrt(d)) v per (b,h).
+ *   q   [B,H,W,d]   W query rows: the summary queries of focused attention, or the generation window
+ *   k,v [B,H,N,d]   all N keys / values
+ *   out [B,H,W,d]   lse [B,H,W] (fp32; may be NULL)
+ * causal_window = 0  every query uses all N keys (Section 3, "Focused Attention"/"Cross Attention").
+ * causal_window = 1  the queries are the LAST W positions of the N-long sequence; query i uses key j
+ *                    iff j <= N-W+i: the history is unmasked and the window is causal (Section 3,
+ *                    "Causal Attention", j <= i, aligned to the end).  One softmax runs over the
+ *                    union of both key sets.  Requires N >= W.
+ * bf16 path: d in {64,128} runs on the tensor cores; any other d that is a multiple of 8 up to 256
+ * runs on the CUDA-core kernel.  f32 path: d a multiple of 4 up to 256 (covers the paper's d = 36).
+ * Uses the workspace when the plan splits the key range (see tlin_workspace_bytes_forward).
+ */
+int tlin_attn_forward(const void* q, const void* k, const void* v, void* out, float* lse,
+                      int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream);
+
+int tlin_attn_forward_f32(const float* q, const float* k, const float* v, float* out, float* lse,
+                          int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream);
+
+/* Same as tlin_attn_forward with HOST input/output buffers (ideally pinned).  *_h are HOST
+ * pointers; *_d are DEVICE staging buffers of the same shapes, supplied by the caller.  Copies
+ * q,k,v host->device, runs the forward, copies out (and lse if lse_h != NULL) device->host, all on
+ * `stream`; the caller synchronises the stream before reading out_h. */
+int tlin_attn_forward_host(const void* q_h, const void* k_h, const void* v_h, void* out_h, float* lse_h,
+                           void* q_d, void* k_d, void* v_d, void* out_d, float* lse_d,
+                           int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Cached decode step ("cache hit", Section 4.2 and Appendix A: only the newest token takes part;
+ * the history cache stays static, Section 5.2).
+ *   k_cache,v_cache [B,H,Ncap,d] bf16, rows [0,pos) valid on entry
+ *   q_new,k_new,v_new [B,H,1,d] bf16;  out [B,H,1,d] bf16;  lse [B,H] fp32 (may be NULL)
+ * Copies k_new,v_new bit-for-bit into row `pos` of the caches, then attends q_new over rows
+ * [0,pos] (its own row included).  Rows above pos are not touched.  The caller advances pos.
+ * Equals row t of the forward over the final sequence with causal_window = 1.
+ * d in {64,128}.  Needs the workspace (tlin_workspace_bytes_decode).  0 <= pos < Ncap.
+ */
+int tlin_decode_step(const void* q_new, const void* k_new, const void* v_new,
+                     void* k_cache, void* v_cache, void* out, float* lse,
+                     int B, int H, int Ncap, int pos, int d, tlin_stream_t stream);
+
+/* tlin_decode_step with HOST q/k/v_new and out/lse (the caches stay on the device).  *_d are
+ * DEVICE staging buffers ([B,H,1,d] each, lse_d [B,H]). */
+int tlin_decode_step_host(const void* q_new_h, const void* k_new_h, const void* v_new_h, void* out_h, float* lse_h,
+                          void* q_new_d, void* k_new_d, void* v_new_d, void* out_d, float* lse_d,
+                          void* k_cache, void* v_cache,
+                          int B, int H, int Ncap, int pos, int d, tlin_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Exact merge of two results over DISJOINT key sets for the same queries (not in the paper; it is
+ * the split-K combine, exposed so that "history" and "window" attention may also be computed
+ * separately and joined): lse = log(e^lse_a + e^lse_b), out = (e^lse_a out_a + e^lse_b out_b)/e^lse.
+ * An lse of -inf marks an empty side.  out_* [rows,d] bf16 (or fp32 for _f32), lse_* [rows] fp32.
+ * out/lse may alias out_a/lse_a.
+ */
+int tlin_merge_lse(const void* out_a, const float* lse_a, const void* out_b, const float* lse_b,
+                   void* out, float* lse, int64_t rows, int d, tlin_stream_t stream);
+int tlin_merge_lse_f32(const float* out_a, const float* lse_a, const float* out_b, const float* lse_b,
+                       float* out, float* lse, int64_t rows, int d, tlin_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Workspace.  Split-K partial results live in one caller-owned device buffer, registered once per
+ * process (per device) and borrowed until replaced.  Calls on different streams that both need the
+ * workspace must not overlap.  The *_bytes functions are pure host arithmetic.
+ */
+size_t tlin_workspace_bytes_forward(int B, int H, int N, int W, int d, int causal_window);
+size_t tlin_workspace_bytes_decode(int B, int H, int Ncap, int d);
+int tlin_set_workspace(void* dev_ptr, size_t bytes);
+
+/* ------------------------------------------------------------------------------------------
+ * Host-side planning (pure integer arithmetic; callable without a GPU).  The paper is silent on
+ * scheduling; its integer shadow is the cost model of Section 4 / Appendix A: the allowed
+ * (query,key) pairs of a call number W*N without a mask and W*(N-W) + W*(W+1)/2 with the window.
+ */
+typedef struct {
+    int32_t tile_m;        /* query rows per CTA                                             */
+    int32_t tile_n;        /* keys per tile                                                  */
+    int32_t q_tiles;       /* ceil(W / tile_m): CTAs that share one key range                */
+    int32_t key_tiles;     /* ceil(N / tile_n) per (b,h)                                     */
+    int32_t n_groups;      /* groups of q_tiles CTAs; group g streams units [start(g), start(g+1)) */
+    int32_t n_ctas;        /* n_groups * q_tiles                                             */
+    int64_t total_units;   /* B*H*key_tiles; unit u = (bh = u / key_tiles, tile = u % key_tiles) */
+    int32_t uses_workspace;/* 1 if any (b,h) is split between groups                         */
+    int32_t tensor_path;   /* 1 = tcgen05 kernel, 0 = CUDA-core kernel                       */
+    int64_t workspace_bytes;
+} tlin_fwd_plan;
+
+typedef struct {
+    int32_t splits;        /* CTAs per (b,h)                                                 */
+    int32_t keys_per_split;/* split s covers keys [s*keys_per_split, min(L, (s+1)*keys_per_split)) */
+    int32_t n_ctas;
+    int64_t workspace_bytes;
+} tlin_decode_plan;
+
+/* num_sms <= 0 means "use the value of the B200 (148)". */
+int tlin_plan_forward(int B, int H, int N, int W, int d, int causal_window, int is_f32, int num_sms, tlin_fwd_plan* plan);
+int tlin_plan_decode(int B, int H, int L, int d, int num_sms, tlin_decode_plan* plan);
+/* First unit of group g: floor(g * total_units / n_groups). */
+int64_t tlin_plan_group_start(const tlin_fwd_plan* plan, int g);
+/* Mask predicate: may query i (0 <= i < W) use key j?  1 or 0. */
+int tlin_allowed(int64_t i, int64_t j, int64_t N, int64_t W, int causal_window);
+/* Class of key tile `kt` for query tile `qt`: 0 = no allowed pair (skipped), 1 = every in-range pair
+ * allowed and the tile lies fully inside [0,N), 2 = mixed (masked element by element). */
+int tlin_tile_class(int64_t N, int64_t W, int causal_window, int tile_m, int tile_n, int qt, int kt);
+
+/* ------------------------------------------------------------------------------------------
+ * Status and options.
+ */
+/* Synchronises `stream`, then returns and clears the device-side error word (TLIN_OK or
+ * TLIN_ERR_TIMEOUT), or TLIN_ERR_CUDA if the stream reports an error. */
+int tlin_get_status(tlin_stream_t stream);
+const char* tlin_status_string(int status);
+const char* tlin_version(void);
+/* Which kernel serves tlin_attn_forward: 0 = automatic, 1 = always the CUDA-core kernel,
+ * 2 = tensor-core kernel (TLIN_ERR_UNSUPPORTED if the shape does not allow it).  Returns the old value. */
+int tlin_set_forward_impl(int impl);
+/* Number of kernels launched by the last tlin_* compute call on this thread. */
+int tlin_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TLIN_H */

@@ -1,0 +1,271 @@
+"""ctypes binding over the C-ABI declared in include/tlin.h.
+
+Argument marshalling only: every function takes torch tensors (device memory, streams) and hands
+raw pointers and sizes to libtlin.so.  No attention arithmetic happens here and there is no
+fallback: if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtlin.so")
+
+TLIN_OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_ARCH = -1, -2, -3, -4, -5, -6
+
+
+class TlinError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class FwdPlan(ctypes.Structure):
+    _fields_ = [("tile_m", ctypes.c_int32), ("tile_n", ctypes.c_int32), ("q_tiles", ctypes.c_int32),
+                ("key_tiles", ctypes.c_int32), ("n_groups", ctypes.c_int32), ("n_ctas", ctypes.c_int32),
+                ("total_units", ctypes.c_int64), ("uses_workspace", ctypes.c_int32),
+                ("tensor_path", ctypes.c_int32), ("workspace_bytes", ctypes.c_int64)]
+
+
+class DecodePlan(ctypes.Structure):
+    _fields_ = [("splits", ctypes.c_int32), ("keys_per_split", ctypes.c_int32), ("n_ctas", ctypes.c_int32),
+                ("workspace_bytes", ctypes.c_int64)]
+
+
+_vp, _i, _i64, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t
+
+# name -> (restype, argtypes); mirrors include/tlin.h one to one
+SIGNATURES = {
+    "tlin_attn_forward": (_i, [_vp] * 5 + [_i] * 6 + [_vp]),
+    "tlin_attn_forward_f32": (_i, [_vp] * 5 + [_i] * 6 + [_vp]),
+    "tlin_attn_forward_host": (_i, [_vp] * 10 + [_i] * 6 + [_vp]),
+    "tlin_decode_step": (_i, [_vp] * 7 + [_i] * 5 + [_vp]),
+    "tlin_decode_step_host": (_i, [_vp] * 12 + [_i] * 5 + [_vp]),
+    "tlin_merge_lse": (_i, [_vp] * 6 + [_i64, _i, _vp]),
+    "tlin_merge_lse_f32": (_i, [_vp] * 6 + [_i64, _i, _vp]),
+    "tlin_workspace_bytes_forward": (_sz, [_i] * 6),
+    "tlin_workspace_bytes_decode": (_sz, [_i] * 4),
+    "tlin_set_workspace": (_i, [_vp, _sz]),
+    "tlin_plan_forward": (_i, [_i] * 8 + [ctypes.POINTER(FwdPlan)]),
+    "tlin_plan_decode": (_i, [_i] * 5 + [ctypes.POINTER(DecodePlan)]),
+    "tlin_plan_group_start": (_i64, [ctypes.POINTER(FwdPlan), _i]),
+    "tlin_allowed": (_i, [_i64] * 4 + [_i]),
+    "tlin_tile_class": (_i, [_i64, _i64, _i, _i, _i, _i, _i]),
+    "tlin_get_status": (_i, [_vp]),
+    "tlin_status_string": (ctypes.c_char_p, [_i]),
+    "tlin_version": (ctypes.c_char_p, []),
+    "tlin_set_forward_impl": (_i, [_i]),
+    "tlin_last_launch_count": (_i, []),
+}
+
+_lib = None
+_workspace_tensor = None  # keeps the registered workspace alive
+
+
+def lib():
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2508_20407_b200.build` "
+                               "(there is no CPU fallback)")
+        l = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(l, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = l
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().tlin_status_string(status).decode()
+
+
+def version() -> str:
+    return lib().tlin_version().decode()
+
+
+def _check(rc: int, where: str):
+    if rc != TLIN_OK:
+        raise TlinError(rc, where)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dev(t, dtype, shape, name):
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous {dtype} of shape {tuple(shape)}, got {t.dtype} {tuple(t.shape)}")
+
+
+# ------------------------------------------------------------------ workspace
+def workspace_bytes_forward(B, H, N, W, d, causal_window) -> int:
+    return int(lib().tlin_workspace_bytes_forward(B, H, N, W, d, int(causal_window)))
+
+
+def workspace_bytes_decode(B, H, Ncap, d) -> int:
+    return int(lib().tlin_workspace_bytes_decode(B, H, Ncap, d))
+
+
+def set_workspace(t: torch.Tensor | None):
+    """Registers a device buffer (any dtype) as split-K scratch; the tensor is kept alive here."""
+    global _workspace_tensor
+    if t is None:
+        _check(lib().tlin_set_workspace(None, 0), "tlin_set_workspace")
+    else:
+        if not t.is_cuda or not t.is_contiguous():
+            raise ValueError("workspace must be a contiguous CUDA tensor")
+        _check(lib().tlin_set_workspace(_ptr(t), t.numel() * t.element_size()), "tlin_set_workspace")
+    _workspace_tensor = t
+
+
+def ensure_workspace(nbytes: int, device="cuda"):
+    """Grows the registered workspace to at least ``nbytes`` (allocation happens here, in torch)."""
+    global _workspace_tensor
+    cur = 0 if _workspace_tensor is None else _workspace_tensor.numel()
+    if nbytes > cur or (_workspace_tensor is not None and str(_workspace_tensor.device) != str(torch.device(device)) and torch.device(device).index is not None):
+        set_workspace(torch.empty(max(nbytes, 1 << 20), dtype=torch.uint8, device=device))
+    return _workspace_tensor
+
+
+# ------------------------------------------------------------------ compute
+def tlin_attn_forward(q, k, v, out=None, lse=None, causal_window=1, stream=None):
+    """bf16 forward.  q [B,H,W,d], k,v [B,H,N,d] -> (out [B,H,W,d] bf16, lse [B,H,W] fp32)."""
+    B, H, W, d = q.shape
+    N = k.shape[2]
+    _dev(q, torch.bfloat16, (B, H, W, d), "q")
+    _dev(k, torch.bfloat16, (B, H, N, d), "k")
+    _dev(v, torch.bfloat16, (B, H, N, d), "v")
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((B, H, W), dtype=torch.float32, device=q.device)
+    _dev(out, torch.bfloat16, (B, H, W, d), "out")
+    _dev(lse, torch.float32, (B, H, W), "lse")
+    ensure_workspace(workspace_bytes_forward(B, H, N, W, d, causal_window), q.device)
+    _check(lib().tlin_attn_forward(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), B, H, N, W, d,
+                                   int(causal_window), _stream(stream)), "tlin_attn_forward")
+    return out, lse
+
+
+def tlin_attn_forward_f32(q, k, v, out=None, lse=None, causal_window=1, stream=None):
+    """fp32 forward (CUDA-core kernel)."""
+    B, H, W, d = q.shape
+    N = k.shape[2]
+    _dev(q, torch.float32, (B, H, W, d), "q")
+    _dev(k, torch.float32, (B, H, N, d), "k")
+    _dev(v, torch.float32, (B, H, N, d), "v")
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((B, H, W), dtype=torch.float32, device=q.device)
+    _dev(out, torch.float32, (B, H, W, d), "out")
+    _dev(lse, torch.float32, (B, H, W), "lse")
+    _check(lib().tlin_attn_forward_f32(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), B, H, N, W, d,
+                                       int(causal_window), _stream(stream)), "tlin_attn_forward_f32")
+    return out, lse
+
+
+def tlin_attn_forward_host(q_h, k_h, v_h, out_h, lse_h, q_d, k_d, v_d, out_d, lse_d, causal_window=1, stream=None):
+    """Forward with HOST (pinned) q/k/v/out/lse and caller-supplied device staging tensors."""
+    B, H, W, d = q_d.shape
+    N = k_d.shape[2]
+    for t, n in ((q_h, "q_h"), (k_h, "k_h"), (v_h, "v_h"), (out_h, "out_h"), (lse_h, "lse_h")):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError(f"{n} must be a contiguous host tensor")
+    ensure_workspace(workspace_bytes_forward(B, H, N, W, d, causal_window), q_d.device)
+    _check(lib().tlin_attn_forward_host(_ptr(q_h), _ptr(k_h), _ptr(v_h), _ptr(out_h), _ptr(lse_h),
+                                        _ptr(q_d), _ptr(k_d), _ptr(v_d), _ptr(out_d), _ptr(lse_d),
+                                        B, H, N, W, d, int(causal_window), _stream(stream)), "tlin_attn_forward_host")
+    return out_h, lse_h
+
+
+def tlin_decode_step(q_new, k_new, v_new, k_cache, v_cache, pos, out=None, lse=None, stream=None):
+    """One cached decode step: appends k_new/v_new at row pos, attends q_new over rows [0,pos]."""
+    B, H, Ncap, d = k_cache.shape
+    for t, n in ((q_new, "q_new"), (k_new, "k_new"), (v_new, "v_new")):
+        _dev(t, torch.bfloat16, (B, H, 1, d), n)
+    _dev(k_cache, torch.bfloat16, (B, H, Ncap, d), "k_cache")
+    _dev(v_cache, torch.bfloat16, (B, H, Ncap, d), "v_cache")
+    if out is None:
+        out = torch.empty_like(q_new)
+    if lse is None:
+        lse = torch.empty((B, H), dtype=torch.float32, device=q_new.device)
+    ensure_workspace(workspace_bytes_decode(B, H, Ncap, d), q_new.device)
+    _check(lib().tlin_decode_step(_ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache),
+                                  _ptr(out), _ptr(lse), B, H, Ncap, int(pos), d, _stream(stream)), "tlin_decode_step")
+    return out, lse
+
+
+def tlin_decode_step_host(q_new_h, k_new_h, v_new_h, out_h, lse_h, q_new_d, k_new_d, v_new_d, out_d, lse_d,
+                          k_cache, v_cache, pos, stream=None):
+    B, H, Ncap, d = k_cache.shape
+    ensure_workspace(workspace_bytes_decode(B, H, Ncap, d), k_cache.device)
+    _check(lib().tlin_decode_step_host(_ptr(q_new_h), _ptr(k_new_h), _ptr(v_new_h), _ptr(out_h), _ptr(lse_h),
+                                       _ptr(q_new_d), _ptr(k_new_d), _ptr(v_new_d), _ptr(out_d), _ptr(lse_d),
+                                       _ptr(k_cache), _ptr(v_cache), B, H, Ncap, int(pos), d, _stream(stream)),
+           "tlin_decode_step_host")
+    return out_h, lse_h
+
+
+def tlin_merge_lse(out_a, lse_a, out_b, lse_b, out=None, lse=None, stream=None):
+    """Exact merge of two results over disjoint key sets (bf16 or fp32 outputs, fp32 lse)."""
+    d = out_a.shape[-1]
+    rows = out_a.numel() // d
+    if out is None:
+        out = torch.empty_like(out_a)
+    if lse is None:
+        lse = torch.empty_like(lse_a)
+    fn = lib().tlin_merge_lse_f32 if out_a.dtype == torch.float32 else lib().tlin_merge_lse
+    _check(fn(_ptr(out_a), _ptr(lse_a), _ptr(out_b), _ptr(lse_b), _ptr(out), _ptr(lse), rows, d, _stream(stream)),
+           "tlin_merge_lse")
+    return out, lse
+
+
+# ------------------------------------------------------------------ host logic
+def tlin_plan_forward(B, H, N, W, d, causal_window, is_f32=False, num_sms=0) -> FwdPlan:
+    p = FwdPlan()
+    _check(lib().tlin_plan_forward(B, H, N, W, d, int(causal_window), int(is_f32), num_sms, ctypes.byref(p)), "tlin_plan_forward")
+    return p
+
+
+def tlin_plan_decode(B, H, L, d, num_sms=0) -> DecodePlan:
+    p = DecodePlan()
+    _check(lib().tlin_plan_decode(B, H, L, d, num_sms, ctypes.byref(p)), "tlin_plan_decode")
+    return p
+
+
+def tlin_plan_group_start(plan: FwdPlan, g: int) -> int:
+    return int(lib().tlin_plan_group_start(ctypes.byref(plan), g))
+
+
+def tlin_allowed(i, j, N, W, causal_window) -> int:
+    return int(lib().tlin_allowed(i, j, N, W, int(causal_window)))
+
+
+def tlin_tile_class(N, W, causal_window, tile_m, tile_n, qt, kt) -> int:
+    return int(lib().tlin_tile_class(N, W, int(causal_window), tile_m, tile_n, qt, kt))
+
+
+def tlin_get_status(stream=None) -> int:
+    return int(lib().tlin_get_status(_stream(stream)))
+
+
+def tlin_set_forward_impl(impl: int) -> int:
+    return int(lib().tlin_set_forward_impl(impl))
+
+
+def tlin_last_launch_count() -> int:
+    return int(lib().tlin_last_launch_count())

@@ -1,0 +1,217 @@
+// C-ABI of libtlin: argument validation, planning, dispatch.  Every check runs on the host before
+// any launch; no exception leaves this file.
+#include "tlin_internal.h"
+#include <atomic>
+#include <mutex>
+
+namespace tlin {
+
+namespace {
+std::mutex g_mu;
+Workspace g_ws = {nullptr, 0};
+std::atomic<int> g_impl{0};
+thread_local int t_launches = 0;
+__device__ int g_status_word = 0;
+
+struct DevInfo { int checked; int major; int sms; };
+DevInfo g_dev[64] = {};
+
+int device_info(int* sms) {
+    int dev = 0;
+    TLIN_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return TLIN_ERR_CUDA;
+    DevInfo& di = g_dev[dev];
+    if (!di.checked) {
+        std::lock_guard<std::mutex> lk(g_mu);
+        TLIN_CUDA_CHECK(cudaDeviceGetAttribute(&di.major, cudaDevAttrComputeCapabilityMajor, dev));
+        TLIN_CUDA_CHECK(cudaDeviceGetAttribute(&di.sms, cudaDevAttrMultiProcessorCount, dev));
+        di.checked = 1;
+    }
+    if (di.major != 10) return TLIN_ERR_ARCH;
+    *sms = di.sms;
+    return TLIN_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+}  // namespace
+
+Workspace workspace() {
+    std::lock_guard<std::mutex> lk(g_mu);
+    return g_ws;
+}
+int* status_word() {
+    int* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_status_word) != cudaSuccess) return nullptr;
+    return p;
+}
+void count_launch(int n) { t_launches += n; }
+int forward_impl() { return g_impl.load(); }
+
+}  // namespace tlin
+
+using namespace tlin;
+
+static int forward_common(const void* q, const void* k, const void* v, void* out, float* lse,
+                          int B, int H, int N, int W, int d, int causal_window, int is_f32, cudaStream_t st) {
+    t_launches = 0;
+    if (!q || !k || !v || !out) return TLIN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || N <= 0 || W <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    if (causal_window != 0 && causal_window != 1) return TLIN_ERR_INVALID_ARG;
+    if (causal_window && N < W) return TLIN_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return TLIN_ERR_INVALID_ARG;
+    if (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)) return TLIN_ERR_INVALID_ARG;
+    int sms = 0;
+    // shape support is decided before the device is looked at, so that it can be tested without one
+    tlin_fwd_plan plan;
+    int rc = tlin_plan_forward(B, H, N, W, d, causal_window, is_f32, 0, &plan);
+    if (rc != TLIN_OK) return rc;
+    rc = device_info(&sms);
+    if (rc != TLIN_OK) return rc;
+    rc = tlin_plan_forward(B, H, N, W, d, causal_window, is_f32, sms, &plan);
+    if (rc != TLIN_OK) return rc;
+    if (is_f32)
+        return launch_fwd_simt_f32((const float*)q, (const float*)k, (const float*)v, (float*)out, lse, B, H, N, W, d, causal_window, st);
+    if (!plan.tensor_path)
+        return launch_fwd_simt_bf16(q, k, v, out, lse, B, H, N, W, d, causal_window, st);
+    float* ws = nullptr;
+    if (plan.uses_workspace) {
+        const Workspace w = workspace();
+        if (!w.ptr || w.bytes < (size_t)plan.workspace_bytes) return TLIN_ERR_WORKSPACE;
+        ws = (float*)w.ptr;
+    }
+    return launch_fwd_tc(q, k, v, out, lse, B, H, N, W, d, causal_window, plan, ws, st);
+}
+
+extern "C" int tlin_attn_forward(const void* q, const void* k, const void* v, void* out, float* lse,
+                                 int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream) {
+    return forward_common(q, k, v, out, lse, B, H, N, W, d, causal_window, 0, (cudaStream_t)stream);
+}
+
+extern "C" int tlin_attn_forward_f32(const float* q, const float* k, const float* v, float* out, float* lse,
+                                     int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream) {
+    return forward_common(q, k, v, out, lse, B, H, N, W, d, causal_window, 1, (cudaStream_t)stream);
+}
+
+extern "C" int tlin_attn_forward_host(const void* q_h, const void* k_h, const void* v_h, void* out_h, float* lse_h,
+                                      void* q_d, void* k_d, void* v_d, void* out_d, float* lse_d,
+                                      int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream) {
+    if (!q_h || !k_h || !v_h || !out_h || !q_d || !k_d || !v_d || !out_d) return TLIN_ERR_INVALID_ARG;
+    if (lse_h && !lse_d) return TLIN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || N <= 0 || W <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t qb = (size_t)B * H * W * d * 2, kb = (size_t)B * H * N * d * 2;
+    TLIN_CUDA_CHECK(cudaMemcpyAsync(q_d, q_h, qb, cudaMemcpyHostToDevice, st));
+    TLIN_CUDA_CHECK(cudaMemcpyAsync(k_d, k_h, kb, cudaMemcpyHostToDevice, st));
+    TLIN_CUDA_CHECK(cudaMemcpyAsync(v_d, v_h, kb, cudaMemcpyHostToDevice, st));
+    const int rc = forward_common(q_d, k_d, v_d, out_d, lse_d, B, H, N, W, d, causal_window, 0, st);
+    if (rc != TLIN_OK) return rc;
+    TLIN_CUDA_CHECK(cudaMemcpyAsync(out_h, out_d, qb, cudaMemcpyDeviceToHost, st));
+    if (lse_h) TLIN_CUDA_CHECK(cudaMemcpyAsync(lse_h, lse_d, (size_t)B * H * W * sizeof(float), cudaMemcpyDeviceToHost, st));
+    return TLIN_OK;
+}
+
+extern "C" int tlin_decode_step(const void* q_new, const void* k_new, const void* v_new,
+                                void* k_cache, void* v_cache, void* out, float* lse,
+                                int B, int H, int Ncap, int pos, int d, tlin_stream_t stream) {
+    t_launches = 0;
+    if (!q_new || !k_new || !v_new || !k_cache || !v_cache || !out) return TLIN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || Ncap <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    if (pos < 0 || pos >= Ncap) return TLIN_ERR_INVALID_ARG;
+    if (!aligned16(q_new) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) ||
+        !aligned16(v_cache) || !aligned16(out)) return TLIN_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return TLIN_ERR_UNSUPPORTED;
+    int sms = 0;
+    int rc = device_info(&sms);
+    if (rc != TLIN_OK) return rc;
+    tlin_decode_plan plan;
+    rc = tlin_plan_decode(B, H, pos + 1, d, sms, &plan);
+    if (rc != TLIN_OK) return rc;
+    const Workspace w = workspace();
+    if (!w.ptr || w.bytes < (size_t)plan.workspace_bytes) return TLIN_ERR_WORKSPACE;
+    return launch_decode(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, d, plan,
+                         (float*)w.ptr, (cudaStream_t)stream);
+}
+
+extern "C" int tlin_decode_step_host(const void* q_new_h, const void* k_new_h, const void* v_new_h, void* out_h, float* lse_h,
+                                     void* q_new_d, void* k_new_d, void* v_new_d, void* out_d, float* lse_d,
+                                     void* k_cache, void* v_cache,
+                                     int B, int H, int Ncap, int pos, int d, tlin_stream_t stream) {
+    if (!q_new_h || !k_new_h || !v_new_h || !out_h || !q_new_d || !k_new_d || !v_new_d || !out_d) return TLIN_ERR_INVALID_ARG;
+    if (lse_h && !lse_d) return TLIN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t nb = (size_t)B * H * d * 2;
+    TLIN_CUDA_CHECK(cudaMemcpyAsync(q_new_d, q_new_h, nb, cudaMemcpyHostToDevice, st));
+    TLIN_CUDA_CHECK(cudaMemcpyAsync(k_new_d, k_new_h, nb, cudaMemcpyHostToDevice, st));
+    TLIN_CUDA_CHECK(cudaMemcpyAsync(v_new_d, v_new_h, nb, cudaMemcpyHostToDevice, st));
+    const int rc = tlin_decode_step(q_new_d, k_new_d, v_new_d, k_cache, v_cache, out_d, lse_d, B, H, Ncap, pos, d, stream);
+    if (rc != TLIN_OK) return rc;
+    TLIN_CUDA_CHECK(cudaMemcpyAsync(out_h, out_d, nb, cudaMemcpyDeviceToHost, st));
+    if (lse_h) TLIN_CUDA_CHECK(cudaMemcpyAsync(lse_h, lse_d, (size_t)B * H * sizeof(float), cudaMemcpyDeviceToHost, st));
+    return TLIN_OK;
+}
+
+static int merge_common(const void* oa, const float* la, const void* ob, const float* lb, void* out, float* lse,
+                        int64_t rows, int d, int is_f32, cudaStream_t st) {
+    t_launches = 0;
+    if (!oa || !la || !ob || !lb || !out) return TLIN_ERR_INVALID_ARG;
+    if (rows < 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    int sms = 0;
+    const int rc = device_info(&sms);
+    if (rc != TLIN_OK) return rc;
+    return is_f32 ? launch_merge_pair_f32((const float*)oa, la, (const float*)ob, lb, (float*)out, lse, rows, d, st)
+                  : launch_merge_pair_bf16(oa, la, ob, lb, out, lse, rows, d, st);
+}
+
+extern "C" int tlin_merge_lse(const void* out_a, const float* lse_a, const void* out_b, const float* lse_b,
+                              void* out, float* lse, int64_t rows, int d, tlin_stream_t stream) {
+    return merge_common(out_a, lse_a, out_b, lse_b, out, lse, rows, d, 0, (cudaStream_t)stream);
+}
+extern "C" int tlin_merge_lse_f32(const float* out_a, const float* lse_a, const float* out_b, const float* lse_b,
+                                  float* out, float* lse, int64_t rows, int d, tlin_stream_t stream) {
+    return merge_common(out_a, lse_a, out_b, lse_b, out, lse, rows, d, 1, (cudaStream_t)stream);
+}
+
+extern "C" int tlin_set_workspace(void* dev_ptr, size_t bytes) {
+    if ((dev_ptr == nullptr) != (bytes == 0)) return TLIN_ERR_INVALID_ARG;
+    if (!aligned16(dev_ptr)) return TLIN_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_ws.ptr = dev_ptr;
+    g_ws.bytes = bytes;
+    return TLIN_OK;
+}
+
+extern "C" int tlin_get_status(tlin_stream_t stream) {
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return TLIN_ERR_CUDA;
+    int* p = status_word();
+    if (!p) return TLIN_ERR_CUDA;
+    int h = 0;
+    if (cudaMemcpy(&h, p, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return TLIN_ERR_CUDA;
+    if (h != 0) {
+        const int zero = 0;
+        if (cudaMemcpy(p, &zero, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return TLIN_ERR_CUDA;
+    }
+    return h;
+}
+
+extern "C" const char* tlin_status_string(int status) {
+    switch (status) {
+        case TLIN_OK: return "ok";
+        case TLIN_ERR_INVALID_ARG: return "invalid argument";
+        case TLIN_ERR_UNSUPPORTED: return "unsupported shape";
+        case TLIN_ERR_WORKSPACE: return "workspace missing or too small";
+        case TLIN_ERR_CUDA: return "CUDA call failed";
+        case TLIN_ERR_TIMEOUT: return "device-side wait timed out";
+        case TLIN_ERR_ARCH: return "device is not compute capability 10.x";
+        default: return "unknown status";
+    }
+}
+
+extern "C" const char* tlin_version(void) { return "libtlin 0.1 (sm_100a)"; }
+
+extern "C" int tlin_set_forward_impl(int impl) {
+    if (impl < 0 || impl > 2) return TLIN_ERR_INVALID_ARG;
+    return g_impl.exchange(impl);
+}
+
+extern "C" int tlin_last_launch_count(void) { return t_launches; }

@@ -1,0 +1,230 @@
+// Cached decode step: append the new key/value row, then one query row per (b,h) over the whole
+// cache.  Appendix A ("Cache Hit": only the newest token takes part) and Section 5.2 (the history
+// cache is static; nothing is re-concatenated).  Pure HBM streaming: every cached K/V byte is read
+// exactly once with 16-byte loads, CUDA cores do the arithmetic in fp32.
+//
+// Grid: (b,h) x splits.  Split s owns keys [s*kps, min(L,(s+1)*kps)), L = pos+1.  Inside a CTA
+// each warp-load covers 512 contiguous bytes (32/LPR rows); the LPR lanes that share a row reduce
+// their partial dot products with xor-shuffles.  Every row-group keeps its own running max/sum and
+// they are combined at the end; the CTA writes one normalised partial (o, lse) to the workspace and
+// a second kernel merges the splits (log-sum-exp weights).
+#include "tlin_internal.h"
+#include <math_constants.h>
+
+namespace tlin {
+namespace {
+
+constexpr int kWarps = 8;
+constexpr int kUnroll = 4;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+__device__ __forceinline__ float dot8(const uint4& kv, const float (&qf)[8]) {
+    float s = bf_lo(kv.x) * qf[0];
+    s = fmaf(bf_hi(kv.x), qf[1], s);
+    s = fmaf(bf_lo(kv.y), qf[2], s);
+    s = fmaf(bf_hi(kv.y), qf[3], s);
+    s = fmaf(bf_lo(kv.z), qf[4], s);
+    s = fmaf(bf_hi(kv.z), qf[5], s);
+    s = fmaf(bf_lo(kv.w), qf[6], s);
+    s = fmaf(bf_hi(kv.w), qf[7], s);
+    return s;
+}
+__device__ __forceinline__ void axpy8(float p, const uint4& vv, float (&acc)[8]) {
+    acc[0] = fmaf(p, bf_lo(vv.x), acc[0]);
+    acc[1] = fmaf(p, bf_hi(vv.x), acc[1]);
+    acc[2] = fmaf(p, bf_lo(vv.y), acc[2]);
+    acc[3] = fmaf(p, bf_hi(vv.y), acc[3]);
+    acc[4] = fmaf(p, bf_lo(vv.z), acc[4]);
+    acc[5] = fmaf(p, bf_hi(vv.z), acc[5]);
+    acc[6] = fmaf(p, bf_lo(vv.w), acc[6]);
+    acc[7] = fmaf(p, bf_hi(vv.w), acc[7]);
+}
+
+// merge (m2,l2,a2) into (m,l,a); both in log2 units
+__device__ __forceinline__ void combine(float& m, float& l, float (&a)[8], float m2, float l2, const float (&a2)[8]) {
+    const float mn = fmaxf(m, m2);
+    const float ms = mn == -CUDART_INF_F ? 0.f : mn;
+    const float c1 = exp2f(m - ms), c2 = exp2f(m2 - ms);
+    l = l * c1 + l2 * c2;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) a[e] = a[e] * c1 + a2[e] * c2;
+    m = mn;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kWarps * 32, kDecodeCtasPerSM)
+decode_splitk_kernel(const uint4* __restrict__ q_new, const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+                     uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
+                     float* __restrict__ part_o, float* __restrict__ part_lse,
+                     int Ncap, int pos, int splits, int kps, float scale_log2e) {
+    constexpr int LPR = D / 8;           // lanes (16-byte chunks) per row
+    constexpr int RPW = 32 / LPR;        // rows per warp-load
+    constexpr int ROWS_PER_IT = kWarps * RPW * kUnroll;
+    const int bh = blockIdx.x / splits, sp = blockIdx.x - bh * splits;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane % LPR, rsel = lane / LPR;
+    const int L = pos + 1;
+    const int j0 = sp * kps, j1 = min(L, j0 + kps);
+
+    const uint4* kc = k_cache + (int64_t)bh * Ncap * LPR;
+    const uint4* vc = v_cache + (int64_t)bh * Ncap * LPR;
+    const uint4* kn = k_new + (int64_t)bh * LPR;
+    const uint4* vn = v_new + (int64_t)bh * LPR;
+
+    // append (bit-exact copy) by the CTA whose range holds row `pos`; nobody reads that row from the
+    // cache in this launch -- the lanes below take it from k_new / v_new.
+    if (pos >= j0 && pos < j1 && warp == 0 && lane < LPR) {
+        k_cache[((int64_t)bh * Ncap + pos) * LPR + lane] = kn[lane];
+        v_cache[((int64_t)bh * Ncap + pos) * LPR + lane] = vn[lane];
+    }
+
+    float qf[8];
+    {
+        const uint4 qv = q_new[(int64_t)bh * LPR + sub];
+        qf[0] = bf_lo(qv.x) * scale_log2e; qf[1] = bf_hi(qv.x) * scale_log2e;
+        qf[2] = bf_lo(qv.y) * scale_log2e; qf[3] = bf_hi(qv.y) * scale_log2e;
+        qf[4] = bf_lo(qv.z) * scale_log2e; qf[5] = bf_hi(qv.z) * scale_log2e;
+        qf[6] = bf_lo(qv.w) * scale_log2e; qf[7] = bf_hi(qv.w) * scale_log2e;
+    }
+
+    float m = -CUDART_INF_F, l = 0.f;
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+
+    for (int base = j0; base < j1; base += ROWS_PER_IT) {
+        uint4 kv[kUnroll], vv[kUnroll];
+        bool ok[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int j = base + (u * kWarps + warp) * RPW + rsel;
+            ok[u] = j < j1;
+            kv[u] = make_uint4(0, 0, 0, 0);
+            vv[u] = make_uint4(0, 0, 0, 0);
+            if (ok[u]) {
+                const bool fresh = j == pos;
+                const uint4* kp = fresh ? kn + sub : kc + (int64_t)j * LPR + sub;
+                const uint4* vp = fresh ? vn + sub : vc + (int64_t)j * LPR + sub;
+                kv[u] = ld_stream(kp);
+                vv[u] = ld_stream(vp);
+            }
+        }
+        float s[kUnroll];
+        float mb = m;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            float x = dot8(kv[u], qf);
+#pragma unroll
+            for (int o = LPR / 2; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+            s[u] = ok[u] ? x : -CUDART_INF_F;
+            mb = fmaxf(mb, s[u]);
+        }
+        const float ms = mb == -CUDART_INF_F ? 0.f : mb;
+        const float corr = exp2f(m - ms);
+        l *= corr;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] *= corr;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const float p = exp2f(s[u] - ms);
+            l += p;
+            axpy8(p, vv[u], acc);
+        }
+        m = mb;
+    }
+
+    // combine the row-groups of the warp
+#pragma unroll
+    for (int o = LPR; o < 32; o <<= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
+        const float l2 = __shfl_xor_sync(0xffffffffu, l, o);
+        float a2[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) a2[e] = __shfl_xor_sync(0xffffffffu, acc[e], o);
+        combine(m, l, acc, m2, l2, a2);
+    }
+    __shared__ float sm_m[kWarps], sm_l[kWarps];
+    __shared__ float sm_a[kWarps][D];
+    if (rsel == 0) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sm_a[warp][sub * 8 + e] = acc[e];
+        if (sub == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+    }
+    __syncthreads();
+    if (threadIdx.x < D) {
+        const int c = threadIdx.x;
+        float mm = -CUDART_INF_F;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) mm = fmaxf(mm, sm_m[w]);
+        const float ms = mm == -CUDART_INF_F ? 0.f : mm;
+        float ll = 0.f, a = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const float c1 = exp2f(sm_m[w] - ms);
+            ll += sm_l[w] * c1;
+            a += sm_a[w][c] * c1;
+        }
+        const int64_t slot = (int64_t)bh * splits + sp;
+        part_o[slot * D + c] = ll > 0.f ? a / ll : 0.f;
+        if (c == 0) part_lse[slot] = ll > 0.f ? (mm + log2f(ll)) * kLn2 : -CUDART_INF_F;
+    }
+}
+
+// One CTA per (b,h): out = sum_s w_s o_s / sum_s w_s with w_s = exp(lse_s - max lse).
+template <int D>
+__global__ void __launch_bounds__(D)
+decode_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse,
+                    __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int splits) {
+    const int bh = blockIdx.x, c = threadIdx.x;
+    const float* pl = part_lse + (int64_t)bh * splits;
+    float mm = -CUDART_INF_F;
+    for (int s = 0; s < splits; ++s) mm = fmaxf(mm, pl[s]);
+    float z = 0.f, a = 0.f;
+    for (int s = 0; s < splits; ++s) {
+        const float w = expf(pl[s] - mm);
+        z += w;
+        a = fmaf(w, part_o[((int64_t)bh * splits + s) * D + c], a);
+    }
+    out[(int64_t)bh * D + c] = __float2bfloat16_rn(a / z);
+    if (lse != nullptr && c == 0) lse[bh] = mm + logf(z);
+}
+
+template <int D>
+int launch_d(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+             void* out, float* lse, int B, int H, int Ncap, int pos, const tlin_decode_plan& plan,
+             float* ws, cudaStream_t st) {
+    const int64_t bh = (int64_t)B * H;
+    float* part_o = ws;
+    float* part_lse = ws + bh * kDecodeMaxSplits * D;
+    const float scale_log2e = kLog2e / sqrtf((float)D);
+    decode_splitk_kernel<D><<<plan.n_ctas, kWarps * 32, 0, st>>>(
+        (const uint4*)q_new, (const uint4*)k_new, (const uint4*)v_new, (uint4*)k_cache, (uint4*)v_cache,
+        part_o, part_lse, Ncap, pos, plan.splits, plan.keys_per_split, scale_log2e);
+    TLIN_CUDA_CHECK(cudaGetLastError());
+    decode_merge_kernel<D><<<(unsigned)bh, D, 0, st>>>(part_o, part_lse, (__nv_bfloat16*)out, lse, plan.splits);
+    TLIN_CUDA_CHECK(cudaGetLastError());
+    count_launch(2);
+    return TLIN_OK;
+}
+
+}  // namespace
+
+int launch_decode(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                  void* out, float* lse, int B, int H, int Ncap, int pos, int d,
+                  const tlin_decode_plan& plan, float* ws, cudaStream_t st) {
+    if (d == 128) return launch_d<128>(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, plan, ws, st);
+    if (d == 64) return launch_d<64>(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, plan, ws, st);
+    return TLIN_ERR_UNSUPPORTED;
+}
+
+}  // namespace tlin

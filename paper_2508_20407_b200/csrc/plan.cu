@@ -1,0 +1,124 @@
+// Host-side planning: pure integer arithmetic, no CUDA calls.  The paper does not schedule
+// anything; what it fixes is the set of (query,key) pairs a call evaluates (Section 3, causal
+// rule; Appendix A, cost terms), and every function here is tested against that count.
+#include "tlin_internal.h"
+
+using namespace tlin;
+
+extern "C" int tlin_allowed(int64_t i, int64_t j, int64_t N, int64_t W, int causal_window) {
+    if (i < 0 || i >= W || j < 0 || j >= N) return 0;
+    if (causal_window) return j <= (N - W) + i ? 1 : 0;
+    return 1;
+}
+
+extern "C" int tlin_tile_class(int64_t N, int64_t W, int causal_window, int tile_m, int tile_n, int qt, int kt) {
+    if (tile_m <= 0 || tile_n <= 0 || qt < 0 || kt < 0) return 0;
+    const int64_t i0 = (int64_t)qt * tile_m, j0 = (int64_t)kt * tile_n;
+    if (i0 >= W || j0 >= N) return 0;
+    const int64_t i1 = (i0 + tile_m < W ? i0 + tile_m : W) - 1;   // last query row of the tile
+    const int64_t j1 = j0 + tile_n - 1;                           // last key column, may lie beyond N
+    if (causal_window) {
+        if (j0 > (N - W) + i1) return 0;                          // even the last row sees nothing
+        if (j1 < N && j1 <= (N - W) + i0) return 1;               // even the first row sees everything
+        return 2;
+    }
+    return j1 < N ? 1 : 2;
+}
+
+extern "C" int64_t tlin_plan_group_start(const tlin_fwd_plan* plan, int g) {
+    if (!plan || plan->n_groups <= 0) return 0;
+    if (g <= 0) return 0;
+    if (g >= plan->n_groups) return plan->total_units;
+    // total_units < 2^31 * 2^24 / n_groups bound: B*H*key_tiles fits comfortably in 63 bits after *g
+    return (int64_t)(((__int128)g * plan->total_units) / plan->n_groups);
+}
+
+extern "C" int tlin_plan_forward(int B, int H, int N, int W, int d, int causal_window, int is_f32,
+                                 int num_sms, tlin_fwd_plan* plan) {
+    if (!plan) return TLIN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || N <= 0 || W <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    if (causal_window && N < W) return TLIN_ERR_INVALID_ARG;
+    if (num_sms <= 0) num_sms = kDefaultSMs;
+    const int impl = forward_impl();
+    const bool tc_shape = !is_f32 && (d == 64 || d == 128);
+    if (impl == 2 && !tc_shape) return TLIN_ERR_UNSUPPORTED;
+    if (is_f32 ? (d % 4 != 0 || d > 256) : (d % 8 != 0 || d > 256)) return TLIN_ERR_UNSUPPORTED;
+    const bool tc = tc_shape && impl == 2;  // automatic = CUDA-core kernel until the tensor path is enabled
+    tlin_fwd_plan p = {};
+    const int64_t bh = (int64_t)B * H;
+    p.tensor_path = tc ? 1 : 0;
+    if (!tc) {
+        p.tile_m = kSimtRows;
+        p.tile_n = kSimtKeys;
+        p.q_tiles = (W + p.tile_m - 1) / p.tile_m;
+        p.key_tiles = (N + p.tile_n - 1) / p.tile_n;
+        p.total_units = bh * p.key_tiles;
+        p.n_groups = (int32_t)(bh < INT32_MAX ? bh : INT32_MAX);   // one group per (b,h): never split
+        if ((int64_t)p.n_groups * p.q_tiles > INT32_MAX) return TLIN_ERR_UNSUPPORTED;
+        p.n_ctas = p.n_groups * p.q_tiles;
+        p.uses_workspace = 0;
+        p.workspace_bytes = 0;
+        *plan = p;
+        return TLIN_OK;
+    }
+    p.tile_m = 128;
+    p.tile_n = kTileN;
+    p.q_tiles = (W + p.tile_m - 1) / p.tile_m;
+    p.key_tiles = (N + p.tile_n - 1) / p.tile_n;
+    p.total_units = bh * p.key_tiles;
+    int64_t groups = num_sms / p.q_tiles;
+    if (groups < 1) groups = 1;
+    if (groups > p.total_units) groups = p.total_units;
+    p.n_groups = (int32_t)groups;
+    p.n_ctas = p.n_groups * p.q_tiles;
+    p.uses_workspace = 0;
+    for (int g = 1; g < p.n_groups; ++g)
+        if (tlin_plan_group_start(&p, g) % p.key_tiles != 0) { p.uses_workspace = 1; break; }
+    // two partial slots per CTA (first and last segment of its unit range), each tile_m x (d + 1) floats
+    p.workspace_bytes = p.uses_workspace ? (int64_t)p.n_ctas * 2 * p.tile_m * (d + 1) * (int64_t)sizeof(float) : 0;
+    *plan = p;
+    return TLIN_OK;
+}
+
+extern "C" int tlin_plan_decode(int B, int H, int L, int d, int num_sms, tlin_decode_plan* plan) {
+    if (!plan) return TLIN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || L <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    if (num_sms <= 0) num_sms = kDefaultSMs;
+    const int64_t bh = (int64_t)B * H;
+    const int64_t slots = (int64_t)num_sms * kDecodeCtasPerSM;
+    int max_s = (L + kDecodeMinKeys - 1) / kDecodeMinKeys;
+    if (max_s > kDecodeMaxSplits) max_s = kDecodeMaxSplits;
+    if (max_s < 1) max_s = 1;
+    int best_s = 1;
+    int64_t best_cost = -1;
+    for (int s = 1; s <= max_s; ++s) {
+        int64_t kps = (L + s - 1) / s;
+        kps = (kps + 7) / 8 * 8;
+        const int64_t waves = (bh * s + slots - 1) / slots;
+        const int64_t cost = waves * (kps + 64);   // + a fixed per-CTA overhead, in keys
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_s = s; }
+    }
+    tlin_decode_plan p = {};
+    int64_t kps = (L + best_s - 1) / best_s;
+    kps = (kps + 7) / 8 * 8;
+    p.keys_per_split = (int32_t)kps;
+    p.splits = (int32_t)((L + kps - 1) / kps);     // drop splits that rounding left empty
+    if (bh * p.splits > INT32_MAX) return TLIN_ERR_UNSUPPORTED;
+    p.n_ctas = (int32_t)(bh * p.splits);
+    p.workspace_bytes = bh * kDecodeMaxSplits * (int64_t)(d + 1) * (int64_t)sizeof(float);
+    *plan = p;
+    return TLIN_OK;
+}
+
+extern "C" size_t tlin_workspace_bytes_forward(int B, int H, int N, int W, int d, int causal_window) {
+    tlin_fwd_plan p;
+    if (tlin_plan_forward(B, H, N, W, d, causal_window, 0, 0, &p) != TLIN_OK) return 0;
+    // sized for a 148-SM part; a device with another SM count is re-planned and re-checked at call time
+    return (size_t)p.workspace_bytes;
+}
+
+extern "C" size_t tlin_workspace_bytes_decode(int B, int H, int Ncap, int d) {
+    tlin_decode_plan p;
+    if (tlin_plan_decode(B, H, Ncap > 0 ? Ncap : 1, d, 0, &p) != TLIN_OK) return 0;
+    return (size_t)p.workspace_bytes;
+}

@@ -1,0 +1,51 @@
+// Internal declarations shared by the translation units of libtlin (never installed).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stdio.h>
+#include "../../include/tlin.h"
+
+namespace tlin {
+
+constexpr int kDefaultSMs = 148;       // B200
+constexpr int kTileN = 128;            // keys per tile on the tensor path
+constexpr int kSimtRows = 8;           // query rows per CTA on the CUDA-core path
+constexpr int kSimtKeys = 32;          // keys per staged tile on the CUDA-core path
+constexpr int kDecodeMaxSplits = 64;   // upper bound on CTAs per (b,h) in the decode step
+constexpr int kDecodeMinKeys = 256;    // do not split the cache finer than this
+constexpr int kDecodeCtasPerSM = 2;
+
+struct Workspace { void* ptr; size_t bytes; };
+Workspace workspace();
+int* status_word();                    // device address of the error word (bounded waits report here)
+void count_launch(int n = 1);
+int forward_impl();
+
+#define TLIN_CUDA_CHECK(expr)                                                              \
+    do {                                                                                   \
+        cudaError_t e__ = (expr);                                                          \
+        if (e__ != cudaSuccess) {                                                          \
+            fprintf(stderr, "libtlin: %s failed: %s (%s:%d)\n", #expr,                     \
+                    cudaGetErrorString(e__), __FILE__, __LINE__);                          \
+            return TLIN_ERR_CUDA;                                                          \
+        }                                                                                  \
+    } while (0)
+
+// ---- launchers (one per kernel family); all validate nothing: api.cu has done it ----------
+int launch_fwd_simt_bf16(const void* q, const void* k, const void* v, void* out, float* lse,
+                         int B, int H, int N, int W, int d, int causal, cudaStream_t st);
+int launch_fwd_simt_f32(const float* q, const float* k, const float* v, float* out, float* lse,
+                        int B, int H, int N, int W, int d, int causal, cudaStream_t st);
+int launch_fwd_tc(const void* q, const void* k, const void* v, void* out, float* lse,
+                  int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& plan,
+                  float* ws, cudaStream_t st);
+int launch_decode(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                  void* out, float* lse, int B, int H, int Ncap, int pos, int d,
+                  const tlin_decode_plan& plan, float* ws, cudaStream_t st);
+int launch_merge_pair_bf16(const void* oa, const float* la, const void* ob, const float* lb,
+                           void* out, float* lse, int64_t rows, int d, cudaStream_t st);
+int launch_merge_pair_f32(const float* oa, const float* la, const float* ob, const float* lb,
+                          float* out, float* lse, int64_t rows, int d, cudaStream_t st);
+
+}  // namespace tlin

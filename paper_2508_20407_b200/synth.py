@@ -183,3 +183,27 @@ def decode_inputs(wl: Workload, device="cpu", dtype=torch.bfloat16, steps: int |
     k_new = normal_tensor(wl.seed, KNEW_ID, shp, dtype, device, wl.scale)
     v_new = normal_tensor(wl.seed, VNEW_ID, shp, dtype, device, wl.scale)
     return (k_cache, v_cache), (q_new, k_new, v_new)
+
+
+def forward_inputs_head(wl: Workload, b: int, h: int, device="cpu", dtype=torch.bfloat16, q_rows: slice | None = None):
+    """The (b,h) slice of ``forward_inputs(wl)``: (q [W',d], k [N,d], v [N,d]), made without the rest.
+
+    Uses the same counters as the full tensors, so the values agree with a slice of them (up to the
+    host/device libm note in the module docstring).
+    """
+    bh = b * wl.H + h
+    r0, r1 = (0, wl.W) if q_rows is None else (q_rows.start or 0, wl.W if q_rows.stop is None else q_rows.stop)
+
+    def rows(tid, first_row, n_rows, peaky):
+        x = normal_flat(wl.seed, tid, first_row * wl.d, n_rows * wl.d, device=device)
+        if wl.scale != 1.0:
+            x = x * wl.scale
+        if peaky is not None:
+            hit = row_hash_mod(wl.seed, tid, first_row, n_rows, peaky[0], device=device) == 0
+            x = (x.view(n_rows, wl.d) * torch.where(hit, float(peaky[1]), 1.0).to(torch.float64)[:, None]).reshape(-1)
+        return x.to(dtype).view(n_rows, wl.d)
+
+    q = rows(Q_ID, bh * wl.W + r0, r1 - r0, None)
+    k = rows(K_ID, bh * wl.N, wl.N, wl.peaky)
+    v = rows(V_ID, bh * wl.N, wl.N, None)
+    return q, k, v

@@ -1,0 +1,139 @@
+"""CPU-side tests of the C-ABI library: it loads without a GPU, exports every symbol the header
+declares, rejects bad arguments before touching a device, and its integer planning is exact."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import cost_model
+from paper_2508_20407_b200 import binding as tl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "tlin.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(tlin_[a-z0-9_]+)\s*\(", header))
+    assert len(declared) >= 18
+    raw = ctypes.CDLL(tl.LIB_PATH)
+    for name in declared:
+        assert hasattr(raw, name), f"{name} is declared in tlin.h but not exported"
+    assert declared == set(tl.SIGNATURES), declared ^ set(tl.SIGNATURES)
+
+
+def test_version_and_status_strings():
+    assert "sm_100a" in tl.version()
+    assert tl.status_string(0) == "ok"
+    for s in range(-6, 0):
+        assert tl.status_string(s) not in ("ok", "unknown status")
+
+
+def test_argument_errors_are_found_on_the_host():
+    L = tl.lib()
+    one = ctypes.c_void_p(16)  # aligned, never dereferenced: every call below fails validation first
+    odd = ctypes.c_void_p(24 + 2)
+    fwd = lambda *a: L.tlin_attn_forward(*a, None)
+    assert fwd(None, one, one, one, one, 1, 1, 8, 4, 64, 1) == tl.ERR_INVALID_ARG
+    assert fwd(one, one, one, one, one, 0, 1, 8, 4, 64, 1) == tl.ERR_INVALID_ARG
+    assert fwd(one, one, one, one, one, 1, 1, 4, 8, 64, 1) == tl.ERR_INVALID_ARG      # N < W with a window
+    assert fwd(odd, one, one, one, one, 1, 1, 8, 4, 64, 1) == tl.ERR_INVALID_ARG      # misaligned
+    assert fwd(one, one, one, one, one, 1, 1, 8, 4, 64, 2) == tl.ERR_INVALID_ARG      # causal flag
+    assert fwd(one, one, one, one, one, 1, 1, 8, 4, 36, 1) == tl.ERR_UNSUPPORTED      # bf16 path needs d % 8 == 0
+    assert L.tlin_attn_forward_f32(one, one, one, one, one, 1, 1, 8, 4, 258, 1, None) == tl.ERR_UNSUPPORTED
+    dec = lambda *a: L.tlin_decode_step(*a, None)
+    assert dec(one, one, one, one, one, one, one, 1, 1, 8, -1, 64) == tl.ERR_INVALID_ARG
+    assert dec(one, one, one, one, one, one, one, 1, 1, 8, 8, 64) == tl.ERR_INVALID_ARG
+    assert dec(one, one, one, one, one, one, one, 1, 1, 8, 3, 48) == tl.ERR_UNSUPPORTED
+    assert L.tlin_set_workspace(None, 16) == tl.ERR_INVALID_ARG
+    assert L.tlin_set_forward_impl(7) == tl.ERR_INVALID_ARG
+
+
+def test_mask_predicate_matches_the_causal_rule_bit_for_bit():
+    for N in range(1, 10):
+        for W in range(1, N + 1):
+            for i in range(W):
+                for j in range(-1, N + 1):
+                    assert tl.tlin_allowed(i, j, N, W, 1) == int(0 <= j < N and j <= N - W + i)
+                    assert tl.tlin_allowed(i, j, N, W, 0) == int(0 <= j < N)
+
+
+@pytest.mark.parametrize("N,W,causal,tm,tn", [(1000, 300, 1, 128, 128), (512, 512, 1, 128, 128), (777, 130, 0, 128, 128),
+                                              (1024, 128, 1, 128, 128), (300, 7, 1, 8, 32), (4096, 256, 1, 256, 128)])
+def test_tile_classes_against_brute_force_and_pair_count(N, W, causal, tm, tn):
+    i = np.arange(W)[:, None]
+    j = np.arange(((N + tn - 1) // tn) * tn)[None, :]
+    allowed = (j < N) & ((j <= N - W + i) if causal else (i >= 0))
+    total = 0
+    for qt in range((W + tm - 1) // tm):
+        for kt in range((N + tn - 1) // tn):
+            blk = allowed[qt * tm:(qt + 1) * tm, kt * tn:(kt + 1) * tn]
+            cls = tl.tlin_tile_class(N, W, causal, tm, tn, qt, kt)
+            if cls == 0:
+                assert not blk.any()
+            elif cls == 1:
+                assert blk.all() and blk.shape[1] == tn
+            else:
+                assert cls == 2 and blk.any() and not (blk.all() and blk.shape[1] == tn)
+            if cls:
+                total += int(blk.sum())
+    # the pairs the planned tiles cover are exactly the pairs the method evaluates
+    assert total == cost_model.allowed_pairs(N, W, causal)
+
+
+CONFIGS = [(1, 4, 1024, 128, 64, 1), (4, 16, 8192, 256, 64, 1), (1, 32, 32768, 512, 128, 1),
+           (1, 32, 131072, 1024, 128, 1), (3, 5, 1000, 77, 128, 0), (1, 1, 100, 100, 64, 1), (2, 2, 129, 1, 64, 1)]
+
+
+@pytest.mark.parametrize("B,H,N,W,d,causal", CONFIGS)
+def test_forward_plan_partitions_the_units(B, H, N, W, d, causal):
+    prev = tl.tlin_set_forward_impl(2)
+    try:
+        p = tl.tlin_plan_forward(B, H, N, W, d, causal, num_sms=148)
+    finally:
+        tl.tlin_set_forward_impl(prev)
+    assert p.tensor_path == 1 and p.tile_n == 128
+    assert p.q_tiles == -(-W // p.tile_m) and p.key_tiles == -(-N // p.tile_n)
+    assert p.total_units == B * H * p.key_tiles
+    assert 1 <= p.n_groups <= p.total_units and p.n_ctas == p.n_groups * p.q_tiles
+    assert p.n_ctas <= 148 or p.n_groups == 1
+    starts = [tl.tlin_plan_group_start(p, g) for g in range(p.n_groups + 1)]
+    assert starts[0] == 0 and starts[-1] == p.total_units
+    sizes = np.diff(starts)
+    assert (sizes >= 1).all() and sizes.max() - sizes.min() <= 1
+    split = any(s % p.key_tiles for s in starts[1:-1])
+    assert bool(p.uses_workspace) == split
+    assert p.workspace_bytes == (p.n_ctas * 2 * p.tile_m * (d + 1) * 4 if split else 0)
+    assert tl.workspace_bytes_forward(B, H, N, W, d, causal) in (0, p.workspace_bytes) or tl.tlin_set_forward_impl(0) == 0
+
+
+def test_forward_plan_fallback_path_never_splits():
+    p = tl.tlin_plan_forward(2, 3, 500, 50, 36, 1, is_f32=True)
+    assert p.tensor_path == 0 and p.uses_workspace == 0 and p.workspace_bytes == 0
+    assert p.tile_m == 8 and p.n_ctas == 6 * 7
+
+
+@pytest.mark.parametrize("B,H,L,d", [(8, 32, 65537, 128), (8, 32, 65792, 128), (1, 1, 1, 64), (1, 4, 300, 64),
+                                     (2, 2, 100000, 128), (64, 32, 4096, 128)])
+def test_decode_plan_covers_every_key_once(B, H, L, d):
+    p = tl.tlin_plan_decode(B, H, L, d, 148)
+    assert 1 <= p.splits <= 64 and p.keys_per_split % 8 == 0
+    assert p.n_ctas == B * H * p.splits
+    covered = 0
+    for s in range(p.splits):
+        lo, hi = s * p.keys_per_split, min(L, (s + 1) * p.keys_per_split)
+        assert hi > lo
+        covered += hi - lo
+    assert covered == L
+    assert p.workspace_bytes == B * H * 64 * (d + 1) * 4 == tl.workspace_bytes_decode(B, H, max(L, 1), d)
+    if L >= 2 * 256:
+        assert p.keys_per_split >= 256
+
+
+def test_decode_plan_balances_the_benchmark_shape():
+    p = tl.tlin_plan_decode(8, 32, 65537, 128, 148)
+    waves = -(-p.n_ctas // 296)
+    ideal = 65537 * 256 / 296
+    assert waves * p.keys_per_split <= 1.05 * ideal

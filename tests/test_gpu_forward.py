@@ -1,0 +1,191 @@
+"""GPU parity of the forward entry points against the CPU oracle (element by element on the same
+seeded inputs; sampled rows at the full benchmark sizes).  Everything goes through the C-ABI."""
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import parity
+from paper_2508_20407_b200 import binding as tl
+from paper_2508_20407_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def run_impl(impl, fn, *a, **kw):
+    prev = tl.tlin_set_forward_impl(impl)
+    try:
+        out = fn(*a, **kw)
+        torch.cuda.synchronize()
+        assert tl.tlin_get_status() == 0
+        assert tl.tlin_last_launch_count() >= 1
+        return out
+    finally:
+        tl.tlin_set_forward_impl(prev)
+
+
+def impls_for(d):
+    return [1, 2] if d in (64, 128) and TC_AVAILABLE else [1]
+
+
+def _tc_available():
+    try:
+        prev = tl.tlin_set_forward_impl(2)
+        try:
+            p = tl.tlin_plan_forward(1, 1, 128, 128, 64, 0)
+            if not torch.cuda.is_available():
+                return False
+            q = torch.zeros(1, 1, 128, 64, dtype=torch.bfloat16, device=DEV)
+            tl.tlin_attn_forward(q, q, q, causal_window=0)
+            torch.cuda.synchronize()
+            return bool(p.tensor_path)
+        finally:
+            tl.tlin_set_forward_impl(prev)
+    except tl.TlinError:
+        return False
+
+
+TC_AVAILABLE = _tc_available() if torch.cuda.is_available() else False
+
+
+def full_compare(wl, impl, kind="bf16", causal=None):
+    causal = wl.causal_window if causal is None else causal
+    dtype = torch.bfloat16 if kind == "bf16" else torch.float32
+    q, k, v = synth.forward_inputs(wl, device=DEV, dtype=dtype)
+    fn = tl.tlin_attn_forward if kind == "bf16" else tl.tlin_attn_forward_f32
+    out, lse = run_impl(impl, fn, q, k, v, causal_window=causal)
+    ref, ref_lse = oracle.attn_forward(q.cpu(), k.cpu(), v.cpu(), causal)
+    return parity.check(out.float().cpu().numpy(), lse.cpu().numpy(), ref, ref_lse, kind, f"{wl.name} impl={impl}")
+
+
+@pytest.mark.parametrize("impl", [0, 1, 2])
+def test_cfg1_tiny_elementwise(impl):
+    if impl == 2 and not TC_AVAILABLE:
+        pytest.skip("tensor path not built")
+    full_compare(synth.WORKLOADS["cfg1_tiny"], impl)
+
+
+SHAPES = [  # B, H, N, W, d, causal
+    (1, 1, 1, 1, 64, 1), (1, 2, 129, 1, 64, 1), (2, 1, 128, 128, 64, 1), (1, 2, 300, 300, 128, 1),
+    (1, 3, 1000, 77, 128, 1), (2, 2, 515, 130, 64, 0), (1, 2, 257, 255, 128, 0), (1, 1, 4096, 384, 128, 1),
+    (1, 2, 2049, 129, 64, 1), (1, 1, 100, 300, 128, 0), (1, 1, 640, 512, 128, 1), (3, 2, 1111, 200, 64, 1),
+]
+
+
+@pytest.mark.parametrize("B,H,N,W,d,causal", SHAPES)
+def test_awkward_shapes_bf16(B, H, N, W, d, causal):
+    wl = synth.Workload("shape", B, H, d, N, W, seed=100 + N + W, causal_window=causal)
+    for impl in impls_for(d):
+        full_compare(wl, impl)
+
+
+@pytest.mark.parametrize("B,H,N,W,d,causal", [(1, 2, 333, 40, 36, 1), (1, 1, 1024, 128, 64, 1), (2, 2, 200, 200, 128, 1),
+                                              (1, 2, 77, 5, 256, 0), (1, 1, 1, 1, 4, 1), (1, 1, 2000, 9, 100, 1)])
+def test_fp32_path(B, H, N, W, d, causal):
+    wl = synth.Workload("f32", B, H, d, N, W, seed=7 + d, causal_window=causal)
+    full_compare(wl, 0, kind="f32")
+
+
+def test_bf16_fallback_head_dims():
+    for d in (8, 72, 256):
+        full_compare(synth.Workload("odd_d", 1, 2, d, 300, 33, seed=d), 0)
+
+
+def test_peaky_keys_stress_rescaling():
+    wl = synth.Workload("peaky", 1, 2, 128, 3000, 256, seed=2, peaky=(100, 8.0))
+    for impl in impls_for(128):
+        full_compare(wl, impl)
+
+
+def test_future_tokens_do_not_change_earlier_rows():
+    wl = synth.Workload("causal_inv", 1, 2, 64, 700, 200, seed=11)
+    q, k, v = synth.forward_inputs(wl, device=DEV)
+    for impl in impls_for(64):
+        out0, lse0 = run_impl(impl, tl.tlin_attn_forward, q, k, v, causal_window=1)
+        i = 57
+        k2, v2 = k.clone(), v.clone()
+        k2[:, :, wl.N - wl.W + i + 1:] += 3.0
+        v2[:, :, wl.N - wl.W + i + 1:] -= 2.0
+        out1, lse1 = run_impl(impl, tl.tlin_attn_forward, q, k2, v2, causal_window=1)
+        assert torch.equal(out0[:, :, :i + 1], out1[:, :, :i + 1]) and torch.equal(lse0[:, :, :i + 1], lse1[:, :, :i + 1])
+        assert not torch.equal(out0[:, :, i + 1:], out1[:, :, i + 1:])
+
+
+def test_run_to_run_bitwise_determinism():
+    wl = synth.Workload("det", 2, 4, 128, 5000, 300, seed=12)
+    q, k, v = synth.forward_inputs(wl, device=DEV)
+    for impl in impls_for(128):
+        a, la = run_impl(impl, tl.tlin_attn_forward, q, k, v, causal_window=1)
+        b, lb = run_impl(impl, tl.tlin_attn_forward, q, k, v, causal_window=1)
+        assert torch.equal(a, b) and torch.equal(la, lb)
+
+
+def test_merge_joins_history_and_window_calls():
+    wl = synth.Workload("merge", 1, 2, 64, 900, 128, seed=13)
+    q, k, v = synth.forward_inputs(wl, device=DEV)
+    joint, joint_lse = tl.tlin_attn_forward(q, k, v, causal_window=1)
+    hist = wl.N - wl.W
+    oh, lh = tl.tlin_attn_forward(q, k[:, :, :hist].contiguous(), v[:, :, :hist].contiguous(), causal_window=0)
+    ow, lw = tl.tlin_attn_forward(q, k[:, :, hist:].contiguous(), v[:, :, hist:].contiguous(), causal_window=1)
+    out, lse = tl.tlin_merge_lse(oh, lh, ow, lw)
+    torch.cuda.synchronize()
+    ref, ref_lse = oracle.attn_forward(q.cpu(), k.cpu(), v.cpu(), 1)
+    parity.check(out.float().cpu().numpy(), lse.cpu().numpy(), ref, ref_lse, "bf16", "merge of two calls")
+    parity.check(joint.float().cpu().numpy(), joint_lse.cpu().numpy(), ref, ref_lse, "bf16", "joint call")
+    # fp32 merge against the oracle's merge on the same partials, empty side included
+    oa = torch.randn(50, 64, device=DEV)
+    ob = torch.randn(50, 64, device=DEV)
+    la = torch.randn(50, device=DEV) * 3
+    lb = torch.randn(50, device=DEV) * 3
+    lb[3] = float("-inf")
+    la[7] = float("-inf")
+    la[9] = lb[9] = float("-inf")
+    o, l = tl.tlin_merge_lse(oa, la, ob, lb)
+    torch.cuda.synchronize()
+    r, rl = oracle.merge_lse(oa.cpu().double().numpy(), la.cpu().double().numpy(), ob.cpu().double().numpy(), lb.cpu().double().numpy())
+    assert np.abs(o.cpu().numpy() - r).max() < 1e-5
+    fin = np.isfinite(rl)
+    assert np.abs(l.cpu().numpy()[fin] - rl[fin]).max() < 1e-5 and (l.cpu().numpy()[~fin] == -np.inf).all()
+
+
+def sampled_rows_compare(wl, impl, rows_per_head, heads, causal):
+    """Full-size run; the oracle recomputes sampled query rows one by one (row i alone over keys [0, limit))."""
+    q, k, v = synth.forward_inputs(wl, device=DEV)
+    out, lse = run_impl(impl, tl.tlin_attn_forward, q, k, v, causal_window=causal)
+    assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
+    rng = np.random.default_rng(wl.seed)
+    jobs = []
+    for (b, h) in heads:
+        kh, vh = k[b, h].cpu(), v[b, h].cpu()
+        rows = sorted(set([0, wl.W - 1] + [int(x) for x in rng.integers(0, wl.W, rows_per_head)]))
+        for i in rows:
+            limit = wl.N - wl.W + i + 1 if causal else wl.N
+            jobs.append((b, h, i, q[b, h, i].cpu().view(1, 1, 1, wl.d), kh[:limit].view(1, 1, limit, wl.d), vh[:limit].view(1, 1, limit, wl.d)))
+    with ThreadPoolExecutor(max_workers=8) as ex:
+        refs = list(ex.map(lambda j: oracle.attn_forward(j[3], j[4], j[5], 0), jobs))
+    got = np.stack([out[b, h, i].float().cpu().numpy() for (b, h, i, *_rest) in jobs])
+    got_lse = np.array([lse[b, h, i].item() for (b, h, i, *_rest) in jobs])
+    ref = np.stack([r[0].reshape(-1) for r in refs])
+    ref_lse = np.array([r[1].item() for r in refs])
+    return parity.check(got, got_lse, ref, ref_lse, "bf16", f"{wl.name} impl={impl} sampled rows")
+
+
+def test_cfg2_mid_sampled_heads_full_rows():
+    wl = synth.WORKLOADS["cfg2_mid"]
+    q, k, v = synth.forward_inputs(wl, device=DEV)
+    for impl in impls_for(wl.d):
+        out, lse = run_impl(impl, tl.tlin_attn_forward, q, k, v, causal_window=1)
+        for (b, h) in [(0, 0), (3, 15), (1, 7)]:
+            sl = lambda t: t[b:b + 1, h:h + 1].contiguous().cpu()
+            ref, ref_lse = oracle.attn_forward(sl(q), sl(k), sl(v), 1)
+            parity.check(sl(out).float().numpy(), sl(lse).numpy(), ref, ref_lse, "bf16", f"cfg2 head {(b, h)} impl={impl}")
+
+
+@pytest.mark.parametrize("name,causal", [("cfg3_long", 1), ("cfg3_long", 0), ("cfg4_vlong", 1)])
+def test_full_size_sampled_rows(name, causal):
+    wl = synth.WORKLOADS[name]
+    impl = 2 if TC_AVAILABLE else 1
+    sampled_rows_compare(wl, impl, 6, [(0, 0), (0, wl.H // 2), (0, wl.H - 1)], causal)
