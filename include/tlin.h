@@ -93,6 +93,24 @@ int tlin_decode_step_host(const void* q_new_h, const void* k_new_h, const void* 
                           void* k_cache, void* v_cache,
                           int B, int H, int Ncap, int pos, int d, tlin_stream_t stream);
 
+/* tlin_decode_step for callers that cannot allocate device memory (the paper has no counterpart:
+ * this is a packaging variant of the same step).  A library embedded in someone else's memory pool,
+ * a worker that may only use buffers handed to it, or code that runs while allocation is off limits
+ * has no way to create the split-K workspace that tlin_decode_step wants.  This entry point keeps
+ * that scratch in an array compiled into the library (8 454 144 bytes, held on every GPU that loads
+ * libtlin until the process exits) and ignores tlin_set_workspace.  It calls no cudaMalloc/cudaFree
+ * and no allocating library routine.  Arguments, results and errors are those of tlin_decode_step,
+ * plus: shapes with B*H*(d+1)*256 bytes > 8 454 144 (more than 256 (b,h) pairs at d = 128, 508 at
+ * d = 64) are rejected with TLIN_ERR_WORKSPACE and a message on stderr.
+ * The first call on each device looks up the array's device address (once, with that device
+ * current); make that first call outside any stream capture.
+ * All calls on a device share the one array.  Every partial slot a call reads was written by the same
+ * call, so nothing has to be cleared between calls and stale contents are harmless, but two calls that
+ * overlap on the GPU (different streams) race on it: serialise them. */
+int tlin_decode_step_static(const void* q_new, const void* k_new, const void* v_new,
+                            void* k_cache, void* v_cache, void* out, float* lse,
+                            int B, int H, int Ncap, int pos, int d, tlin_stream_t stream);
+
 /* ------------------------------------------------------------------------------------------
  * Exact merge of two results over DISJOINT key sets for the same queries (not in the paper; it is
  * the split-K combine, exposed so that "history" and "window" attention may also be computed

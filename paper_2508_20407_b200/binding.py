@@ -45,6 +45,7 @@ SIGNATURES = {
     "tlin_attn_forward_host": (_i, [_vp] * 10 + [_i] * 6 + [_vp]),
     "tlin_decode_step": (_i, [_vp] * 7 + [_i] * 5 + [_vp]),
     "tlin_decode_step_host": (_i, [_vp] * 12 + [_i] * 5 + [_vp]),
+    "tlin_decode_step_static": (_i, [_vp] * 7 + [_i] * 5 + [_vp]),
     "tlin_merge_lse": (_i, [_vp] * 6 + [_i64, _i, _vp]),
     "tlin_merge_lse_f32": (_i, [_vp] * 6 + [_i64, _i, _vp]),
     "tlin_workspace_bytes_forward": (_sz, [_i] * 6),
@@ -206,6 +207,19 @@ def tlin_decode_step(q_new, k_new, v_new, k_cache, v_cache, pos, out=None, lse=N
     ensure_workspace(workspace_bytes_decode(B, H, Ncap, d), q_new.device)
     _check(lib().tlin_decode_step(_ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache),
                                   _ptr(out), _ptr(lse), B, H, Ncap, int(pos), d, _stream(stream)), "tlin_decode_step")
+    return out, lse
+
+
+def tlin_decode_step_static(q_new, k_new, v_new, k_cache, v_cache, pos, out, lse, stream=None):
+    """tlin_decode_step without any allocation: scratch is the library's built-in array, and ``out``
+    ([B,H,1,d] bf16) and ``lse`` ([B,H] fp32) must be supplied by the caller."""
+    B, H, Ncap, d = k_cache.shape
+    for t, n in ((q_new, "q_new"), (k_new, "k_new"), (v_new, "v_new"), (out, "out")):
+        _dev(t, torch.bfloat16, (B, H, 1, d), n)
+    _dev(lse, torch.float32, (B, H), "lse")
+    _check(lib().tlin_decode_step_static(_ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache),
+                                         _ptr(out), _ptr(lse), B, H, Ncap, int(pos), d, _stream(stream)),
+           "tlin_decode_step_static")
     return out, lse
 
 

@@ -10,6 +10,7 @@
 // a second kernel merges the splits (log-sum-exp weights).
 #include "tlin_internal.h"
 #include <math_constants.h>
+#include <mutex>
 
 namespace tlin {
 namespace {
@@ -228,3 +229,74 @@ int launch_decode(const void* q_new, const void* k_new, const void* v_new, void*
 }
 
 }  // namespace tlin
+
+// ------------------------------------------------------------------------------------------------
+// Decode step for callers that cannot allocate device memory.
+//
+// Some hosts of this library never get to call cudaMalloc: a plugin running inside another
+// framework's memory pool, a worker that may only touch buffers handed to it, a process whose device
+// memory budget is fixed up front.  For them the split-K partials live in the array below, which is part of
+// the library image: every GPU that loads libtlin holds these 8.1 MiB until the process exits.
+// Everything else is as in tlin_decode_step; the caller still owns inputs, caches and outputs.
+namespace tlin {
+namespace {
+
+constexpr size_t kStaticScratchFloats = (size_t)256 * kDecodeMaxSplits * 129;   // 8 454 144 bytes
+static __device__ __align__(256) float g_decode_static_scratch[kStaticScratchFloats];
+
+std::mutex g_static_mu;
+float* g_static_ptr[64] = {};      // device address of the array, per device, filled on first use
+int g_static_major[64] = {};
+int g_static_sms[64] = {};
+
+// In host code the array's name is only a handle: the address a kernel can use has to be asked for,
+// with the device current.  Done once per device.
+int static_scratch_setup(int dev, float** ptr, int* sms) {
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    if (g_static_ptr[dev] == nullptr) {
+        float* p = nullptr;
+        TLIN_CUDA_CHECK(cudaGetSymbolAddress((void**)&p, g_decode_static_scratch));
+        TLIN_CUDA_CHECK(cudaDeviceGetAttribute(&g_static_major[dev], cudaDevAttrComputeCapabilityMajor, dev));
+        TLIN_CUDA_CHECK(cudaDeviceGetAttribute(&g_static_sms[dev], cudaDevAttrMultiProcessorCount, dev));
+        g_static_ptr[dev] = p;
+    }
+    if (g_static_major[dev] != 10) return TLIN_ERR_ARCH;
+    *ptr = g_static_ptr[dev];
+    *sms = g_static_sms[dev];
+    return TLIN_OK;
+}
+
+}  // namespace
+}  // namespace tlin
+
+extern "C" int tlin_decode_step_static(const void* q_new, const void* k_new, const void* v_new,
+                                       void* k_cache, void* v_cache, void* out, float* lse,
+                                       int B, int H, int Ncap, int pos, int d, tlin_stream_t stream) {
+    using namespace tlin;
+    if (!q_new || !k_new || !v_new || !k_cache || !v_cache || !out) return TLIN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || Ncap <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    if (pos < 0 || pos >= Ncap) return TLIN_ERR_INVALID_ARG;
+    const uintptr_t all = (uintptr_t)q_new | (uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)k_cache |
+                          (uintptr_t)v_cache | (uintptr_t)out;
+    if (all & 15u) return TLIN_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return TLIN_ERR_UNSUPPORTED;
+    const size_t need = (size_t)B * H * kDecodeMaxSplits * (size_t)(d + 1);
+    if (need > kStaticScratchFloats) {
+        fprintf(stderr, "libtlin: tlin_decode_step_static needs %zu bytes of scratch for B*H=%lld, d=%d but the "
+                        "built-in array holds %zu bytes; use tlin_decode_step with a workspace instead\n",
+                need * sizeof(float), (long long)B * H, d, kStaticScratchFloats * sizeof(float));
+        return TLIN_ERR_WORKSPACE;
+    }
+    int dev = 0;
+    TLIN_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return TLIN_ERR_CUDA;
+    float* scratch = nullptr;
+    int sms = 0;
+    int rc = static_scratch_setup(dev, &scratch, &sms);
+    if (rc != TLIN_OK) return rc;
+    tlin_decode_plan plan;
+    rc = tlin_plan_decode(B, H, pos + 1, d, sms, &plan);
+    if (rc != TLIN_OK) return rc;
+    return launch_decode(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, d, plan, scratch,
+                         (cudaStream_t)stream);
+}
