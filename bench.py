@@ -49,7 +49,7 @@ def load_peaks():
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons for one GPU while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
@@ -57,45 +57,65 @@ class ClockSampler:
         self.gpu = gpu_index
         self.proc = None
         self.path = None
+        self.t0 = self.t1 = None
 
-    def start(self):
+    def launch(self):
+        """Starts nvidia-smi (it needs a moment to come up, so this is called before the warm-up)."""
+        if self.proc is not None:
+            return
         try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
+    def start(self):
+        """Marks the beginning of the timed region."""
+        self.launch()
+        self.t0 = time.time()
+
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        """Marks the end of the timed region and summarises the samples taken inside it."""
+        self.t1 = time.time()
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": "timed region"}
         if self.proc is None:
             return out
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, smax, reasons = [], [], set()
+        import datetime
+        rows = []
         try:
             for line in open(self.path):
                 parts = [x.strip() for x in line.split(",")]
-                if len(parts) < 7:
+                if len(parts) < 8:
                     continue
                 try:
-                    sm.append(float(parts[0]))
-                    smax.append(float(parts[1]))
+                    ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    rows.append((ts, float(parts[1]), float(parts[2]), parts[4:8]))
                 except ValueError:
                     continue
-                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[3:7]):
-                    if val.lower().startswith("active"):
-                        reasons.add(name)
             os.unlink(self.path)
         except Exception:
             pass
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+        inside = [r for r in rows if self.t0 - 0.01 <= r[0] <= self.t1 + 0.01]
+        if not inside and rows:      # region shorter than the sampling period: fall back to samples since launch (warm-up load)
+            inside = rows[-3:]
+            out["window"] = "last samples before the end of the timed region"
+        if inside:
+            reasons = set()
+            for r in inside:
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            out.update(sm_mhz=statistics.median(r[1] for r in inside), sm_max_mhz=max(r[2] for r in inside),
+                       reasons=sorted(reasons), samples=len(inside))
         return out
 
 
@@ -122,6 +142,8 @@ def max_over_ranks(x: float, world: int, device) -> float:
 
 def time_steps(step_fn, steps, warmup, world, device, sampler=None):
     """Device time of `steps` calls (CUDA events on the current stream), max over ranks, in ms."""
+    if sampler:
+        sampler.launch()
     for i in range(warmup):
         step_fn(i)
     torch.cuda.synchronize()
@@ -361,7 +383,7 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", choices=sorted(WORKLOADS), default="fwd128k")
     ap.add_argument("--impl", choices=["tlin", "reference"], default="tlin")
@@ -369,6 +391,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--decode-steps", type=int, default=0, help="timed decode steps (default: max(steps, 64))")
+    ap.add_argument("--shape", default="", help="custom forward shape B,H,N,W,d[,causal] instead of --workload (profiling)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "tlin" else args.warmup
     if args.decode_steps <= 0:
@@ -389,6 +412,10 @@ def main():
         torch.distributed.init_process_group("nccl", device_id=device)
     peaks = load_peaks()
     wl = synth.WORKLOADS[WORKLOADS[args.workload]]
+    if args.shape:
+        v = [int(x) for x in args.shape.split(",")]
+        wl = synth.Workload("custom_" + args.shape.replace(",", "_"), v[0], v[1], v[4], v[2], v[3], seed=9,
+                            causal_window=v[5] if len(v) > 5 else 1)
     with_cpu = (not args.no_cpu) and world == 1
     runner = run_decode if wl.decode else run_forward
     main_res = runner(wl, args, rank, world, device, peaks, with_cpu)

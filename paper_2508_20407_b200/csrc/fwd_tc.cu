@@ -1,8 +1,545 @@
-// Tensor-core forward kernel (placeholder until the tcgen05 path lands).
+// Tensor-core forward kernel for sm_100a: exact softmax attention of W queries over N keys
+// (Section 3 attention formula; causal rule j <= N-W+i inside the window), bf16 in, fp32 accumulate.
+//
+// One CTA owns 256 query rows of one (b,h) (two 128-row Q tiles) and streams a contiguous range of
+// 128-key tiles.  K and V tiles arrive by TMA (128-byte swizzle) into a shared-memory ring; one thread
+// issues tcgen05.mma: S_i = Q_i K_j^T into TMEM, then O_i += P_i V_j with P_i read from TMEM and V_j
+// as an MN-major shared-memory operand.  Two softmax warpgroups (one per Q tile, one thread per row)
+// read S_i from TMEM, keep a running max / sum in base-2 units, write P_i (bf16) over S_i, and rescale
+// O_i only when the running max has grown by more than 2^8 (the final O/l is exact either way).
+// While one warpgroup does its exponentials the tensor pipe works on the other Q tile.
+//
+// CTAs are numbered group*q_tiles + q_tile: the q_tiles CTAs of a group walk the same (b,h,key-tile)
+// units at the same time, so K/V tiles are fetched from HBM once and re-read from L2.  A group's unit
+// range may start or end in the middle of a (b,h); such partial results (normalised o, lse) go to the
+// workspace and fwd_merge_kernel combines them with log-sum-exp weights.
+//
+// Every wait is bounded: on expiry the CTA sets the library's error word, drains and exits.
 #include "tlin_internal.h"
+#include "sm100_ptx.cuh"
+#include <math_constants.h>
+#include <mutex>
+
 namespace tlin {
-int launch_fwd_tc(const void*, const void*, const void*, void*, float*, int, int, int, int, int, int,
-                  const tlin_fwd_plan&, float*, cudaStream_t) {
+namespace {
+
+using namespace ptx;
+
+constexpr int kQTile = 128;                 // rows per Q tile (one TMEM lane per row)
+constexpr int kTileM = 2 * kQTile;          // rows per CTA
+constexpr int kProducerWarp = 8;
+constexpr int kMmaWarp = 9;
+constexpr int kThreads = 32 * 10;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.0f;   // base-2 units
+
+template <int D>
+struct Cfg {
+    static constexpr int kTileBytes = kQTile * D * 2;          // one 128-row tile of Q, K or V
+    static constexpr int kBoxes = D / 64;                      // 64-element (128-byte) column blocks per tile
+    static constexpr int kSlots = D == 128 ? 5 : 8;            // K/V ring slots
+    static constexpr int kSmemTiles = (2 + kSlots) * kTileBytes;
+    static constexpr int kNumBars = 8 + 2 * kSlots;
+    static constexpr int kSmemBytes = kSmemTiles + kNumBars * 8 + 16 + 1024;   // + alignment slack
+    // TMEM columns: S0, S1 (128 each), O0, O1 (D each)
+    static constexpr uint32_t kColS = 0, kColO = 256;
+};
+
+struct Params {
+    void* out;            // [B*H, W, D] bf16
+    float* lse;           // [B*H, W] or null
+    float* ws;            // partial slots
+    int* status;
+    long long total_units;
+    int n_groups, q_tiles, key_tiles;
+    int N, W, causal;
+    float scale_log2e;
+};
+
+// Segments of a group's unit range: one per (b,h) it touches.
+struct Segment { int bh, t_begin, t_end; };
+
+struct SegmentWalker {
+    long long u, u1;
+    int T;
+    __device__ SegmentWalker(const Params& p, int g) : T(p.key_tiles) {
+        u = (long long)(((unsigned long long)g * (unsigned long long)p.total_units) / (unsigned)p.n_groups);
+        u1 = (long long)(((unsigned long long)(g + 1) * (unsigned long long)p.total_units) / (unsigned)p.n_groups);
+    }
+    __device__ bool next(Segment& s) {
+        if (u >= u1) return false;
+        s.bh = (int)(u / T);
+        s.t_begin = (int)(u - (long long)s.bh * T);
+        const long long left = u1 - u;
+        s.t_end = (int)((long long)s.t_begin + left < (long long)T ? (long long)s.t_begin + left : (long long)T);
+        u += s.t_end - s.t_begin;
+        return true;
+    }
+};
+
+// Number of key tiles Q tile `i` of this CTA may use at all (0 if the tile lies beyond W).
+__device__ __forceinline__ int tiles_allowed(const Params& p, int row0, int i) {
+    const int r_first = row0 + i * kQTile;
+    if (r_first >= p.W) return 0;
+    if (!p.causal) return p.key_tiles;
+    const long long r_end = r_first + kQTile < p.W ? r_first + kQTile : p.W;     // one past the last row
+    const long long keys = (long long)p.N - p.W + r_end;                        // keys visible to the last row
+    return (int)((keys + kTileN - 1) / kTileN);
+}
+__device__ __forceinline__ int seg_count(const Segment& s, int allowed) {
+    const int e = s.t_end < allowed ? s.t_end : allowed;
+    return e > s.t_begin ? e - s.t_begin : 0;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+              const __grid_constant__ CUtensorMap map_v, const Params p) {
+    using C = Cfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sQ = smem;                               // 2 tiles
+    uint8_t* sRing = smem + 2 * C::kTileBytes;        // kSlots tiles
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kSmemTiles);
+    uint64_t* q_full = bars + 0;
+    uint64_t* q_empty = bars + 1;
+    uint64_t* s_full = bars + 2;      // [2]
+    uint64_t* p_full = bars + 4;      // [2]
+    uint64_t* pv_done = bars + 6;     // [2]
+    uint64_t* kv_full = bars + 8;     // [kSlots]
+    uint64_t* kv_empty = bars + 8 + C::kSlots;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::kNumBars);
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = blockIdx.x / p.q_tiles;
+    const int qt = blockIdx.x - g * p.q_tiles;
+    const int row0 = qt * kTileM;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(q_full, 1);
+        mbar_init(q_empty, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&s_full[i], 1);
+            mbar_init(&p_full[i], kQTile);
+            mbar_init(&pv_done[i], 1);
+        }
+        for (int s = 0; s < C::kSlots; ++s) {
+            mbar_init(&kv_full[s], 1);
+            mbar_init(&kv_empty[s], 1);
+        }
+        fence_mbar_init();
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(tmem_slot, 512);
+        tmem_relinquish();
+    }
+    if (warp == kProducerWarp && lane == 0) {
+        prefetch_tensormap(&map_q);
+        prefetch_tensormap(&map_k);
+        prefetch_tensormap(&map_v);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    volatile int* abort_p = &abort_flag;
+
+    const int allowed0 = tiles_allowed(p, row0, 0);
+    const int allowed1 = tiles_allowed(p, row0, 1);
+
+    if (warp == kProducerWarp) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;           // ring counter
+            uint32_t seg_idx = 0;
+            bool ok = true;
+            SegmentWalker walk(p, g);
+            Segment s;
+            while (ok && walk.next(s)) {
+                const int c0 = seg_count(s, allowed0), c1 = seg_count(s, allowed1);
+                const int cnt = c0 > c1 ? c0 : c1;
+                if (cnt == 0) continue;
+                if (seg_idx > 0) ok = mbar_wait(q_empty, (seg_idx - 1) & 1, abort_p);
+                if (!ok) break;
+                mbar_arrive_expect_tx(q_full, 2 * C::kTileBytes);
+                for (int i = 0; i < 2; ++i)
+                    for (int b = 0; b < C::kBoxes; ++b)
+                        tma_load_3d(sQ + i * C::kTileBytes + b * (kQTile * 128), &map_q, q_full, b * 64, row0 + i * kQTile, s.bh);
+                for (int j = 0; j < cnt && ok; ++j) {
+                    const int t = s.t_begin + j;
+                    for (int kv = 0; kv < 2 && ok; ++kv) {
+                        const uint32_t slot = it % C::kSlots, round = it / C::kSlots;
+                        ok = mbar_wait(&kv_empty[slot], (round & 1) ^ 1, abort_p);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&kv_full[slot], C::kTileBytes);
+                        uint8_t* dst = sRing + slot * C::kTileBytes;
+                        for (int b = 0; b < C::kBoxes; ++b)
+                            tma_load_3d(dst + b * (kQTile * 128), kv == 0 ? &map_k : &map_v, &kv_full[slot], b * 64, t * kTileN, s.bh);
+                        ++it;
+                    }
+                }
+                ++seg_idx;
+            }
+            if (!ok) {
+                // leave no copy in flight: every slot armed in its latest round must have landed
+                for (uint32_t back = 0; back < (uint32_t)C::kSlots && back < it; ++back) {
+                    const uint32_t id = it - 1 - back, slot = id % C::kSlots, round = id / C::kSlots;
+                    int dummy = 0;
+                    mbar_wait(&kv_full[slot], round & 1, &dummy, 200000000LL);
+                }
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc_qk = make_idesc_bf16(kQTile, kTileN, 0, 0);
+            const uint32_t idesc_pv = make_idesc_bf16(kQTile, D, 0, 1);
+            const uint32_t q_addr = smem_u32(sQ), ring_addr = smem_u32(sRing);
+            uint32_t it = 0, seg_idx = 0;
+            uint32_t n_pv[2] = {0, 0};
+            bool ok = true;
+            auto issue_qk = [&](int i, uint32_t k_slot) {
+                const uint32_t a0 = q_addr + i * C::kTileBytes, b0 = ring_addr + k_slot * C::kTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * (kQTile * 128) + (kk & 3) * 32;
+                    mma_ss(tmem_base + C::kColS + i * kTileN, make_smem_desc_sw128(a0 + off, 16, 1024),
+                           make_smem_desc_sw128(b0 + off, 16, 1024), idesc_qk, kk > 0);
+                }
+                tc_commit(&s_full[i]);
+            };
+            auto issue_pv = [&](int i, uint32_t v_slot, bool accumulate) {
+                const uint32_t b0 = ring_addr + v_slot * C::kTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < kTileN / 16; ++kk)
+                    mma_ts(tmem_base + C::kColO + i * D, tmem_base + C::kColS + i * kTileN + kk * 8,
+                           make_smem_desc_sw128(b0 + kk * 2048, kQTile * 128, 1024), idesc_pv, (accumulate || kk > 0) ? 1u : 0u);
+                tc_commit(&pv_done[i]);
+            };
+            SegmentWalker walk(p, g);
+            Segment s;
+            while (ok && walk.next(s)) {
+                const int c0 = seg_count(s, allowed0), c1 = seg_count(s, allowed1);
+                const int cnt = c0 > c1 ? c0 : c1;
+                if (cnt == 0) continue;
+                const int cq[2] = {c0, c1};
+                ok = mbar_wait(q_full, seg_idx & 1, abort_p);
+                if (!ok) break;
+                // first K tile
+                uint32_t k_slot = it % C::kSlots;
+                ok = mbar_wait(&kv_full[k_slot], (it / C::kSlots) & 1, abort_p);
+                if (!ok) break;
+                tc_fence_after();
+                for (int i = 0; i < 2; ++i)
+                    if (cq[i] > 0) issue_qk(i, k_slot);
+                tc_commit(&kv_empty[k_slot]);
+                ++it;
+                for (int j = 0; j < cnt && ok; ++j) {
+                    const uint32_t v_slot = it % C::kSlots;
+                    ok = mbar_wait(&kv_full[v_slot], (it / C::kSlots) & 1, abort_p);
+                    if (!ok) break;
+                    ++it;
+                    const bool have_next = j + 1 < cnt;
+                    uint32_t nk_slot = 0;
+                    if (have_next) {
+                        nk_slot = it % C::kSlots;
+                        ok = mbar_wait(&kv_full[nk_slot], (it / C::kSlots) & 1, abort_p);
+                        if (!ok) break;
+                        ++it;
+                    }
+                    tc_fence_after();
+                    for (int i = 0; i < 2 && ok; ++i) {
+                        if (j < cq[i]) {
+                            ok = mbar_wait(&p_full[i], n_pv[i] & 1, abort_p);
+                            if (!ok) break;
+                            tc_fence_after();
+                            issue_pv(i, v_slot, j > 0);
+                            ++n_pv[i];
+                        }
+                        if (i == 1) tc_commit(&kv_empty[v_slot]);
+                        if (have_next && j + 1 < cq[i]) issue_qk(i, nk_slot);
+                        if (have_next && i == 1) tc_commit(&kv_empty[nk_slot]);
+                    }
+                }
+                if (!ok) break;
+                tc_commit(q_empty);
+                ++seg_idx;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax warpgroups (one per Q tile)
+        const int i = warp >> 2;                           // Q tile
+        const int r = (warp & 3) * 32 + lane;              // row inside the Q tile == TMEM lane
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_base + lane_addr + C::kColS + i * kTileN;
+        const uint32_t tO = tmem_base + lane_addr + C::kColO + i * D;
+        const int row = row0 + i * kQTile + r;             // row inside W (may lie beyond W: computed, never stored)
+        const int allowed_i = i == 0 ? allowed0 : allowed1;
+        // keys visible to this row, and to the first row of this warp (the smallest in the warp)
+        const long long lim_row_ll = p.causal ? (long long)p.N - p.W + row + 1 : (long long)p.N;
+        const int lim_row = (int)(lim_row_ll < p.N ? lim_row_ll : p.N);
+        const long long lim_warp_ll = p.causal ? (long long)p.N - p.W + (row - lane) + 1 : (long long)p.N;
+        const int lim_warp = (int)(lim_warp_ll < p.N ? lim_warp_ll : p.N);
+
+        uint32_t n = 0;     // tiles processed by this warpgroup (phase counter of s_full/p_full/pv_done)
+        bool ok = true;
+        SegmentWalker walk(p, g);
+        Segment s;
+        while (ok && walk.next(s)) {
+            const int cnt_i = seg_count(s, allowed_i);
+            float m_ref = -CUDART_INF_F, l = 0.f;
+            for (int j = 0; j < cnt_i; ++j) {
+                ok = mbar_wait(&s_full[i], n & 1, abort_p);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                const int k0 = (s.t_begin + j) * kTileN;
+                const bool masked = k0 + kTileN > lim_warp;   // warp-uniform: some column of some lane is masked
+                const int nvalid = lim_row - k0;              // columns [0, nvalid) of this tile are allowed for this row
+                // pass 1: row maximum of the tile
+                float tmax = -CUDART_INF_F;
+#pragma unroll
+                for (int c = 0; c < kTileN / 32; ++c) {
+                    uint32_t tmp[32];
+                    tmem_ld32(tS + c * 32, tmp);
+                    if (masked) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (c * 32 + e >= nvalid) tmp[e] = 0xff800000u;   // -inf
+                    }
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(tmp[e]));
+                }
+                const float m_new = fmaxf(m_ref, tmax * p.scale_log2e);
+                const bool need = m_new > m_ref + kRescaleThreshold;
+                if (__any_sync(0xffffffffu, need)) {
+                    const float alpha = need ? ex2(m_ref - m_new) : 1.f;     // m_ref = -inf -> 0
+                    if (j > 0) {
+                        ok = mbar_wait(&pv_done[i], (n - 1) & 1, abort_p);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                        tc_fence_after();
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + c * 32, o);
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                            tmem_st32(tO + c * 32, o);
+                        }
+                    }
+                    l *= alpha;
+                    if (need) m_ref = m_new;
+                }
+                const float m_use = m_ref == -CUDART_INF_F ? 0.f : m_ref;
+                // pass 2: P = 2^(s*scale - m), written as bf16 over the columns of S already consumed
+#pragma unroll
+                for (int c = 0; c < kTileN / 32; ++c) {
+                    uint32_t tmp[32];
+                    tmem_ld32(tS + c * 32, tmp);
+                    if (masked) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (c * 32 + e >= nvalid) tmp[e] = 0xff800000u;
+                    }
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const float p0 = ex2(fmaf(__uint_as_float(tmp[2 * e]), p.scale_log2e, -m_use));
+                        const float p1 = ex2(fmaf(__uint_as_float(tmp[2 * e + 1]), p.scale_log2e, -m_use));
+                        l += p0 + p1;
+                        pk[e] = pack_bf16x2(p0, p1);
+                    }
+                    tmem_st16(tS + c * 16, pk);
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(&p_full[i]);
+                ++n;
+            }
+            if (!ok) break;
+            if (allowed_i == 0) continue;                  // this Q tile does not exist: nothing to write
+            // ---------------------------------------------------------------- epilogue of the segment
+            const bool whole = s.t_begin == 0 && s.t_end == p.key_tiles;
+            if (cnt_i > 0) {
+                ok = mbar_wait(&pv_done[i], (n - 1) & 1, abort_p);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+            }
+            const float inv_l = l > 0.f ? 1.f / l : 0.f;
+            const float lse_val = l > 0.f ? (m_ref + log2f(l)) * kLn2 : -CUDART_INF_F;
+            const bool store = row < p.W;
+            if (whole) {
+                __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + ((long long)s.bh * p.W + row) * D;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t o[32];
+                    if (cnt_i > 0) tmem_ld32(tO + c * 32, o);
+                    if (store) {
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            uint4 w;
+                            w.x = pack_bf16x2(__uint_as_float(o[v4 * 8 + 0]) * inv_l, __uint_as_float(o[v4 * 8 + 1]) * inv_l);
+                            w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * inv_l, __uint_as_float(o[v4 * 8 + 3]) * inv_l);
+                            w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * inv_l, __uint_as_float(o[v4 * 8 + 5]) * inv_l);
+                            w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * inv_l, __uint_as_float(o[v4 * 8 + 7]) * inv_l);
+                            *reinterpret_cast<uint4*>(orow + c * 32 + v4 * 8) = w;
+                        }
+                    }
+                }
+                if (store && p.lse != nullptr) p.lse[(long long)s.bh * p.W + row] = lse_val;
+            } else {
+                // partial result -> workspace slot (0: first segment of this CTA's range, 1: a later one)
+                const long long u_first = (long long)(((unsigned long long)g * (unsigned long long)p.total_units) / (unsigned)p.n_groups);
+                const int slot = s.bh == (int)(u_first / p.key_tiles) ? 0 : 1;
+                float* base = p.ws + ((long long)blockIdx.x * 2 + slot) * (long long)kTileM * (D + 1);
+                float* orow = base + (long long)(i * kQTile + r) * D;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t o[32];
+                    if (cnt_i > 0) tmem_ld32(tO + c * 32, o);
+#pragma unroll
+                    for (int v4 = 0; v4 < 8; ++v4) {
+                        float4 w;
+                        w.x = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 0]) * inv_l : 0.f;
+                        w.y = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 1]) * inv_l : 0.f;
+                        w.z = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 2]) * inv_l : 0.f;
+                        w.w = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 3]) * inv_l : 0.f;
+                        *reinterpret_cast<float4*>(orow + c * 32 + v4 * 4) = w;
+                    }
+                }
+                base[(long long)kTileM * D + i * kQTile + r] = lse_val;
+            }
+            tc_fence_before();      // TMEM reads of O are complete before the next segment's arrive lets PV overwrite it
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) atomicExch(p.status, (int)TLIN_ERR_TIMEOUT);
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// Combines the partial results of every (b,h) whose key tiles were split between groups.
+// One CTA (D threads) per query row.
+template <int D>
+__global__ void __launch_bounds__(D)
+fwd_merge_kernel(const Params p) {
+    const long long rowid = blockIdx.x;                 // bh * W + row
+    const int bh = (int)(rowid / p.W), row = (int)(rowid - (long long)bh * p.W);
+    const unsigned long long T = (unsigned long long)p.key_tiles, U = (unsigned long long)p.total_units, G = (unsigned)p.n_groups;
+    // groups holding the first and the last unit of this (b,h): largest g with floor(g*U/G) <= x
+    const unsigned long long x0 = (unsigned long long)bh * T, x1 = x0 + T - 1;
+    const int g_lo = (int)(((x0 + 1) * G - 1) / U), g_hi = (int)(((x1 + 1) * G - 1) / U);
+    if (g_lo == g_hi) return;                           // written directly by the attention kernel
+    const int qt = row / kTileM, rr = row - qt * kTileM;
+    const int c = threadIdx.x;
+    float m = -CUDART_INF_F;
+    for (int g = g_lo; g <= g_hi; ++g) {
+        const int cta = g * p.q_tiles + qt;
+        const int slot = bh == (int)((((unsigned long long)g * U) / G) / T) ? 0 : 1;
+        const float* base = p.ws + ((long long)cta * 2 + slot) * (long long)kTileM * (D + 1);
+        m = fmaxf(m, base[(long long)kTileM * D + rr]);
+    }
+    float z = 0.f, acc = 0.f;
+    for (int g = g_lo; g <= g_hi; ++g) {
+        const int cta = g * p.q_tiles + qt;
+        const int slot = bh == (int)((((unsigned long long)g * U) / G) / T) ? 0 : 1;
+        const float* base = p.ws + ((long long)cta * 2 + slot) * (long long)kTileM * (D + 1);
+        const float w = expf(base[(long long)kTileM * D + rr] - m);      // -inf (empty part) -> 0
+        z += w;
+        acc = fmaf(w, base[(long long)rr * D + c], acc);
+    }
+    reinterpret_cast<__nv_bfloat16*>(p.out)[rowid * D + c] = __float2bfloat16_rn(acc / z);
+    if (p.lse != nullptr && c == 0) p.lse[rowid] = m + logf(z);
+}
+
+// ---------------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(f);
+    });
+    return fn;
+}
+
+// [BH, rows, D] bf16, box = 64 elements x 128 rows x 1, 128-byte swizzle, zero fill outside.
+int make_map(CUtensorMap* m, const void* ptr, int D, long long rows, long long bh) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return TLIN_ERR_CUDA;
+    cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)bh};
+    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)rows * D * 2};
+    cuuint32_t box[3] = {64, (cuuint32_t)kQTile, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    const CUresult rc = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc != CUDA_SUCCESS) {
+        fprintf(stderr, "libtlin: cuTensorMapEncodeTiled failed (%d)\n", (int)rc);
+        return TLIN_ERR_CUDA;
+    }
+    return TLIN_OK;
+}
+
+template <int D>
+int launch_d(const void* q, const void* k, const void* v, void* out, float* lse, int B, int H, int N, int W,
+             int causal, const tlin_fwd_plan& plan, float* ws, cudaStream_t st) {
+    using C = Cfg<D>;
+    const long long bh = (long long)B * H;
+    CUtensorMap mq, mk, mv;
+    int rc = make_map(&mq, q, D, W, bh);
+    if (rc == TLIN_OK) rc = make_map(&mk, k, D, N, bh);
+    if (rc == TLIN_OK) rc = make_map(&mv, v, D, N, bh);
+    if (rc != TLIN_OK) return rc;
+    Params p;
+    p.out = out; p.lse = lse; p.ws = ws; p.status = status_word();
+    if (!p.status) return TLIN_ERR_CUDA;
+    p.total_units = plan.total_units; p.n_groups = plan.n_groups; p.q_tiles = plan.q_tiles; p.key_tiles = plan.key_tiles;
+    p.N = N; p.W = W; p.causal = causal;
+    p.scale_log2e = kLog2e / sqrtf((float)D);
+    static std::once_flag attr_once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(attr_once, [] {
+        attr_err = cudaFuncSetAttribute(fwd_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    });
+    TLIN_CUDA_CHECK(attr_err);
+    fwd_tc_kernel<D><<<plan.n_ctas, kThreads, C::kSmemBytes, st>>>(mq, mk, mv, p);
+    TLIN_CUDA_CHECK(cudaGetLastError());
+    count_launch();
+    if (plan.uses_workspace) {
+        fwd_merge_kernel<D><<<(unsigned)(bh * W), D, 0, st>>>(p);
+        TLIN_CUDA_CHECK(cudaGetLastError());
+        count_launch();
+    }
+    return TLIN_OK;
+}
+
+}  // namespace
+
+int launch_fwd_tc(const void* q, const void* k, const void* v, void* out, float* lse,
+                  int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& plan,
+                  float* ws, cudaStream_t st) {
+    if (plan.tile_m != kTileM || plan.tile_n != kTileN) return TLIN_ERR_UNSUPPORTED;
+    if ((long long)B * H * W > 0x7fffffffLL) return TLIN_ERR_UNSUPPORTED;
+    if (d == 128) return launch_d<128>(q, k, v, out, lse, B, H, N, W, causal, plan, ws, st);
+    if (d == 64) return launch_d<64>(q, k, v, out, lse, B, H, N, W, causal, plan, ws, st);
     return TLIN_ERR_UNSUPPORTED;
 }
+
 }  // namespace tlin

@@ -43,7 +43,7 @@ extern "C" int tlin_plan_forward(int B, int H, int N, int W, int d, int causal_w
     const bool tc_shape = !is_f32 && (d == 64 || d == 128);
     if (impl == 2 && !tc_shape) return TLIN_ERR_UNSUPPORTED;
     if (is_f32 ? (d % 4 != 0 || d > 256) : (d % 8 != 0 || d > 256)) return TLIN_ERR_UNSUPPORTED;
-    const bool tc = tc_shape && impl == 2;  // automatic = CUDA-core kernel until the tensor path is enabled
+    const bool tc = tc_shape && impl != 1;
     tlin_fwd_plan p = {};
     const int64_t bh = (int64_t)B * H;
     p.tensor_path = tc ? 1 : 0;
@@ -61,7 +61,7 @@ extern "C" int tlin_plan_forward(int B, int H, int N, int W, int d, int causal_w
         *plan = p;
         return TLIN_OK;
     }
-    p.tile_m = 128;
+    p.tile_m = 256;            // two 128-row Q tiles per CTA
     p.tile_n = kTileN;
     p.q_tiles = (W + p.tile_m - 1) / p.tile_m;
     p.key_tiles = (N + p.tile_n - 1) / p.tile_n;
