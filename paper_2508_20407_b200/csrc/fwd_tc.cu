@@ -6,7 +6,7 @@
 // issues tcgen05.mma: S_i = Q_i K_j^T into TMEM, then O_i += P_i V_j with P_i read from TMEM and V_j
 // as an MN-major shared-memory operand.  Two softmax warpgroups (one per Q tile, one thread per row)
 // read S_i from TMEM, keep a running max / sum in base-2 units, write P_i (bf16) over S_i, and rescale
-// O_i only when the running max has grown by more than 2^8 (the final O/l is exact either way).
+// O_i only when the running max has grown by more than 2^32 (the final O/l is exact either way).
 // While one warpgroup does its exponentials the tensor pipe works on the other Q tile.
 //
 // CTAs are numbered group*q_tiles + q_tile: the q_tiles CTAs of a group walk the same (b,h,key-tile)
@@ -32,7 +32,7 @@ constexpr int kMmaWarp = 9;
 constexpr int kThreads = 32 * 10;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr float kRescaleThreshold = 8.0f;   // base-2 units
+constexpr float kRescaleThreshold = 32.0f;  // base-2 units: P stays below 2^32, far inside bf16/fp32 range
 
 template <int D>
 struct Cfg {
@@ -40,7 +40,7 @@ struct Cfg {
     static constexpr int kBoxes = D / 64;                      // 64-element (128-byte) column blocks per tile
     static constexpr int kSlots = D == 128 ? 5 : 8;            // K/V ring slots
     static constexpr int kSmemTiles = (2 + kSlots) * kTileBytes;
-    static constexpr int kNumBars = 8 + 2 * kSlots;
+    static constexpr int kNumBars = 10 + 2 * kSlots;
     static constexpr int kSmemBytes = kSmemTiles + kNumBars * 8 + 16 + 1024;   // + alignment slack
     // TMEM columns: S0, S1 (128 each), O0, O1 (D each)
     static constexpr uint32_t kColS = 0, kColO = 256;
@@ -107,8 +107,9 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     uint64_t* s_full = bars + 2;      // [2]
     uint64_t* p_full = bars + 4;      // [2]
     uint64_t* pv_done = bars + 6;     // [2]
-    uint64_t* kv_full = bars + 8;     // [kSlots]
-    uint64_t* kv_empty = bars + 8 + C::kSlots;
+    uint64_t* p_half = bars + 8;      // [2]  first 64 keys of P written (PV may start on them)
+    uint64_t* kv_full = bars + 10;    // [kSlots]
+    uint64_t* kv_empty = bars + 10 + C::kSlots;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::kNumBars);
     __shared__ int abort_flag;
 
@@ -124,6 +125,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         for (int i = 0; i < 2; ++i) {
             mbar_init(&s_full[i], 1);
             mbar_init(&p_full[i], kQTile);
+            mbar_init(&p_half[i], kQTile);
             mbar_init(&pv_done[i], 1);
         }
         for (int s = 0; s < C::kSlots; ++s) {
@@ -211,13 +213,15 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 }
                 tc_commit(&s_full[i]);
             };
-            auto issue_pv = [&](int i, uint32_t v_slot, bool accumulate) {
+            auto issue_pv_half = [&](int i, uint32_t v_slot, bool accumulate, int half) {
                 const uint32_t b0 = ring_addr + v_slot * C::kTileBytes;
 #pragma unroll
-                for (int kk = 0; kk < kTileN / 16; ++kk)
+                for (int k4 = 0; k4 < kTileN / 32; ++k4) {
+                    const int kk = half * (kTileN / 32) + k4;
                     mma_ts(tmem_base + C::kColO + i * D, tmem_base + C::kColS + i * kTileN + kk * 8,
                            make_smem_desc_sw128(b0 + kk * 2048, kQTile * 128, 1024), idesc_pv, (accumulate || kk > 0) ? 1u : 0u);
-                tc_commit(&pv_done[i]);
+                }
+                if (half == 1) tc_commit(&pv_done[i]);
             };
             SegmentWalker walk(p, g);
             Segment s;
@@ -253,10 +257,14 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     tc_fence_after();
                     for (int i = 0; i < 2 && ok; ++i) {
                         if (j < cq[i]) {
+                            ok = mbar_wait(&p_half[i], n_pv[i] & 1, abort_p);
+                            if (!ok) break;
+                            tc_fence_after();
+                            issue_pv_half(i, v_slot, j > 0, 0);
                             ok = mbar_wait(&p_full[i], n_pv[i] & 1, abort_p);
                             if (!ok) break;
                             tc_fence_after();
-                            issue_pv(i, v_slot, j > 0);
+                            issue_pv_half(i, v_slot, j > 0, 1);
                             ++n_pv[i];
                         }
                         if (i == 1) tc_commit(&kv_empty[v_slot]);
@@ -299,19 +307,24 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 const int k0 = (s.t_begin + j) * kTileN;
                 const bool masked = k0 + kTileN > lim_warp;   // warp-uniform: some column of some lane is masked
                 const int nvalid = lim_row - k0;              // columns [0, nvalid) of this tile are allowed for this row
-                // pass 1: row maximum of the tile
+                // pass 1: row maximum of the tile (the load of chunk c+1 is in flight while chunk c is reduced)
                 float tmax = -CUDART_INF_F;
+                {
+                    uint32_t buf[2][32];
+                    tmem_ld32_async(tS, buf[0]);
 #pragma unroll
-                for (int c = 0; c < kTileN / 32; ++c) {
-                    uint32_t tmp[32];
-                    tmem_ld32(tS + c * 32, tmp);
-                    if (masked) {
+                    for (int c = 0; c < kTileN / 32; ++c) {
+                        uint32_t(&cur)[32] = buf[c & 1];
+                        tmem_wait_ld(cur);
+                        if (c + 1 < kTileN / 32) tmem_ld32_async(tS + (c + 1) * 32, buf[(c + 1) & 1]);
+                        if (masked) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (c * 32 + e >= nvalid) tmp[e] = 0xff800000u;   // -inf
+                            for (int e = 0; e < 32; ++e)
+                                if (c * 32 + e >= nvalid) cur[e] = 0xff800000u;   // -inf
+                        }
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(cur[e]));
                     }
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(tmp[e]));
                 }
                 const float m_new = fmaxf(m_ref, tmax * p.scale_log2e);
                 const bool need = m_new > m_ref + kRescaleThreshold;
@@ -336,24 +349,34 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 }
                 const float m_use = m_ref == -CUDART_INF_F ? 0.f : m_ref;
                 // pass 2: P = 2^(s*scale - m), written as bf16 over the columns of S already consumed
+                {
+                    uint32_t buf[2][32];
+                    tmem_ld32_async(tS, buf[0]);
 #pragma unroll
-                for (int c = 0; c < kTileN / 32; ++c) {
-                    uint32_t tmp[32];
-                    tmem_ld32(tS + c * 32, tmp);
-                    if (masked) {
+                    for (int c = 0; c < kTileN / 32; ++c) {
+                        uint32_t(&cur)[32] = buf[c & 1];
+                        tmem_wait_ld(cur);
+                        if (c + 1 < kTileN / 32) tmem_ld32_async(tS + (c + 1) * 32, buf[(c + 1) & 1]);
+                        if (masked) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (c * 32 + e >= nvalid) tmp[e] = 0xff800000u;
+                            for (int e = 0; e < 32; ++e)
+                                if (c * 32 + e >= nvalid) cur[e] = 0xff800000u;
+                        }
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const float p0 = ex2(fmaf(__uint_as_float(cur[2 * e]), p.scale_log2e, -m_use));
+                            const float p1 = ex2(fmaf(__uint_as_float(cur[2 * e + 1]), p.scale_log2e, -m_use));
+                            l += p0 + p1;
+                            pk[e] = pack_bf16x2(p0, p1);
+                        }
+                        tmem_st16(tS + c * 16, pk);
+                        if (c == kTileN / 64 - 1) {        // first 64 keys are in place: let the PV MMAs start on them
+                            tc_wait_st();
+                            tc_fence_before();
+                            mbar_arrive(&p_half[i]);
+                        }
                     }
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const float p0 = ex2(fmaf(__uint_as_float(tmp[2 * e]), p.scale_log2e, -m_use));
-                        const float p1 = ex2(fmaf(__uint_as_float(tmp[2 * e + 1]), p.scale_log2e, -m_use));
-                        l += p0 + p1;
-                        pk[e] = pack_bf16x2(p0, p1);
-                    }
-                    tmem_st16(tS + c * 16, pk);
                 }
                 tc_wait_st();
                 tc_fence_before();
@@ -428,37 +451,95 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 }
 
 // Combines the partial results of every (b,h) whose key tiles were split between groups.
-// One CTA (D threads) per query row.
+// One CTA per (b,h, q-tile pair, quarter): 8 warps, one query row per warp at a time, 4 (or 2) columns per lane.
+constexpr int kMergeRows = 64;
+constexpr int kMaxParts = 8;          // more partials than this per row are merged in a slower loop
+
 template <int D>
-__global__ void __launch_bounds__(D)
+__global__ void __launch_bounds__(256)
 fwd_merge_kernel(const Params p) {
-    const long long rowid = blockIdx.x;                 // bh * W + row
-    const int bh = (int)(rowid / p.W), row = (int)(rowid - (long long)bh * p.W);
-    const unsigned long long T = (unsigned long long)p.key_tiles, U = (unsigned long long)p.total_units, G = (unsigned)p.n_groups;
-    // groups holding the first and the last unit of this (b,h): largest g with floor(g*U/G) <= x
-    const unsigned long long x0 = (unsigned long long)bh * T, x1 = x0 + T - 1;
-    const int g_lo = (int)(((x0 + 1) * G - 1) / U), g_hi = (int)(((x1 + 1) * G - 1) / U);
-    if (g_lo == g_hi) return;                           // written directly by the attention kernel
-    const int qt = row / kTileM, rr = row - qt * kTileM;
-    const int c = threadIdx.x;
-    float m = -CUDART_INF_F;
-    for (int g = g_lo; g <= g_hi; ++g) {
-        const int cta = g * p.q_tiles + qt;
-        const int slot = bh == (int)((((unsigned long long)g * U) / G) / T) ? 0 : 1;
-        const float* base = p.ws + ((long long)cta * 2 + slot) * (long long)kTileM * (D + 1);
-        m = fmaxf(m, base[(long long)kTileM * D + rr]);
+    constexpr int CPL = D / 32;                           // columns per lane
+    const int blocks_per_tile = kTileM / kMergeRows;
+    const int quarter = blockIdx.x % blocks_per_tile;
+    const int tile_id = blockIdx.x / blocks_per_tile;     // bh * q_tiles + qt
+    const int bh = tile_id / p.q_tiles, qt = tile_id - bh * p.q_tiles;
+    __shared__ const float* part_base[kMaxParts];
+    __shared__ int n_parts_s, g_lo_s;
+    if (threadIdx.x == 0) {
+        const unsigned long long T = (unsigned long long)p.key_tiles, U = (unsigned long long)p.total_units, G = (unsigned)p.n_groups;
+        // groups holding the first and the last unit of this (b,h): largest g with floor(g*U/G) <= x
+        const unsigned long long x0 = (unsigned long long)bh * T, x1 = x0 + T - 1;
+        const int g_lo = (int)(((x0 + 1) * G - 1) / U), g_hi = (int)(((x1 + 1) * G - 1) / U);
+        g_lo_s = g_lo;
+        n_parts_s = g_hi - g_lo + 1;
+        for (int g = g_lo; g <= g_hi && g - g_lo < kMaxParts; ++g) {
+            const int cta = g * p.q_tiles + qt;
+            const int slot = bh == (int)((((unsigned long long)g * U) / G) / T) ? 0 : 1;
+            part_base[g - g_lo] = p.ws + ((long long)cta * 2 + slot) * (long long)kTileM * (D + 1);
+        }
     }
-    float z = 0.f, acc = 0.f;
-    for (int g = g_lo; g <= g_hi; ++g) {
-        const int cta = g * p.q_tiles + qt;
-        const int slot = bh == (int)((((unsigned long long)g * U) / G) / T) ? 0 : 1;
-        const float* base = p.ws + ((long long)cta * 2 + slot) * (long long)kTileM * (D + 1);
-        const float w = expf(base[(long long)kTileM * D + rr] - m);      // -inf (empty part) -> 0
-        z += w;
-        acc = fmaf(w, base[(long long)rr * D + c], acc);
+    __syncthreads();
+    const int n_parts = n_parts_s;
+    if (n_parts <= 1) return;                             // written directly by the attention kernel
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int rq = warp; rq < kMergeRows; rq += 8) {
+        const int rr = quarter * kMergeRows + rq;         // row inside the 256-row tile
+        const int row = qt * kTileM + rr;
+        if (row >= p.W) break;
+        float m = -CUDART_INF_F;
+        if (n_parts <= kMaxParts) {
+            float ls[kMaxParts];
+#pragma unroll
+            for (int i = 0; i < kMaxParts; ++i) {
+                ls[i] = i < n_parts ? part_base[i][(long long)kTileM * D + rr] : -CUDART_INF_F;
+                m = fmaxf(m, ls[i]);
+            }
+            float z = 0.f, acc[CPL];
+#pragma unroll
+            for (int e = 0; e < CPL; ++e) acc[e] = 0.f;
+#pragma unroll
+            for (int i = 0; i < kMaxParts; ++i) {
+                if (i < n_parts) {
+                    const float w = expf(ls[i] - m);      // -inf (empty part) -> 0
+                    z += w;
+                    const float* src = part_base[i] + (long long)rr * D + lane * CPL;
+#pragma unroll
+                    for (int e = 0; e < CPL; ++e) acc[e] = fmaf(w, src[e], acc[e]);
+                }
+            }
+            const float inv = 1.f / z;
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + ((long long)bh * p.W + row) * D + lane * CPL;
+#pragma unroll
+            for (int e = 0; e < CPL; e += 2)
+                *reinterpret_cast<uint32_t*>(dst + e) = pack_bf16x2(acc[e] * inv, acc[e + 1] * inv);
+            if (p.lse != nullptr && lane == 0) p.lse[(long long)bh * p.W + row] = m + logf(z);
+        } else {
+            // many small groups per (b,h): recompute the slot addresses on the fly
+            const unsigned long long T = (unsigned long long)p.key_tiles, U = (unsigned long long)p.total_units, G = (unsigned)p.n_groups;
+            auto base_of = [&](int g) {
+                const int cta = g * p.q_tiles + qt;
+                const int slot = bh == (int)((((unsigned long long)g * U) / G) / T) ? 0 : 1;
+                return p.ws + ((long long)cta * 2 + slot) * (long long)kTileM * (D + 1);
+            };
+            for (int i = 0; i < n_parts; ++i) m = fmaxf(m, base_of(g_lo_s + i)[(long long)kTileM * D + rr]);
+            float z = 0.f, acc[CPL];
+#pragma unroll
+            for (int e = 0; e < CPL; ++e) acc[e] = 0.f;
+            for (int i = 0; i < n_parts; ++i) {
+                const float* base = base_of(g_lo_s + i);
+                const float w = expf(base[(long long)kTileM * D + rr] - m);
+                z += w;
+#pragma unroll
+                for (int e = 0; e < CPL; ++e) acc[e] = fmaf(w, base[(long long)rr * D + lane * CPL + e], acc[e]);
+            }
+            const float inv = 1.f / z;
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + ((long long)bh * p.W + row) * D + lane * CPL;
+#pragma unroll
+            for (int e = 0; e < CPL; e += 2)
+                *reinterpret_cast<uint32_t*>(dst + e) = pack_bf16x2(acc[e] * inv, acc[e + 1] * inv);
+            if (p.lse != nullptr && lane == 0) p.lse[(long long)bh * p.W + row] = m + logf(z);
+        }
     }
-    reinterpret_cast<__nv_bfloat16*>(p.out)[rowid * D + c] = __float2bfloat16_rn(acc / z);
-    if (p.lse != nullptr && c == 0) p.lse[rowid] = m + logf(z);
 }
 
 // ---------------------------------------------------------------------------------------- host side
@@ -523,7 +604,7 @@ int launch_d(const void* q, const void* k, const void* v, void* out, float* lse,
     TLIN_CUDA_CHECK(cudaGetLastError());
     count_launch();
     if (plan.uses_workspace) {
-        fwd_merge_kernel<D><<<(unsigned)(bh * W), D, 0, st>>>(p);
+        fwd_merge_kernel<D><<<(unsigned)(bh * plan.q_tiles * (kTileM / kMergeRows)), 256, 0, st>>>(p);
         TLIN_CUDA_CHECK(cudaGetLastError());
         count_launch();
     }
