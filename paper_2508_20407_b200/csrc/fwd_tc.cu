@@ -298,7 +298,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         Segment s;
         while (ok && walk.next(s)) {
             const int cnt_i = seg_count(s, allowed_i);
-            float m_ref = -CUDART_INF_F, l = 0.f;
+            float m_ref = -CUDART_INF_F;
+            uint64_t l2[2] = {0ull, 0ull};          // four partial row sums as two packed fp32 pairs
             for (int j = 0; j < cnt_i; ++j) {
                 ok = mbar_wait(&s_full[i], n & 1, abort_p);
                 ok = __all_sync(0xffffffffu, ok);
@@ -308,7 +309,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 const bool masked = k0 + kTileN > lim_warp;   // warp-uniform: some column of some lane is masked
                 const int nvalid = lim_row - k0;              // columns [0, nvalid) of this tile are allowed for this row
                 // pass 1: row maximum of the tile (the load of chunk c+1 is in flight while chunk c is reduced)
-                float tmax = -CUDART_INF_F;
+                float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};   // independent chains
                 {
                     uint32_t buf[2][32];
                     tmem_ld32_async(tS, buf[0]);
@@ -323,9 +324,11 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                                 if (c * 32 + e >= nvalid) cur[e] = 0xff800000u;   // -inf
                         }
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(cur[e]));
+                        for (int e = 0; e < 16; ++e)
+                            mx[e & 3] = max3(mx[e & 3], __uint_as_float(cur[2 * e]), __uint_as_float(cur[2 * e + 1]));
                     }
                 }
+                const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
                 const float m_new = fmaxf(m_ref, tmax * p.scale_log2e);
                 const bool need = m_new > m_ref + kRescaleThreshold;
                 if (__any_sync(0xffffffffu, need)) {
@@ -344,12 +347,15 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                             tmem_st32(tO + c * 32, o);
                         }
                     }
-                    l *= alpha;
+                    const uint64_t alpha2 = f2_pack(alpha, alpha);
+                    l2[0] = f2_mul(l2[0], alpha2);
+                    l2[1] = f2_mul(l2[1], alpha2);
                     if (need) m_ref = m_new;
                 }
                 const float m_use = m_ref == -CUDART_INF_F ? 0.f : m_ref;
                 // pass 2: P = 2^(s*scale - m), written as bf16 over the columns of S already consumed
                 {
+                    const uint64_t scale2 = f2_pack(p.scale_log2e, p.scale_log2e), negm2 = f2_pack(-m_use, -m_use);
                     uint32_t buf[2][32];
                     tmem_ld32_async(tS, buf[0]);
 #pragma unroll
@@ -365,9 +371,10 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                         uint32_t pk[16];
 #pragma unroll
                         for (int e = 0; e < 16; ++e) {
-                            const float p0 = ex2(fmaf(__uint_as_float(cur[2 * e]), p.scale_log2e, -m_use));
-                            const float p1 = ex2(fmaf(__uint_as_float(cur[2 * e + 1]), p.scale_log2e, -m_use));
-                            l += p0 + p1;
+                            float x0, x1;
+                            f2_unpack(f2_fma(f2_pack_bits(cur[2 * e], cur[2 * e + 1]), scale2, negm2), x0, x1);
+                            const float p0 = ex2(x0), p1 = ex2(x1);
+                            l2[e & 1] = f2_add(l2[e & 1], f2_pack(p0, p1));
                             pk[e] = pack_bf16x2(p0, p1);
                         }
                         tmem_st16(tS + c * 16, pk);
@@ -392,6 +399,13 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
+            }
+            float l;
+            {
+                float a, b, c, d2;
+                f2_unpack(l2[0], a, b);
+                f2_unpack(l2[1], c, d2);
+                l = (a + b) + (c + d2);
             }
             const float inv_l = l > 0.f ? 1.f / l : 0.f;
             const float lse_val = l > 0.f ? (m_ref + log2f(l)) * kLn2 : -CUDART_INF_F;
