@@ -5,8 +5,10 @@
 // 128-key tiles.  K and V tiles arrive by TMA (128-byte swizzle) into a shared-memory ring; one thread
 // issues tcgen05.mma: S_i = Q_i K_j^T into TMEM, then O_i += P_i V_j with P_i read from TMEM and V_j
 // as an MN-major shared-memory operand.  Two softmax warpgroups (one per Q tile, one thread per row)
-// read S_i from TMEM, keep a running max / sum in base-2 units, write P_i (bf16) over S_i, and rescale
-// O_i only when the running max has grown by more than 2^32 (the final O/l is exact either way).
+// read a whole row of S_i from TMEM into registers once, keep a running max / sum in base-2 units, write
+// P_i (bf16) over S_i, and rescale O_i only when the running max has grown by more than 2^32 (the final
+// O/l is exact either way).  A fixed share of the exponentials is evaluated by a cubic on the FMA pipe,
+// the rest by the special-function unit, so that neither pipe alone bounds the softmax.
 // While one warpgroup does its exponentials the tensor pipe works on the other Q tile.
 //
 // CTAs are numbered group*q_tiles + q_tile: the q_tiles CTAs of a group walk the same (b,h,key-tile)
@@ -29,10 +31,35 @@ constexpr int kQTile = 128;                 // rows per Q tile (one TMEM lane pe
 constexpr int kTileM = 2 * kQTile;          // rows per CTA
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
-constexpr int kThreads = 32 * 10;
+constexpr int kThreads = 32 * 12;          // warps 10 and 11 only lend their registers
+constexpr int kSoftmaxRegs = 216, kOtherRegs = 72;   // 256*224 + 128*56 = 384*168 registers
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kPolyPairs = 5;                // of every 16 column pairs, this many get 2^x from the polynomial
 constexpr float kRescaleThreshold = 32.0f;  // base-2 units: P stays below 2^32, far inside bf16/fp32 range
+
+// 2^x for a packed pair without the special-function unit: x = n + f with n = floor(x) (taken by adding
+// 1.5*2^23 rounding down, which leaves n in the low mantissa bits), 2^f on [0,1) by a cubic fitted for
+// minimum relative error (7.9e-5, well below the 2^-9 rounding of P to bf16), n added into the exponent field.
+// x is clamped to [-126, inf) first; values the caller produces stay far below the upper exponent limit.
+__device__ __forceinline__ void exp2_poly2(uint64_t x2, float& p0, float& p1) {
+    float x0, x1;
+    f2_unpack(x2, x0, x1);
+    x0 = fmaxf(x0, -126.f);
+    x1 = fmaxf(x1, -126.f);
+    const uint64_t xc = f2_pack(x0, x1);
+    const uint64_t magic = f2_pack(12582912.f, 12582912.f);
+    const uint64_t xf = f2_add_rm(xc, magic);
+    const uint64_t fr = f2_sub(xc, f2_sub(xf, magic));
+    uint64_t y = f2_fma(f2_pack(0.07806939631700516f, 0.07806939631700516f), fr, f2_pack(0.22593535482883453f, 0.22593535482883453f));
+    y = f2_fma(y, fr, f2_pack(0.6959162950515747f, 0.6959162950515747f));
+    y = f2_fma(y, fr, f2_pack(0.9999210238456726f, 0.9999210238456726f));
+    uint32_t n0, n1, y0, y1;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(n0), "=r"(n1) : "l"(xf));
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(y0), "=r"(y1) : "l"(y));
+    p0 = __uint_as_float(y0 + (n0 << 23));
+    p1 = __uint_as_float(y1 + (n1 << 23));
+}
 
 template <int D>
 struct Cfg {
@@ -148,10 +175,13 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     volatile int* abort_p = &abort_flag;
+    // the softmax warpgroups hold a whole row of S in registers; the third warpgroup gives them its share
 
     const int allowed0 = tiles_allowed(p, row0, 0);
     const int allowed1 = tiles_allowed(p, row0, 1);
 
+    if (warp >= 8) {
+    setmaxnreg_dec<kOtherRegs>();
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -199,27 +229,33 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         if (lane == 0) {
             const uint32_t idesc_qk = make_idesc_bf16(kQTile, kTileN, 0, 0);
             const uint32_t idesc_pv = make_idesc_bf16(kQTile, D, 0, 1);
-            const uint32_t q_addr = smem_u32(sQ), ring_addr = smem_u32(sRing);
+            // Descriptors are built once; per MMA only the 14-bit address field of the low word moves
+            // (one 32-bit add of a compile-time constant), which keeps this single thread ahead of the tensor pipe.
+            const uint64_t q_desc = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
+            const uint64_t k_desc = make_smem_desc_sw128(smem_u32(sRing), 16, 1024);            // K-major tile (K)
+            const uint64_t v_desc = make_smem_desc_sw128(smem_u32(sRing), kQTile * 128, 1024);  // MN-major tile (V)
+            const uint32_t desc_hi = (uint32_t)(q_desc >> 32);        // identical for all three
+            const uint32_t q_lo[2] = {(uint32_t)q_desc, (uint32_t)q_desc + (C::kTileBytes >> 4)};
+            const uint32_t k_lo0 = (uint32_t)k_desc, v_lo0 = (uint32_t)v_desc;
+            const uint32_t tS0 = tmem_base + C::kColS, tO0 = tmem_base + C::kColO;
             uint32_t it = 0, seg_idx = 0;
             uint32_t n_pv[2] = {0, 0};
             bool ok = true;
             auto issue_qk = [&](int i, uint32_t k_slot) {
-                const uint32_t a0 = q_addr + i * C::kTileBytes, b0 = ring_addr + k_slot * C::kTileBytes;
+                const uint32_t a_lo = q_lo[i], b_lo = k_lo0 + k_slot * (C::kTileBytes >> 4), d = tS0 + i * kTileN;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * (kQTile * 128) + (kk & 3) * 32;
-                    mma_ss(tmem_base + C::kColS + i * kTileN, make_smem_desc_sw128(a0 + off, 16, 1024),
-                           make_smem_desc_sw128(b0 + off, 16, 1024), idesc_qk, kk > 0);
+                    const uint32_t off16 = ((kk >> 2) * (kQTile * 128) + (kk & 3) * 32) >> 4;
+                    mma_ss_parts(d, a_lo + off16, b_lo + off16, desc_hi, idesc_qk, kk > 0);
                 }
                 tc_commit(&s_full[i]);
             };
             auto issue_pv_half = [&](int i, uint32_t v_slot, bool accumulate, int half) {
-                const uint32_t b0 = ring_addr + v_slot * C::kTileBytes;
+                const uint32_t b_lo = v_lo0 + v_slot * (C::kTileBytes >> 4), d = tO0 + i * D, a = tS0 + i * kTileN;
 #pragma unroll
                 for (int k4 = 0; k4 < kTileN / 32; ++k4) {
                     const int kk = half * (kTileN / 32) + k4;
-                    mma_ts(tmem_base + C::kColO + i * D, tmem_base + C::kColS + i * kTileN + kk * 8,
-                           make_smem_desc_sw128(b0 + kk * 2048, kQTile * 128, 1024), idesc_pv, (accumulate || kk > 0) ? 1u : 0u);
+                    mma_ts_parts(d, a + kk * 8, b_lo + kk * (2048 >> 4), desc_hi, idesc_pv, (accumulate || kk > 0) ? 1u : 0u);
                 }
                 if (half == 1) tc_commit(&pv_done[i]);
             };
@@ -277,8 +313,10 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 ++seg_idx;
             }
         }
+    }
     } else {
         // ------------------------------------------------------------------ softmax warpgroups (one per Q tile)
+        setmaxnreg_inc<kSoftmaxRegs>();
         const int i = warp >> 2;                           // Q tile
         const int r = (warp & 3) * 32 + lane;              // row inside the Q tile == TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
@@ -308,26 +346,21 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 const int k0 = (s.t_begin + j) * kTileN;
                 const bool masked = k0 + kTileN > lim_warp;   // warp-uniform: some column of some lane is masked
                 const int nvalid = lim_row - k0;              // columns [0, nvalid) of this tile are allowed for this row
-                // pass 1: row maximum of the tile (the load of chunk c+1 is in flight while chunk c is reduced)
-                float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};   // independent chains
-                {
-                    uint32_t buf[2][32];
-                    tmem_ld32_async(tS, buf[0]);
+                // the whole row of S (128 fp32) comes into registers once
+                uint32_t sv[kTileN / 32][32];
 #pragma unroll
-                    for (int c = 0; c < kTileN / 32; ++c) {
-                        uint32_t(&cur)[32] = buf[c & 1];
-                        tmem_wait_ld(cur);
-                        if (c + 1 < kTileN / 32) tmem_ld32_async(tS + (c + 1) * 32, buf[(c + 1) & 1]);
-                        if (masked) {
+                for (int c = 0; c < kTileN / 32; ++c) tmem_ld32_async(tS + c * 32, sv[c]);
 #pragma unroll
-                            for (int e = 0; e < 32; ++e)
-                                if (c * 32 + e >= nvalid) cur[e] = 0xff800000u;   // -inf
-                        }
+                for (int c = 0; c < kTileN / 32; ++c) tmem_wait_ld(sv[c]);
+                if (masked) {
 #pragma unroll
-                        for (int e = 0; e < 16; ++e)
-                            mx[e & 3] = max3(mx[e & 3], __uint_as_float(cur[2 * e]), __uint_as_float(cur[2 * e + 1]));
-                    }
+                    for (int e = 0; e < kTileN; ++e)
+                        if (e >= nvalid) sv[e >> 5][e & 31] = 0xff800000u;   // -inf
                 }
+                float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};   // independent chains
+#pragma unroll
+                for (int e = 0; e < kTileN / 2; ++e)
+                    mx[e & 3] = max3(mx[e & 3], __uint_as_float(sv[e >> 4][(2 * e) & 31]), __uint_as_float(sv[e >> 4][(2 * e + 1) & 31]));
                 const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
                 const float m_new = fmaxf(m_ref, tmax * p.scale_log2e);
                 const bool need = m_new > m_ref + kRescaleThreshold;
@@ -339,12 +372,12 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                         if (!ok) break;
                         tc_fence_after();
 #pragma unroll
-                        for (int c = 0; c < D / 32; ++c) {
-                            uint32_t o[32];
-                            tmem_ld32(tO + c * 32, o);
+                        for (int c = 0; c < D / 8; ++c) {      // narrow pieces: the row of S stays in registers meanwhile
+                            uint32_t o[8];
+                            tmem_ld8(tO + c * 8, o);
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                            tmem_st32(tO + c * 32, o);
+                            for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                            tmem_st8(tO + c * 8, o);
                         }
                     }
                     const uint64_t alpha2 = f2_pack(alpha, alpha);
@@ -353,29 +386,35 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     if (need) m_ref = m_new;
                 }
                 const float m_use = m_ref == -CUDART_INF_F ? 0.f : m_ref;
-                // pass 2: P = 2^(s*scale - m), written as bf16 over the columns of S already consumed
+                // P = 2^(s*scale - m) as bf16 over the columns of S; kPolyPairs of every 16 pairs take the
+                // polynomial route (FMA pipe), the rest the special-function unit
                 {
                     const uint64_t scale2 = f2_pack(p.scale_log2e, p.scale_log2e), negm2 = f2_pack(-m_use, -m_use);
-                    uint32_t buf[2][32];
-                    tmem_ld32_async(tS, buf[0]);
 #pragma unroll
                     for (int c = 0; c < kTileN / 32; ++c) {
-                        uint32_t(&cur)[32] = buf[c & 1];
-                        tmem_wait_ld(cur);
-                        if (c + 1 < kTileN / 32) tmem_ld32_async(tS + (c + 1) * 32, buf[(c + 1) & 1]);
-                        if (masked) {
+                        float pe[32];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const uint64_t x2 = f2_fma(f2_pack_bits(sv[c][2 * e], sv[c][2 * e + 1]), scale2, negm2);
+                            if ((e % 16) * kPolyPairs / 16 != ((e % 16) + 1) * kPolyPairs / 16) {
+                                exp2_poly2(x2, pe[2 * e], pe[2 * e + 1]);
+                            } else {
+                                float x0, x1;
+                                f2_unpack(x2, x0, x1);
+                                pe[2 * e] = ex2(x0);
+                                pe[2 * e + 1] = ex2(x1);
+                            }
+                        }
+                        if (masked) {          // the polynomial gives 2^-126, not 0, for a masked column
 #pragma unroll
                             for (int e = 0; e < 32; ++e)
-                                if (c * 32 + e >= nvalid) cur[e] = 0xff800000u;
+                                if (c * 32 + e >= nvalid) pe[e] = 0.f;
                         }
                         uint32_t pk[16];
 #pragma unroll
                         for (int e = 0; e < 16; ++e) {
-                            float x0, x1;
-                            f2_unpack(f2_fma(f2_pack_bits(cur[2 * e], cur[2 * e + 1]), scale2, negm2), x0, x1);
-                            const float p0 = ex2(x0), p1 = ex2(x1);
-                            l2[e & 1] = f2_add(l2[e & 1], f2_pack(p0, p1));
-                            pk[e] = pack_bf16x2(p0, p1);
+                            l2[e & 1] = f2_add(l2[e & 1], f2_pack(pe[2 * e], pe[2 * e + 1]));
+                            pk[e] = pack_bf16x2(pe[2 * e], pe[2 * e + 1]);
                         }
                         tmem_st16(tS + c * 16, pk);
                         if (c == kTileN / 64 - 1) {        // first 64 keys are in place: let the PV MMAs start on them
