@@ -105,6 +105,10 @@ struct SegmentWalker {
     }
 };
 
+__device__ __forceinline__ void commit_elected(uint64_t* bar) {
+    if (elect_one()) tc_commit(bar);
+}
+
 // Number of key tiles Q tile `i` of this CTA may use at all (0 if the tile lies beyond W).
 __device__ __forceinline__ int tiles_allowed(const Params& p, int row0, int i) {
     const int r_first = row0 + i * kQTile;
@@ -226,18 +230,22 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         }
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // The whole warp walks the schedule (every value below is the same in all lanes) and one elected
+        // lane issues: descriptors and addresses then live in uniform registers and an MMA costs a few
+        // instructions, which matters because the tensor pipe takes the next MMA only when it has room.
+        {
             const uint32_t idesc_qk = make_idesc_bf16(kQTile, kTileN, 0, 0);
             const uint32_t idesc_pv = make_idesc_bf16(kQTile, D, 0, 1);
             // Descriptors are built once; per MMA only the 14-bit address field of the low word moves
-            // (one 32-bit add of a compile-time constant), which keeps this single thread ahead of the tensor pipe.
+            // (one 32-bit add of a compile-time constant).
             const uint64_t q_desc = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
             const uint64_t k_desc = make_smem_desc_sw128(smem_u32(sRing), 16, 1024);            // K-major tile (K)
             const uint64_t v_desc = make_smem_desc_sw128(smem_u32(sRing), kQTile * 128, 1024);  // MN-major tile (V)
             const uint32_t desc_hi = (uint32_t)(q_desc >> 32);        // identical for all three
             const uint32_t q_lo[2] = {(uint32_t)q_desc, (uint32_t)q_desc + (C::kTileBytes >> 4)};
             const uint32_t k_lo0 = (uint32_t)k_desc, v_lo0 = (uint32_t)v_desc;
-            const uint32_t tS0 = tmem_base + C::kColS, tO0 = tmem_base + C::kColO;
+            const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
+            const uint32_t tS0 = tmem_u + C::kColS, tO0 = tmem_u + C::kColO;
             uint32_t it = 0, seg_idx = 0;
             uint32_t n_pv[2] = {0, 0};
             bool ok = true;
@@ -246,18 +254,18 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off16 = ((kk >> 2) * (kQTile * 128) + (kk & 3) * 32) >> 4;
-                    mma_ss_parts(d, a_lo + off16, b_lo + off16, desc_hi, idesc_qk, kk > 0);
+                    if (elect_one()) mma_ss_parts(d, a_lo + off16, b_lo + off16, desc_hi, idesc_qk, kk > 0);
                 }
-                tc_commit(&s_full[i]);
+                commit_elected(&s_full[i]);
             };
             auto issue_pv_half = [&](int i, uint32_t v_slot, bool accumulate, int half) {
                 const uint32_t b_lo = v_lo0 + v_slot * (C::kTileBytes >> 4), d = tO0 + i * D, a = tS0 + i * kTileN;
 #pragma unroll
                 for (int k4 = 0; k4 < kTileN / 32; ++k4) {
                     const int kk = half * (kTileN / 32) + k4;
-                    mma_ts_parts(d, a + kk * 8, b_lo + kk * (2048 >> 4), desc_hi, idesc_pv, (accumulate || kk > 0) ? 1u : 0u);
+                    if (elect_one()) mma_ts_parts(d, a + kk * 8, b_lo + kk * (2048 >> 4), desc_hi, idesc_pv, (accumulate || kk > 0) ? 1u : 0u);
                 }
-                if (half == 1) tc_commit(&pv_done[i]);
+                if (half == 1) commit_elected(&pv_done[i]);
             };
             SegmentWalker walk(p, g);
             Segment s;
@@ -266,50 +274,50 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 const int cnt = c0 > c1 ? c0 : c1;
                 if (cnt == 0) continue;
                 const int cq[2] = {c0, c1};
-                ok = mbar_wait(q_full, seg_idx & 1, abort_p);
+                ok = __all_sync(0xffffffffu, mbar_wait(q_full, seg_idx & 1, abort_p));
                 if (!ok) break;
                 // first K tile
                 uint32_t k_slot = it % C::kSlots;
-                ok = mbar_wait(&kv_full[k_slot], (it / C::kSlots) & 1, abort_p);
+                ok = __all_sync(0xffffffffu, mbar_wait(&kv_full[k_slot], (it / C::kSlots) & 1, abort_p));
                 if (!ok) break;
                 tc_fence_after();
                 for (int i = 0; i < 2; ++i)
                     if (cq[i] > 0) issue_qk(i, k_slot);
-                tc_commit(&kv_empty[k_slot]);
+                commit_elected(&kv_empty[k_slot]);
                 ++it;
                 for (int j = 0; j < cnt && ok; ++j) {
                     const uint32_t v_slot = it % C::kSlots;
-                    ok = mbar_wait(&kv_full[v_slot], (it / C::kSlots) & 1, abort_p);
+                    ok = __all_sync(0xffffffffu, mbar_wait(&kv_full[v_slot], (it / C::kSlots) & 1, abort_p));
                     if (!ok) break;
                     ++it;
                     const bool have_next = j + 1 < cnt;
                     uint32_t nk_slot = 0;
                     if (have_next) {
                         nk_slot = it % C::kSlots;
-                        ok = mbar_wait(&kv_full[nk_slot], (it / C::kSlots) & 1, abort_p);
+                        ok = __all_sync(0xffffffffu, mbar_wait(&kv_full[nk_slot], (it / C::kSlots) & 1, abort_p));
                         if (!ok) break;
                         ++it;
                     }
                     tc_fence_after();
                     for (int i = 0; i < 2 && ok; ++i) {
                         if (j < cq[i]) {
-                            ok = mbar_wait(&p_half[i], n_pv[i] & 1, abort_p);
+                            ok = __all_sync(0xffffffffu, mbar_wait(&p_half[i], n_pv[i] & 1, abort_p));
                             if (!ok) break;
                             tc_fence_after();
                             issue_pv_half(i, v_slot, j > 0, 0);
-                            ok = mbar_wait(&p_full[i], n_pv[i] & 1, abort_p);
+                            ok = __all_sync(0xffffffffu, mbar_wait(&p_full[i], n_pv[i] & 1, abort_p));
                             if (!ok) break;
                             tc_fence_after();
                             issue_pv_half(i, v_slot, j > 0, 1);
                             ++n_pv[i];
                         }
-                        if (i == 1) tc_commit(&kv_empty[v_slot]);
+                        if (i == 1) commit_elected(&kv_empty[v_slot]);
                         if (have_next && j + 1 < cq[i]) issue_qk(i, nk_slot);
-                        if (have_next && i == 1) tc_commit(&kv_empty[nk_slot]);
+                        if (have_next && i == 1) commit_elected(&kv_empty[nk_slot]);
                     }
                 }
                 if (!ok) break;
-                tc_commit(q_empty);
+                commit_elected(q_empty);
                 ++seg_idx;
             }
         }
