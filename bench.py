@@ -391,7 +391,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--decode-steps", type=int, default=0, help="timed decode steps (default: max(steps, 64))")
-    ap.add_argument("--shape", default="", help="custom forward shape B,H,N,W,d[,causal] instead of --workload (profiling)")
+    ap.add_argument("--shape", default="", help="custom shape B,H,N,W,d[,causal] instead of the named workload (profiling); with --workload decode, N is the "
+                         "number of cached rows and W the number of decode steps available")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "tlin" else args.warmup
     if args.decode_steps <= 0:
@@ -415,7 +416,7 @@ def main():
     if args.shape:
         v = [int(x) for x in args.shape.split(",")]
         wl = synth.Workload("custom_" + args.shape.replace(",", "_"), v[0], v[1], v[4], v[2], v[3], seed=9,
-                            causal_window=v[5] if len(v) > 5 else 1)
+                            causal_window=v[5] if len(v) > 5 else 1, decode=args.workload == "decode")
     with_cpu = (not args.no_cpu) and world == 1
     runner = run_decode if wl.decode else run_forward
     main_res = runner(wl, args, rank, world, device, peaks, with_cpu)
