@@ -142,12 +142,19 @@ typedef struct {
     int32_t tile_n;        /* keys per tile                                                  */
     int32_t q_tiles;       /* ceil(W / tile_m): CTAs that share one key range                */
     int32_t key_tiles;     /* ceil(N / tile_n) per (b,h)                                     */
-    int32_t n_groups;      /* groups of q_tiles CTAs; group g streams units [start(g), start(g+1)) */
-    int32_t n_ctas;        /* n_groups * q_tiles                                             */
-    int64_t total_units;   /* B*H*key_tiles; unit u = (bh = u / key_tiles, tile = u % key_tiles) */
+    int32_t n_groups;      /* group g owns units [start(g), start(g+1)); see `schedule`       */
+    int32_t n_ctas;        /* schedule 0: n_groups * q_tiles; schedule 1: n_groups            */
+    int64_t total_units;   /* schedule 0: B*H*key_tiles, unit u = (bh = u / key_tiles, tile = u % key_tiles);
+                              schedule 1: B*H*q_tiles,  unit u = (bh = u / q_tiles,  q tile = u % q_tiles) */
     int32_t uses_workspace;/* 1 if any (b,h) is split between groups                         */
     int32_t tensor_path;   /* 1 = tcgen05 kernel, 0 = CUDA-core kernel                       */
     int64_t workspace_bytes;
+    int32_t schedule;      /* 0: a group of q_tiles CTAs streams a range of (b,h,key tile) units, the key range of
+                              a (b,h) may be split between groups (few query rows, long context: Section 3,
+                              focused attention and the generation window);
+                              1: every CTA works through whole (b,h,query tile) problems, keys never split
+                              (many query rows, short context: the restoring cross-attention of Section 3) */
+    int32_t reserved;
 } tlin_fwd_plan;
 
 typedef struct {

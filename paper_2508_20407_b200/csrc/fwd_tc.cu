@@ -81,21 +81,35 @@ struct Params {
     long long total_units;
     int n_groups, q_tiles, key_tiles;
     int N, W, causal;
+    int schedule;         // 0: groups of q_tiles CTAs stream key ranges; 1: every CTA walks whole (b,h,q-tile) problems
     float scale_log2e;
 };
 
-// Segments of a group's unit range: one per (b,h) it touches.
-struct Segment { int bh, t_begin, t_end; };
+// Work of one CTA as a list of segments: a (b,h), a pair of Q tiles (256 query rows) and a range of key tiles.
+// Schedule 0: CTA = (group, q-tile pair); the group's unit range [u, u1) over (b,h,key tile) is cut at the (b,h)
+// borders.  Schedule 1: the units are whole (b,h,q-tile pair) problems and a CTA takes a contiguous run of them.
+struct Segment { int bh, qt, t_begin, t_end; };
 
 struct SegmentWalker {
     long long u, u1;
-    int T;
-    __device__ SegmentWalker(const Params& p, int g) : T(p.key_tiles) {
+    int T, q_tiles, qt_fixed, schedule;
+    __device__ SegmentWalker(const Params& p) : T(p.key_tiles), q_tiles(p.q_tiles), schedule(p.schedule) {
+        const int g = schedule == 0 ? (int)(blockIdx.x / p.q_tiles) : (int)blockIdx.x;
+        qt_fixed = schedule == 0 ? (int)(blockIdx.x - g * p.q_tiles) : 0;
         u = (long long)(((unsigned long long)g * (unsigned long long)p.total_units) / (unsigned)p.n_groups);
         u1 = (long long)(((unsigned long long)(g + 1) * (unsigned long long)p.total_units) / (unsigned)p.n_groups);
     }
     __device__ bool next(Segment& s) {
         if (u >= u1) return false;
+        if (schedule != 0) {
+            s.bh = (int)(u / q_tiles);
+            s.qt = (int)(u - (long long)s.bh * q_tiles);
+            s.t_begin = 0;
+            s.t_end = T;
+            ++u;
+            return true;
+        }
+        s.qt = qt_fixed;
         s.bh = (int)(u / T);
         s.t_begin = (int)(u - (long long)s.bh * T);
         const long long left = u1 - u;
@@ -145,9 +159,6 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     __shared__ int abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int g = blockIdx.x / p.q_tiles;
-    const int qt = blockIdx.x - g * p.q_tiles;
-    const int row0 = qt * kTileM;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -181,9 +192,6 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     volatile int* abort_p = &abort_flag;
     // the softmax warpgroups hold a whole row of S in registers; the third warpgroup gives them its share
 
-    const int allowed0 = tiles_allowed(p, row0, 0);
-    const int allowed1 = tiles_allowed(p, row0, 1);
-
     if (warp >= 8) {
     setmaxnreg_dec<kOtherRegs>();
     if (warp == kProducerWarp) {
@@ -192,10 +200,11 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             uint32_t it = 0;           // ring counter
             uint32_t seg_idx = 0;
             bool ok = true;
-            SegmentWalker walk(p, g);
+            SegmentWalker walk(p);
             Segment s;
             while (ok && walk.next(s)) {
-                const int c0 = seg_count(s, allowed0), c1 = seg_count(s, allowed1);
+                const int row0 = s.qt * kTileM;
+                const int c0 = seg_count(s, tiles_allowed(p, row0, 0)), c1 = seg_count(s, tiles_allowed(p, row0, 1));
                 const int cnt = c0 > c1 ? c0 : c1;
                 if (cnt == 0) continue;
                 if (seg_idx > 0) ok = mbar_wait(q_empty, (seg_idx - 1) & 1, abort_p);
@@ -267,10 +276,11 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 }
                 if (half == 1) commit_elected(&pv_done[i]);
             };
-            SegmentWalker walk(p, g);
+            SegmentWalker walk(p);
             Segment s;
             while (ok && walk.next(s)) {
-                const int c0 = seg_count(s, allowed0), c1 = seg_count(s, allowed1);
+                const int row0 = s.qt * kTileM;
+                const int c0 = seg_count(s, tiles_allowed(p, row0, 0)), c1 = seg_count(s, tiles_allowed(p, row0, 1));
                 const int cnt = c0 > c1 ? c0 : c1;
                 if (cnt == 0) continue;
                 const int cq[2] = {c0, c1};
@@ -284,6 +294,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 for (int i = 0; i < 2; ++i)
                     if (cq[i] > 0) issue_qk(i, k_slot);
                 commit_elected(&kv_empty[k_slot]);
+                if (cnt == 1) commit_elected(q_empty);      // the segment's last use of Q is issued: its successor may load
                 ++it;
                 for (int j = 0; j < cnt && ok; ++j) {
                     const uint32_t v_slot = it % C::kSlots;
@@ -313,11 +324,15 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                         }
                         if (i == 1) commit_elected(&kv_empty[v_slot]);
                         if (have_next && j + 1 < cq[i]) issue_qk(i, nk_slot);
-                        if (have_next && i == 1) commit_elected(&kv_empty[nk_slot]);
+                        if (have_next && i == 1) {
+                            commit_elected(&kv_empty[nk_slot]);
+                            // Q is last read by the S of the segment's last key tile: releasing it here lets the
+                            // producer fetch the next segment's Q while this one finishes
+                            if (j + 2 == cnt) commit_elected(q_empty);
+                        }
                     }
                 }
                 if (!ok) break;
-                commit_elected(q_empty);
                 ++seg_idx;
             }
         }
@@ -330,19 +345,19 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_base + lane_addr + C::kColS + i * kTileN;
         const uint32_t tO = tmem_base + lane_addr + C::kColO + i * D;
-        const int row = row0 + i * kQTile + r;             // row inside W (may lie beyond W: computed, never stored)
-        const int allowed_i = i == 0 ? allowed0 : allowed1;
-        // keys visible to this row, and to the first row of this warp (the smallest in the warp)
-        const long long lim_row_ll = p.causal ? (long long)p.N - p.W + row + 1 : (long long)p.N;
-        const int lim_row = (int)(lim_row_ll < p.N ? lim_row_ll : p.N);
-        const long long lim_warp_ll = p.causal ? (long long)p.N - p.W + (row - lane) + 1 : (long long)p.N;
-        const int lim_warp = (int)(lim_warp_ll < p.N ? lim_warp_ll : p.N);
-
         uint32_t n = 0;     // tiles processed by this warpgroup (phase counter of s_full/p_full/pv_done)
         bool ok = true;
-        SegmentWalker walk(p, g);
+        SegmentWalker walk(p);
         Segment s;
         while (ok && walk.next(s)) {
+            const int row0 = s.qt * kTileM;
+            const int row = row0 + i * kQTile + r;         // row inside W (may lie beyond W: computed, never stored)
+            const int allowed_i = tiles_allowed(p, row0, i);
+            // keys visible to this row, and to the first row of this warp (the smallest in the warp)
+            const long long lim_row_ll = p.causal ? (long long)p.N - p.W + row + 1 : (long long)p.N;
+            const int lim_row = (int)(lim_row_ll < p.N ? lim_row_ll : p.N);
+            const long long lim_warp_ll = p.causal ? (long long)p.N - p.W + (row - lane) + 1 : (long long)p.N;
+            const int lim_warp = (int)(lim_warp_ll < p.N ? lim_warp_ll : p.N);
             const int cnt_i = seg_count(s, allowed_i);
             float m_ref = -CUDART_INF_F;
             uint64_t l2[2] = {0ull, 0ull};          // four partial row sums as two packed fp32 pairs
@@ -478,6 +493,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 if (store && p.lse != nullptr) p.lse[(long long)s.bh * p.W + row] = lse_val;
             } else {
                 // partial result -> workspace slot (0: first segment of this CTA's range, 1: a later one)
+                const int g = (int)(blockIdx.x / p.q_tiles);          // partial segments exist only under schedule 0
                 const long long u_first = (long long)(((unsigned long long)g * (unsigned long long)p.total_units) / (unsigned)p.n_groups);
                 const int slot = s.bh == (int)(u_first / p.key_tiles) ? 0 : 1;
                 float* base = p.ws + ((long long)blockIdx.x * 2 + slot) * (long long)kTileM * (D + 1);
@@ -653,7 +669,7 @@ int launch_d(const void* q, const void* k, const void* v, void* out, float* lse,
     p.out = out; p.lse = lse; p.ws = ws; p.status = status_word();
     if (!p.status) return TLIN_ERR_CUDA;
     p.total_units = plan.total_units; p.n_groups = plan.n_groups; p.q_tiles = plan.q_tiles; p.key_tiles = plan.key_tiles;
-    p.N = N; p.W = W; p.causal = causal;
+    p.N = N; p.W = W; p.causal = causal; p.schedule = plan.schedule;
     p.scale_log2e = kLog2e / sqrtf((float)D);
     static std::once_flag attr_once;
     static cudaError_t attr_err = cudaSuccess;

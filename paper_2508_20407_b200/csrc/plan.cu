@@ -65,6 +65,21 @@ extern "C" int tlin_plan_forward(int B, int H, int N, int W, int d, int causal_w
     p.tile_n = kTileN;
     p.q_tiles = (W + p.tile_m - 1) / p.tile_m;
     p.key_tiles = (N + p.tile_n - 1) / p.tile_n;
+    // Many query tiles and a short key range (the restoring cross-attention of Section 3: every history token
+    // queries the few summary tokens): splitting keys would leave each group a fraction of a problem and every
+    // CTA a merge; instead each CTA works through whole (b,h,query tile) problems, as many as the SMs share out evenly.
+    if (p.q_tiles * 2 > num_sms || (p.key_tiles <= 16 && bh * p.q_tiles >= 2 * (int64_t)num_sms)) {
+        p.schedule = 1;
+        p.total_units = bh * p.q_tiles;
+        if (p.total_units > INT32_MAX) return TLIN_ERR_UNSUPPORTED;
+        int64_t ctas = num_sms < p.total_units ? num_sms : p.total_units;
+        p.n_groups = (int32_t)ctas;
+        p.n_ctas = (int32_t)ctas;
+        p.uses_workspace = 0;
+        p.workspace_bytes = 0;
+        *plan = p;
+        return TLIN_OK;
+    }
     p.total_units = bh * p.key_tiles;
     int64_t groups = num_sms / p.q_tiles;
     if (groups < 1) groups = 1;

@@ -94,7 +94,7 @@ def test_forward_plan_partitions_the_units(B, H, N, W, d, causal):
         p = tl.tlin_plan_forward(B, H, N, W, d, causal, num_sms=148)
     finally:
         tl.tlin_set_forward_impl(prev)
-    assert p.tensor_path == 1 and p.tile_n == 128
+    assert p.tensor_path == 1 and p.tile_n == 128 and p.schedule == 0
     assert p.q_tiles == -(-W // p.tile_m) and p.key_tiles == -(-N // p.tile_n)
     assert p.total_units == B * H * p.key_tiles
     assert 1 <= p.n_groups <= p.total_units and p.n_ctas == p.n_groups * p.q_tiles
@@ -107,6 +107,32 @@ def test_forward_plan_partitions_the_units(B, H, N, W, d, causal):
     assert bool(p.uses_workspace) == split
     assert p.workspace_bytes == (p.n_ctas * 2 * p.tile_m * (d + 1) * 4 if split else 0)
     assert tl.workspace_bytes_forward(B, H, N, W, d, causal) in (0, p.workspace_bytes) or tl.tlin_set_forward_impl(0) == 0
+
+
+WIDE = [(1, 32, 1024, 130048, 128, 0), (1, 32, 512, 32256, 128, 0), (2, 3, 300, 40000, 64, 0), (8, 16, 1024, 1024, 64, 1),
+        (8, 16, 1024, 1024, 64, 0)]
+
+
+@pytest.mark.parametrize("B,H,N,W,d,causal", WIDE)
+def test_forward_plan_many_queries_few_keys(B, H, N, W, d, causal):
+    """Many query tiles over a short key range: whole (b,h,query tile) problems per CTA, keys never split."""
+    prev = tl.tlin_set_forward_impl(2)
+    try:
+        p = tl.tlin_plan_forward(B, H, N, W, d, causal, num_sms=148)
+    finally:
+        tl.tlin_set_forward_impl(prev)
+    assert p.tensor_path == 1 and p.schedule == 1
+    assert p.q_tiles == -(-W // p.tile_m) and p.key_tiles == -(-N // p.tile_n)
+    assert p.total_units == B * H * p.q_tiles
+    assert p.n_ctas == p.n_groups == min(148, p.total_units)
+    assert p.uses_workspace == 0 and p.workspace_bytes == 0
+    starts = [tl.tlin_plan_group_start(p, g) for g in range(p.n_groups + 1)]
+    assert starts[0] == 0 and starts[-1] == p.total_units
+    sizes = np.diff(starts)
+    assert (sizes >= 1).all() and sizes.max() - sizes.min() <= 1
+    # every (b,h,query tile) problem belongs to exactly one CTA and covers all its key tiles:
+    # the evaluated pairs are the method's (Appendix A: restoring cross-attention costs D*(N-W_og)*W_oh)
+    assert sum(int(x) for x in sizes) * p.key_tiles == B * H * p.q_tiles * p.key_tiles
 
 
 def test_forward_plan_fallback_path_never_splits():

@@ -89,6 +89,32 @@ def test_fp32_path(B, H, N, W, d, causal):
     full_compare(wl, 0, kind="f32")
 
 
+@pytest.mark.parametrize("B,H,N,W,d,causal", [(1, 2, 256, 40000, 128, 0), (2, 1, 300, 38000, 64, 0), (5, 16, 1024, 1000, 64, 1),
+                                              (1, 160, 384, 512, 64, 0)])
+def test_many_queries_few_keys_schedule(B, H, N, W, d, causal):
+    """Restoring cross-attention shape (Section 3): every history token queries a few summary tokens.
+    The planner hands whole (b,h,query tile) problems to the CTAs; parity on sampled heads and rows."""
+    wl = synth.Workload("wide", B, H, d, N, W, seed=300 + N, causal_window=causal)
+    assert tl.tlin_plan_forward(B, H, N, W, d, causal).schedule == 1
+    q, k, v = synth.forward_inputs(wl, device=DEV)
+    out, lse = run_impl(2 if TC_AVAILABLE else 1, tl.tlin_attn_forward, q, k, v, causal_window=causal)
+    assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
+    rng = np.random.default_rng(N)
+    for (b, h) in {(0, 0), (B - 1, H - 1)}:
+        rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, W - 1], rng.integers(0, W, 250)]))
+        qs = q[b:b + 1, h:h + 1, rows].contiguous().cpu()
+        if causal:      # row i sees keys j <= N - W + i: compare row by row through the unmasked oracle call
+            for idx, i in enumerate(rows[:40]):
+                lim = N - W + int(i) + 1
+                if lim < 1:
+                    continue
+                ref, ref_lse = oracle.attn_forward(qs[:, :, idx:idx + 1], k[b:b + 1, h:h + 1, :lim].cpu(), v[b:b + 1, h:h + 1, :lim].cpu(), 0)
+                parity.check(out[b, h, int(i)].float().cpu().numpy()[None], lse[b, h, int(i)].cpu().numpy()[None], ref.reshape(1, -1), ref_lse.reshape(1), "bf16", f"wide causal row {i}")
+        else:
+            ref, ref_lse = oracle.attn_forward(qs, k[b:b + 1, h:h + 1].cpu(), v[b:b + 1, h:h + 1].cpu(), 0)
+            parity.check(out[b, h, rows].float().cpu().numpy(), lse[b, h, rows].cpu().numpy(), ref[0, 0], ref_lse[0, 0], "bf16", f"wide head {(b, h)}")
+
+
 def test_bf16_fallback_head_dims():
     for d in (8, 72, 256):
         full_compare(synth.Workload("odd_d", 1, 2, d, 300, 33, seed=d), 0)
