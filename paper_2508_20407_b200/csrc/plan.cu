@@ -65,10 +65,32 @@ extern "C" int tlin_plan_forward(int B, int H, int N, int W, int d, int causal_w
     p.tile_n = kTileN;
     p.q_tiles = (W + p.tile_m - 1) / p.tile_m;
     p.key_tiles = (N + p.tile_n - 1) / p.tile_n;
-    // Many query tiles and a short key range (the restoring cross-attention of Section 3: every history token
-    // queries the few summary tokens): splitting keys would leave each group a fraction of a problem and every
-    // CTA a merge; instead each CTA works through whole (b,h,query tile) problems, as many as the SMs share out evenly.
-    if (p.q_tiles * 2 > num_sms || (p.key_tiles <= 16 && bh * p.q_tiles >= 2 * (int64_t)num_sms)) {
+    // Two ways to share the work out (both evaluate exactly the same (query,key) pairs):
+    //   schedule 0: groups of q_tiles CTAs stream ranges of (b,h,key tile) units; a (b,h) may be split between
+    //               groups, whose partial results a second kernel merges.  Fills the SMs however few (b,h) there are,
+    //               and the CTAs of a group read each K/V tile at the same time (once from HBM).
+    //   schedule 1: every CTA works through whole (b,h,query tile) problems; no split, no merge, but a K/V tile
+    //               is read by the q_tiles problems of its (b,h) at unrelated times, so K and V have to stay in L2.
+    // Costs in key-tile times per CTA; the constants (merge pass ~ 6 tiles, start/finish of a problem ~ 2 tiles)
+    // are measured on B200.
+    bool wide = false;
+    {
+        int64_t groups0 = num_sms / p.q_tiles;
+        if (groups0 < 1) groups0 = 1;
+        if (groups0 > bh * p.key_tiles) groups0 = bh * p.key_tiles;
+        const int64_t waves0 = (p.q_tiles + num_sms - 1) / num_sms;              // > 1 only if q_tiles exceeds the SMs
+        const int64_t per_group = (bh * p.key_tiles + groups0 - 1) / groups0;
+        const bool splits0 = (bh * p.key_tiles) % groups0 != 0 || (bh * p.key_tiles / groups0) % p.key_tiles != 0;
+        const int64_t segments0 = per_group / p.key_tiles + 1;                   // (b,h) pieces a group walks through
+        const int64_t cost0 = waves0 * (per_group + 2 * segments0) + (splits0 ? 6 : 0);
+        const int64_t problems = bh * p.q_tiles;
+        const int64_t ctas1 = num_sms < problems ? num_sms : problems;
+        const int64_t cost1 = ((problems + ctas1 - 1) / ctas1) * ((int64_t)p.key_tiles + 2);
+        const int64_t kv_bytes = 2 * bh * (int64_t)N * d * 2;
+        const bool kv_in_l2 = p.q_tiles == 1 || kv_bytes <= (int64_t)64 << 20;
+        wide = kv_in_l2 && cost1 < cost0;
+    }
+    if (wide) {
         p.schedule = 1;
         p.total_units = bh * p.q_tiles;
         if (p.total_units > INT32_MAX) return TLIN_ERR_UNSUPPORTED;

@@ -148,6 +148,13 @@ WORKLOADS = {
     "cfg4_vlong": _w("cfg4_vlong", 1, 32, 128, 131072, 1024, 3),
     # cached decode: 65536 cached rows + 256 single-token steps
     "cfg5_decode": _w("cfg5_decode", 8, 32, 128, 65536, 256, 4, decode=True),
+    # --- the other attention layers of a block, at the sizes of the very long configuration (W_oh = W_og = 1024) ---
+    # restoring cross-attention: every history token queries the W_oh summary tokens (unmasked)
+    "restore_vlong": _w("restore_vlong", 1, 32, 128, 1024, 131072 - 1024, 5, causal_window=0),
+    # inner context layer: self-attention among the W_oh summary tokens (unmasked)
+    "inner_self": _w("inner_self", 1, 32, 128, 1024, 1024, 6, causal_window=0),
+    # inner generation layer: W_og window queries over [summary tokens; window], causal inside the window
+    "inner_gen": _w("inner_gen", 1, 32, 128, 2048, 1024, 7, causal_window=1),
 }
 
 Q_ID, K_ID, V_ID, QNEW_ID, KNEW_ID, VNEW_ID = 0, 1, 2, 3, 4, 5

@@ -87,52 +87,67 @@ CONFIGS = [(1, 4, 1024, 128, 64, 1), (4, 16, 8192, 256, 64, 1), (1, 32, 32768, 5
            (1, 32, 131072, 1024, 128, 1), (3, 5, 1000, 77, 128, 0), (1, 1, 100, 100, 64, 1), (2, 2, 129, 1, 64, 1)]
 
 
-@pytest.mark.parametrize("B,H,N,W,d,causal", CONFIGS)
-def test_forward_plan_partitions_the_units(B, H, N, W, d, causal):
+def _plan_tc(B, H, N, W, d, causal):
     prev = tl.tlin_set_forward_impl(2)
     try:
-        p = tl.tlin_plan_forward(B, H, N, W, d, causal, num_sms=148)
+        return tl.tlin_plan_forward(B, H, N, W, d, causal, num_sms=148)
     finally:
         tl.tlin_set_forward_impl(prev)
-    assert p.tensor_path == 1 and p.tile_n == 128 and p.schedule == 0
+
+
+def _check_plan(p, B, H, N, W, d, causal):
+    """Whatever the schedule, the groups partition the units and so cover every (query tile, key tile) once."""
+    assert p.tensor_path == 1 and p.tile_n == 128 and p.schedule in (0, 1)
     assert p.q_tiles == -(-W // p.tile_m) and p.key_tiles == -(-N // p.tile_n)
-    assert p.total_units == B * H * p.key_tiles
-    assert 1 <= p.n_groups <= p.total_units and p.n_ctas == p.n_groups * p.q_tiles
-    assert p.n_ctas <= 148 or p.n_groups == 1
     starts = [tl.tlin_plan_group_start(p, g) for g in range(p.n_groups + 1)]
     assert starts[0] == 0 and starts[-1] == p.total_units
     sizes = np.diff(starts)
     assert (sizes >= 1).all() and sizes.max() - sizes.min() <= 1
-    split = any(s % p.key_tiles for s in starts[1:-1])
-    assert bool(p.uses_workspace) == split
-    assert p.workspace_bytes == (p.n_ctas * 2 * p.tile_m * (d + 1) * 4 if split else 0)
+    if p.schedule == 0:
+        # unit = (b,h,key tile); a group is q_tiles CTAs (one per pair of query tiles) walking the same units
+        assert p.total_units == B * H * p.key_tiles
+        assert 1 <= p.n_groups <= p.total_units and p.n_ctas == p.n_groups * p.q_tiles
+        assert p.n_ctas <= 148 or p.n_groups == 1
+        split = any(s % p.key_tiles for s in starts[1:-1])
+        assert bool(p.uses_workspace) == split
+        assert p.workspace_bytes == (p.n_ctas * 2 * p.tile_m * (d + 1) * 4 if split else 0)
+        covered = int(sizes.sum()) * p.q_tiles
+    else:
+        # unit = whole (b,h,query tile pair) problem: all its key tiles, never split, nothing to merge
+        assert p.total_units == B * H * p.q_tiles
+        assert p.n_ctas == p.n_groups == min(148, p.total_units)
+        assert p.uses_workspace == 0 and p.workspace_bytes == 0
+        covered = int(sizes.sum()) * p.key_tiles
+    assert covered == B * H * p.q_tiles * p.key_tiles
+
+
+@pytest.mark.parametrize("B,H,N,W,d,causal", CONFIGS)
+def test_forward_plan_partitions_the_units(B, H, N, W, d, causal):
+    p = _plan_tc(B, H, N, W, d, causal)
+    _check_plan(p, B, H, N, W, d, causal)
+    if N >= 8192:
+        # few query rows over a long context (focused attention, generation window): key ranges are split
+        assert p.schedule == 0 and p.n_ctas == 148
     assert tl.workspace_bytes_forward(B, H, N, W, d, causal) in (0, p.workspace_bytes) or tl.tlin_set_forward_impl(0) == 0
 
 
 WIDE = [(1, 32, 1024, 130048, 128, 0), (1, 32, 512, 32256, 128, 0), (2, 3, 300, 40000, 64, 0), (8, 16, 1024, 1024, 64, 1),
-        (8, 16, 1024, 1024, 64, 0)]
+        (1, 32, 1024, 1024, 128, 0), (1, 32, 2048, 1024, 128, 1)]
 
 
 @pytest.mark.parametrize("B,H,N,W,d,causal", WIDE)
 def test_forward_plan_many_queries_few_keys(B, H, N, W, d, causal):
-    """Many query tiles over a short key range: whole (b,h,query tile) problems per CTA, keys never split."""
-    prev = tl.tlin_set_forward_impl(2)
-    try:
-        p = tl.tlin_plan_forward(B, H, N, W, d, causal, num_sms=148)
-    finally:
-        tl.tlin_set_forward_impl(prev)
-    assert p.tensor_path == 1 and p.schedule == 1
-    assert p.q_tiles == -(-W // p.tile_m) and p.key_tiles == -(-N // p.tile_n)
-    assert p.total_units == B * H * p.q_tiles
-    assert p.n_ctas == p.n_groups == min(148, p.total_units)
-    assert p.uses_workspace == 0 and p.workspace_bytes == 0
-    starts = [tl.tlin_plan_group_start(p, g) for g in range(p.n_groups + 1)]
-    assert starts[0] == 0 and starts[-1] == p.total_units
-    sizes = np.diff(starts)
-    assert (sizes >= 1).all() and sizes.max() - sizes.min() <= 1
-    # every (b,h,query tile) problem belongs to exactly one CTA and covers all its key tiles:
-    # the evaluated pairs are the method's (Appendix A: restoring cross-attention costs D*(N-W_og)*W_oh)
-    assert sum(int(x) for x in sizes) * p.key_tiles == B * H * p.q_tiles * p.key_tiles
+    """Restoring cross-attention and the inner layers (Section 3): many (b,h,query tile) problems over a short
+    key range go to the CTAs whole; the evaluated pairs are unchanged (Appendix A: D*(N-W_og)*W_oh)."""
+    p = _plan_tc(B, H, N, W, d, causal)
+    _check_plan(p, B, H, N, W, d, causal)
+    assert p.schedule == 1
+
+
+def test_forward_plan_keeps_key_splitting_when_kv_exceed_l2():
+    """Whole problems per CTA would read every K/V tile q_tiles times from HBM once K and V no longer fit in L2."""
+    p = _plan_tc(1, 64, 16384, 1024, 128, 1)        # 512 MB of K and V
+    assert p.schedule == 0
 
 
 def test_forward_plan_fallback_path_never_splits():
