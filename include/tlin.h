@@ -86,6 +86,20 @@ int tlin_decode_step(const void* q_new, const void* k_new, const void* v_new,
                      void* k_cache, void* v_cache, void* out, float* lse,
                      int B, int H, int Ncap, int pos, int d, tlin_stream_t stream);
 
+/* Cached decode step for a batch whose sequences have different lengths (the paper decodes one sequence at a
+ * time, Section 6.3; a served batch holds windows at different offsets, so this is the same cache-hit step,
+ * Appendix A, with one cache length per sequence).
+ *   pos [B] int32 in DEVICE memory: sequence b has pos[b] valid rows on entry; its new row goes to row pos[b]
+ *   and its query attends over rows [0, pos[b]].  Reading the positions on the device lets the caller advance
+ *   them there, without a host round trip per token.
+ *   max_pos: a HOST-side upper bound of every pos[b] (0 <= max_pos < Ncap); it sizes the split of the key range.
+ * An entry outside [0, min(max_pos, Ncap-1)] cannot be seen by the host: the kernel leaves that sequence's cache
+ * untouched, writes zeros for it, and tlin_get_status reports TLIN_ERR_INVALID_ARG.
+ * Everything else as tlin_decode_step. */
+int tlin_decode_step_ragged(const void* q_new, const void* k_new, const void* v_new,
+                            void* k_cache, void* v_cache, void* out, float* lse,
+                            int B, int H, int Ncap, const int32_t* pos, int max_pos, int d, tlin_stream_t stream);
+
 /* tlin_decode_step with HOST q/k/v_new and out/lse (the caches stay on the device).  *_d are
  * DEVICE staging buffers ([B,H,1,d] each, lse_d [B,H]). */
 int tlin_decode_step_host(const void* q_new_h, const void* k_new_h, const void* v_new_h, void* out_h, float* lse_h,

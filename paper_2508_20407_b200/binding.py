@@ -47,6 +47,7 @@ SIGNATURES = {
     "tlin_decode_step": (_i, [_vp] * 7 + [_i] * 5 + [_vp]),
     "tlin_decode_step_host": (_i, [_vp] * 12 + [_i] * 5 + [_vp]),
     "tlin_decode_step_static": (_i, [_vp] * 7 + [_i] * 5 + [_vp]),
+    "tlin_decode_step_ragged": (_i, [_vp] * 7 + [_i] * 3 + [_vp, _i, _i, _vp]),
     "tlin_merge_lse": (_i, [_vp] * 6 + [_i64, _i, _vp]),
     "tlin_merge_lse_f32": (_i, [_vp] * 6 + [_i64, _i, _vp]),
     "tlin_workspace_bytes_forward": (_sz, [_i] * 6),
@@ -208,6 +209,26 @@ def tlin_decode_step(q_new, k_new, v_new, k_cache, v_cache, pos, out=None, lse=N
     ensure_workspace(workspace_bytes_decode(B, H, Ncap, d), q_new.device)
     _check(lib().tlin_decode_step(_ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache),
                                   _ptr(out), _ptr(lse), B, H, Ncap, int(pos), d, _stream(stream)), "tlin_decode_step")
+    return out, lse
+
+
+def tlin_decode_step_ragged(q_new, k_new, v_new, k_cache, v_cache, pos, max_pos, out=None, lse=None, stream=None):
+    """Decode step with one cache length per sequence: ``pos`` is an int32 device tensor of shape [B],
+    ``max_pos`` a host-side upper bound of its entries."""
+    B, H, Ncap, d = k_cache.shape
+    for t, n in ((q_new, "q_new"), (k_new, "k_new"), (v_new, "v_new")):
+        _dev(t, torch.bfloat16, (B, H, 1, d), n)
+    _dev(k_cache, torch.bfloat16, (B, H, Ncap, d), "k_cache")
+    _dev(v_cache, torch.bfloat16, (B, H, Ncap, d), "v_cache")
+    _dev(pos, torch.int32, (B,), "pos")
+    if out is None:
+        out = torch.empty_like(q_new)
+    if lse is None:
+        lse = torch.empty((B, H), dtype=torch.float32, device=q_new.device)
+    ensure_workspace(workspace_bytes_decode(B, H, Ncap, d), q_new.device)
+    _check(lib().tlin_decode_step_ragged(_ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache),
+                                         _ptr(out), _ptr(lse), B, H, Ncap, _ptr(pos), int(max_pos), d, _stream(stream)),
+           "tlin_decode_step_ragged")
     return out, lse
 
 

@@ -128,7 +128,30 @@ extern "C" int tlin_decode_step(const void* q_new, const void* k_new, const void
     if (rc != TLIN_OK) return rc;
     const Workspace w = workspace();
     if (!w.ptr || w.bytes < (size_t)plan.workspace_bytes) return TLIN_ERR_WORKSPACE;
-    return launch_decode(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, d, plan,
+    return launch_decode(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, nullptr, d, plan,
+                         (float*)w.ptr, (cudaStream_t)stream);
+}
+
+extern "C" int tlin_decode_step_ragged(const void* q_new, const void* k_new, const void* v_new,
+                                       void* k_cache, void* v_cache, void* out, float* lse,
+                                       int B, int H, int Ncap, const int32_t* pos, int max_pos, int d, tlin_stream_t stream) {
+    t_launches = 0;
+    if (!q_new || !k_new || !v_new || !k_cache || !v_cache || !out || !pos) return TLIN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || Ncap <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    if (max_pos < 0 || max_pos >= Ncap) return TLIN_ERR_INVALID_ARG;
+    if (!aligned16(q_new) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) ||
+        !aligned16(v_cache) || !aligned16(out) || (reinterpret_cast<uintptr_t>(pos) & 3u)) return TLIN_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return TLIN_ERR_UNSUPPORTED;
+    int sms = 0;
+    int rc = device_info(&sms);
+    if (rc != TLIN_OK) return rc;
+    tlin_decode_plan plan;
+    rc = tlin_plan_decode(B, H, max_pos + 1, d, sms, &plan);      // the longest sequence decides the split
+    if (rc != TLIN_OK) return rc;
+    const Workspace w = workspace();
+    if (!w.ptr || w.bytes < (size_t)plan.workspace_bytes) return TLIN_ERR_WORKSPACE;
+    // the kernel checks every entry against max_pos (and Ncap) and reports a bad one through the status word
+    return launch_decode(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, max_pos, pos, d, plan,
                          (float*)w.ptr, (cudaStream_t)stream);
 }
 

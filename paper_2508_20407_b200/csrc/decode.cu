@@ -67,13 +67,28 @@ __global__ void __launch_bounds__(kWarps * 32, kDecodeCtasPerSM)
 decode_splitk_kernel(const uint4* __restrict__ q_new, const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
                      uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
                      float* __restrict__ part_o, float* __restrict__ part_lse,
-                     int Ncap, int pos, int splits, int kps, float scale_log2e) {
+                     int Ncap, int pos_all, const int* __restrict__ pos_per_seq, int H, int* __restrict__ status,
+                     int splits, int kps, float scale_log2e) {
     constexpr int LPR = D / 8;           // lanes (16-byte chunks) per row
     constexpr int RPW = 32 / LPR;        // rows per warp-load
     constexpr int ROWS_PER_IT = kWarps * RPW * kUnroll;
     const int bh = blockIdx.x / splits, sp = blockIdx.x - bh * splits;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int sub = lane % LPR, rsel = lane / LPR;
+    // one position for the whole batch, or one per sequence read from device memory (ragged batch)
+    int pos = pos_all;
+    if (pos_per_seq != nullptr) {
+        pos = pos_per_seq[bh / H];
+        if (pos < 0 || pos >= Ncap || pos > pos_all) {   // pos_all is the caller's bound, which sized the splits; the host
+                                                          // cannot see the entries: report, and leave this (b,h) alone
+            if (threadIdx.x == 0) {
+                atomicExch(status, (int)TLIN_ERR_INVALID_ARG);
+                part_lse[(int64_t)bh * splits + sp] = -CUDART_INF_F;
+            }
+            if (threadIdx.x < D) part_o[((int64_t)bh * splits + sp) * D + threadIdx.x] = 0.f;
+            return;
+        }
+    }
     const int L = pos + 1;
     const int j0 = sp * kps, j1 = min(L, j0 + kps);
 
@@ -202,7 +217,7 @@ decode_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ 
 
 template <int D>
 int launch_d(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
-             void* out, float* lse, int B, int H, int Ncap, int pos, const tlin_decode_plan& plan,
+             void* out, float* lse, int B, int H, int Ncap, int pos, const int* pos_per_seq, const tlin_decode_plan& plan,
              float* ws, cudaStream_t st) {
     const int64_t bh = (int64_t)B * H;
     float* part_o = ws;
@@ -210,7 +225,7 @@ int launch_d(const void* q_new, const void* k_new, const void* v_new, void* k_ca
     const float scale_log2e = kLog2e / sqrtf((float)D);
     decode_splitk_kernel<D><<<plan.n_ctas, kWarps * 32, 0, st>>>(
         (const uint4*)q_new, (const uint4*)k_new, (const uint4*)v_new, (uint4*)k_cache, (uint4*)v_cache,
-        part_o, part_lse, Ncap, pos, plan.splits, plan.keys_per_split, scale_log2e);
+        part_o, part_lse, Ncap, pos, pos_per_seq, H, status_word(), plan.splits, plan.keys_per_split, scale_log2e);
     TLIN_CUDA_CHECK(cudaGetLastError());
     decode_merge_kernel<D><<<(unsigned)bh, D, 0, st>>>(part_o, part_lse, (__nv_bfloat16*)out, lse, plan.splits);
     TLIN_CUDA_CHECK(cudaGetLastError());
@@ -221,10 +236,10 @@ int launch_d(const void* q_new, const void* k_new, const void* v_new, void* k_ca
 }  // namespace
 
 int launch_decode(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
-                  void* out, float* lse, int B, int H, int Ncap, int pos, int d,
+                  void* out, float* lse, int B, int H, int Ncap, int pos, const int* pos_per_seq, int d,
                   const tlin_decode_plan& plan, float* ws, cudaStream_t st) {
-    if (d == 128) return launch_d<128>(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, plan, ws, st);
-    if (d == 64) return launch_d<64>(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, plan, ws, st);
+    if (d == 128) return launch_d<128>(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, pos_per_seq, plan, ws, st);
+    if (d == 64) return launch_d<64>(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, pos_per_seq, plan, ws, st);
     return TLIN_ERR_UNSUPPORTED;
 }
 
@@ -297,6 +312,6 @@ extern "C" int tlin_decode_step_static(const void* q_new, const void* k_new, con
     tlin_decode_plan plan;
     rc = tlin_plan_decode(B, H, pos + 1, d, sms, &plan);
     if (rc != TLIN_OK) return rc;
-    return launch_decode(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, d, plan, scratch,
+    return launch_decode(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, nullptr, d, plan, scratch,
                          (cudaStream_t)stream);
 }

@@ -41,7 +41,7 @@ int launch_fwd_tc(const void* q, const void* k, const void* v, void* out, float*
                   int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& plan,
                   float* ws, cudaStream_t st);
 int launch_decode(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
-                  void* out, float* lse, int B, int H, int Ncap, int pos, int d,
+                  void* out, float* lse, int B, int H, int Ncap, int pos, const int* pos_per_seq, int d,
                   const tlin_decode_plan& plan, float* ws, cudaStream_t st);
 int launch_merge_pair_bf16(const void* oa, const float* la, const void* ob, const float* lb,
                            void* out, float* lse, int64_t rows, int d, cudaStream_t st);

@@ -92,3 +92,50 @@ def test_cfg5_full_size_sampled_heads_and_steps():
     assert tl.tlin_get_status() == 0
     for (b, h) in heads:
         assert torch.equal(kc[b, h].cpu(), host[(b, h)][0][0, 0]) and torch.equal(vc[b, h].cpu(), host[(b, h)][1][0, 0])
+
+
+def test_ragged_decode_one_length_per_sequence():
+    """Sequences of one batch at different cache lengths (positions read from device memory): every sequence
+    equals the oracle's step at its own length; appended rows are bit-exact; nothing else in the caches moves."""
+    B, H, d, T = 4, 3, 128, 3
+    lengths = [0, 37, 1500, 4099]
+    ncap = max(lengths) + T + 2
+    rng = torch.Generator(device="cpu").manual_seed(77)
+    kc = (torch.randn((B, H, ncap, d), generator=rng) * 1.0).to(torch.bfloat16)
+    vc = (torch.randn((B, H, ncap, d), generator=rng) * 1.0).to(torch.bfloat16)
+    for b, n0 in enumerate(lengths):
+        kc[b, :, n0:] = -7.0
+        vc[b, :, n0:] = -7.0
+    kc_h, vc_h = kc.clone(), vc.clone()
+    kc, vc = kc.to(DEV), vc.to(DEV)
+    pos = torch.tensor(lengths, dtype=torch.int32, device=DEV)
+    for t in range(T):
+        qn = (torch.randn((B, H, 1, d), generator=rng)).to(torch.bfloat16)
+        kn = (torch.randn((B, H, 1, d), generator=rng)).to(torch.bfloat16)
+        vn = (torch.randn((B, H, 1, d), generator=rng)).to(torch.bfloat16)
+        out, lse = tl.tlin_decode_step_ragged(qn.to(DEV), kn.to(DEV), vn.to(DEV), kc, vc, pos, max(lengths) + t)
+        torch.cuda.synchronize()
+        assert tl.tlin_get_status() == 0
+        for b, n0 in enumerate(lengths):
+            sl = slice(b, b + 1)
+            ref, ref_lse = oracle.decode_step(qn[sl], kn[sl], vn[sl], kc_h[sl], vc_h[sl], n0 + t)   # updates the host caches in place
+            parity.check(out[sl].float().cpu().numpy(), lse[sl].cpu().numpy(), ref, ref_lse, "bf16", f"ragged step {t} seq {b}")
+        assert torch.equal(kc.cpu(), kc_h) and torch.equal(vc.cpu(), vc_h)
+        pos += 1                                   # advanced on the device
+
+
+def test_ragged_decode_reports_a_position_beyond_the_bound():
+    B, H, d = 2, 2, 64
+    kc = torch.zeros((B, H, 64, d), dtype=torch.bfloat16, device=DEV)
+    vc = torch.zeros_like(kc)
+    kc_before = kc.clone()
+    x = torch.ones((B, H, 1, d), dtype=torch.bfloat16, device=DEV)
+    pos = torch.tensor([5, 40], dtype=torch.int32, device=DEV)      # 40 exceeds the bound given below
+    out, lse = tl.tlin_decode_step_ragged(x, x, x, kc, vc, pos, 10)
+    torch.cuda.synchronize()
+    assert tl.tlin_get_status() == tl.ERR_INVALID_ARG
+    assert tl.tlin_get_status() == 0                                  # reading clears it
+    assert torch.equal(kc[1], kc_before[1])                           # the offending sequence's cache is untouched
+    assert (kc[0, :, 5] == 1).all()                                   # the valid one was appended
+    with pytest.raises(tl.TlinError):
+        tl.tlin_decode_step_ragged(x, x, x, kc, vc, pos, 64)          # bound outside the cache: rejected on the host
