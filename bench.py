@@ -184,6 +184,14 @@ def time_steps(step_fn, steps, warmup, world, device, sampler=None, flush_buf=No
 
 L2_BYTES = 126e6
 
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from one-pass ncu captures of these
+# very workloads (profiles/dram_traffic_forward_cfg3_cfg4.md).  To be set to None whenever the kernel changes.
+FWD_TRAFFIC = {"cfg4_vlong": (2.17e9 + 23.09e6, "ncu, full workload, fwd_tc_kernel<128>"),
+               "cfg3_long": (546.06e6 + 12.98e6, "ncu, full workload, fwd_tc_kernel<128>")}
+# decode: captured on a smaller cache (B8 H32, 4096 rows: 537.35 MB read + 3.9 MB written for 537.3 MB of cache) and
+# scaled by the cached rows of the timed steps; the kernel streams every cached byte once at any size
+DECODE_TRAFFIC_RATIO = (537.35 + 3.9) / 537.3
+
 
 # ----------------------------------------------------------------------------- the oracle as a timed baseline
 def oracle_forward_sample(wl, k_head, v_head, q_head, rows):
@@ -259,7 +267,9 @@ def run_forward(wl, args, rank, world, device, peaks, with_cpu):
     else:
         gbs = fwd_bytes(wl) / (ms_step * 1e-3) / 1e9
         roof = dict(bound="hbm", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s", frac=gbs / peaks["hbm_gbs"])
-    roof.update(traffic=None, peak_source=peaks["source"] + " (burst)", kernel="forward (attention kernel + split merge)",
+    traffic, traffic_source = FWD_TRAFFIC.get(wl.name, (None, None))
+    roof.update(traffic=traffic, traffic_source=traffic_source, algorithmic_bytes=fwd_bytes(wl),
+                peak_source=peaks["source"] + " (burst)", kernel="forward (attention kernel + split merge)",
                 roofline_ms=max(t_tensor, t_hbm) * 1e3)
     if bound == "tensor" and "bf16_tflops_sustained" in peaks:
         roof["frac_of_sustained_peak"] = tflops / peaks["bf16_tflops_sustained"]
@@ -328,7 +338,9 @@ def run_decode(wl, args, rank, world, device, peaks, with_cpu):
         tot += 2 * wl.B * wl.H * (pos + 1) * wl.d * 2 + 4 * wl.B * wl.H * wl.d * 2 + 4 * wl.B * wl.H
     gbs = tot / (ms * 1e-3) / 1e9
     roof = dict(bound="hbm", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s", frac=gbs / peaks["hbm_gbs"],
-                traffic=None, peak_source=peaks["source"], kernel="decode (split-K kernel + merge)",
+                traffic=tot / steps * DECODE_TRAFFIC_RATIO, algorithmic_bytes=tot / steps,
+                traffic_source="ncu on a 4096-row cache, scaled by the cached rows (traffic is proportional to them)",
+                peak_source=peaks["source"], kernel="decode (split-K kernel + merge)",
                 roofline_ms=tot / steps / (peaks["hbm_gbs"] * 1e9) * 1e3)
     e2e = None
     if not args.no_e2e:
