@@ -139,3 +139,56 @@ def test_ragged_decode_reports_a_position_beyond_the_bound():
     assert (kc[0, :, 5] == 1).all()                                   # the valid one was appended
     with pytest.raises(tl.TlinError):
         tl.tlin_decode_step_ragged(x, x, x, kc, vc, pos, 64)          # bound outside the cache: rejected on the host
+
+
+def test_ragged_decode_loop_replays_from_a_cuda_graph():
+    """With the positions in device memory a whole decode loop can be recorded once and replayed: the captured
+    sequence is [step; pos += 1] and a replay continues where the previous one stopped."""
+    B, H, d, n0 = 2, 4, 64, 300
+    steps_per_graph, replays = 4, 3
+    total = steps_per_graph * replays
+    ncap = n0 + total + 8
+    wl = synth.Workload("graph", B, H, d, n0, total, seed=91, decode=True)
+    (kc0, vc0), (qn, kn, vn) = synth.decode_inputs(wl, device=DEV)
+    kc = torch.zeros((B, H, ncap, d), dtype=torch.bfloat16, device=DEV)
+    vc = torch.zeros_like(kc)
+    kc[:, :, :n0], vc[:, :, :n0] = kc0[:, :, :n0], vc0[:, :, :n0]
+    kc_ref, vc_ref = kc.clone(), vc.clone()
+    # eager reference run: the same entry point with the same bound (hence the same split of the key range), call by call
+    ref_out = []
+    pos_ref = torch.full((B,), n0, dtype=torch.int32, device=DEV)
+    for t in range(total):
+        o, _ = tl.tlin_decode_step_ragged(qn[t], kn[t], vn[t], kc_ref, vc_ref, pos_ref, ncap - 1)
+        pos_ref += 1
+        ref_out.append(o.clone())
+    torch.cuda.synchronize()
+    # captured run: the graph reads its tokens from staging tensors that are refilled before every replay
+    tl.ensure_workspace(tl.workspace_bytes_decode(B, H, ncap, d), torch.device(DEV))
+    pos = torch.full((B,), n0, dtype=torch.int32, device=DEV)
+    q_st, k_st, v_st = (torch.empty((steps_per_graph, B, H, 1, d), dtype=torch.bfloat16, device=DEV) for _ in range(3))
+    outs = torch.empty((steps_per_graph, B, H, 1, d), dtype=torch.bfloat16, device=DEV)
+    lses = torch.empty((steps_per_graph, B, H), dtype=torch.float32, device=DEV)
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        # one eager warm-up step on scratch copies so that nothing is initialised for the first time under capture
+        tl.tlin_decode_step_ragged(qn[0], kn[0], vn[0], kc.clone(), vc.clone(), pos.clone(), ncap - 1, stream=stream)
+        stream.synchronize()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(steps_per_graph):
+                tl.tlin_decode_step_ragged(q_st[i], k_st[i], v_st[i], kc, vc, pos, ncap - 1, outs[i], lses[i], stream=stream)
+                pos.add_(1)
+    got = []
+    for r in range(replays):
+        sl = slice(r * steps_per_graph, (r + 1) * steps_per_graph)
+        q_st.copy_(qn[sl]); k_st.copy_(kn[sl]); v_st.copy_(vn[sl])
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        got.extend(outs[i].clone() for i in range(steps_per_graph))
+    assert tl.tlin_get_status() == 0
+    assert int(pos[0]) == n0 + total
+    for t in range(total):
+        assert torch.equal(got[t], ref_out[t]), f"step {t}"
+    assert torch.equal(kc[:, :, :n0 + total], kc_ref[:, :, :n0 + total])
