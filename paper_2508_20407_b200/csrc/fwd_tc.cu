@@ -528,8 +528,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 }
 
 // Combines the partial results of every (b,h) whose key tiles were split between groups.
-// One CTA per (b,h, q-tile pair, quarter): 8 warps, one query row per warp at a time, 4 (or 2) columns per lane.
-constexpr int kMergeRows = 64;
+// One CTA per 8 query rows of a (b,h, q-tile pair): 8 warps, one row each, 4 (or 2) columns per lane.
+constexpr int kMergeRows = 8;            // one row per warp: many small CTAs hide the latency of the scattered partial reads
 constexpr int kMaxParts = 8;          // more partials than this per row are merged in a slower loop
 
 template <int D>
