@@ -468,6 +468,7 @@ def main():
             if name == args.workload:
                 continue
             torch.cuda.empty_cache()
+            time.sleep(1.0)     # the legs are independent measurements: let the power state of the previous one settle
             w2 = synth.WORKLOADS[WORKLOADS[name]]
             a2 = argparse.Namespace(**vars(args))
             a2.no_e2e = args.no_e2e or name not in ("fwd32k", "decode")     # host-buffer legs only where they are cheap to set up
