@@ -185,7 +185,7 @@ def time_steps(step_fn, steps, warmup, world, device, sampler=None, flush_buf=No
 L2_BYTES = 126e6
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from one-pass ncu captures of these
-# very workloads (profiles/dram_traffic_forward_cfg3_cfg4.md).  To be set to None whenever the kernel changes.
+# very workloads.  To be set to None whenever the kernel changes.
 FWD_TRAFFIC = {"cfg4_vlong": (2.17e9 + 23.09e6, "ncu, full workload, fwd_tc_kernel<128>"),
                "cfg3_long": (546.06e6 + 12.98e6, "ncu, full workload, fwd_tc_kernel<128>")}
 # decode: captured on a smaller cache (B8 H32, 4096 rows: 537.35 MB read + 3.9 MB written for 537.3 MB of cache) and
