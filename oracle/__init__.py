@@ -35,6 +35,7 @@ def _load():
         lib = ctypes.CDLL(build())
         vp, dp, i32, i64 = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
         lib.tlin_ref_attn_forward.argtypes = [vp, vp, vp, i32, dp, dp, i32, i32, i64, i64, i32, i32]
+        lib.tlin_ref_attn_backward.argtypes = [vp, vp, vp, vp, i32, dp, dp, dp, i32, i32, i64, i64, i32, i32]
         lib.tlin_ref_decode_step.argtypes = [vp, vp, vp, vp, vp, i32, dp, dp, i32, i32, i64, i64, i32]
         lib.tlin_ref_merge_lse.argtypes = [dp, dp, dp, dp, dp, dp, i64, i32]
         lib.tlin_ref_allowed.argtypes = [i64, i64, i64, i64, i32]
@@ -95,6 +96,31 @@ def attn_forward(q, k, v, causal_window: int):
     if rc != 0:
         raise ValueError(f"tlin_ref_attn_forward rejected its arguments (rc={rc})")
     return out, lse
+
+
+def attn_backward(q, k, v, dout, causal_window: int):
+    """Gradients of ``attn_forward`` for a loss with dL/dout = dout (and no dependence on lse).
+
+    q,dout:[B,H,W,d], k,v:[B,H,N,d] (one element type) -> (dq [B,H,W,d], dk, dv [B,H,N,d]), all float64.
+    """
+    qa, tq = _as_elems(q)
+    ka, tk = _as_elems(k)
+    va, tv = _as_elems(v)
+    da, td = _as_elems(dout)
+    if not (tq == tk == tv == td):
+        raise TypeError("q, k, v, dout must share one element type")
+    B, H, W, d = qa.shape
+    Bk, Hk, N, dk_ = ka.shape
+    if (Bk, Hk, dk_) != (B, H, d) or va.shape != ka.shape or da.shape != qa.shape:
+        raise ValueError("shape mismatch")
+    dq = np.empty((B, H, W, d), dtype=np.float64)
+    dk = np.empty((B, H, N, d), dtype=np.float64)
+    dv = np.empty((B, H, N, d), dtype=np.float64)
+    rc = _load().tlin_ref_attn_backward(_ptr(qa), _ptr(ka), _ptr(va), _ptr(da), tq, _ptr(dq), _ptr(dk), _ptr(dv),
+                                        B, H, N, W, d, int(causal_window))
+    if rc != 0:
+        raise ValueError(f"tlin_ref_attn_backward rejected its arguments (rc={rc})")
+    return dq, dk, dv
 
 
 def decode_step(q_new, k_new, v_new, k_cache, v_cache, pos: int):

@@ -199,3 +199,81 @@ int tlin_ref_merge_lse(const double *out_a, const double *lse_a, const double *o
     }
     return 0;
 }
+
+/*
+ * Gradient of the forward above (training runs the same attention as a forward and a backward pass; Section 4.1
+ * counts training as "cache miss" throughout).  The paper gives no formula of its own: this is the chain rule
+ * applied to the attention formula of Section 3, written out row by row with the probabilities materialised.
+ * For a loss L with dout = dL/dout (dL/dlse taken as zero):
+ *     p_ij  = softmax_j(s_ij),  s_ij = q_i.k_j / sqrt(d)   over the allowed j
+ *     dv_j  = sum_i p_ij dout_i
+ *     dp_ij = dout_i . v_j
+ *     ds_ij = p_ij (dp_ij - sum_j' p_ij' dp_ij')
+ *     dq_i  = sum_j ds_ij k_j / sqrt(d)      dk_j = sum_i ds_ij q_i / sqrt(d)
+ * q,dout:[B,H,W,d]  k,v:[B,H,N,d] (elem_type as above)  ->  dq:[B,H,W,d]  dk,dv:[B,H,N,d] (double).
+ * (b,h) pairs are independent and handed out to threads; inside one the rows run in order.
+ */
+int tlin_ref_attn_backward(const void *q, const void *k, const void *v, const void *dout, int elem_type,
+                           double *dq, double *dk, double *dv,
+                           int B, int H, int64_t N, int64_t W, int d, int causal_window)
+{
+    if (!q || !k || !v || !dout || !dq || !dk || !dv) return -1;
+    if (B <= 0 || H <= 0 || N <= 0 || W <= 0 || d <= 0) return -1;
+    if (causal_window && N < W) return -1;
+    if (elem_type != TLIN_REF_BF16 && elem_type != TLIN_REF_F32) return -1;
+    const double inv_sqrt_d = 1.0 / sqrt((double)d);
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t bh = 0; bh < (int64_t)B * H; ++bh) {
+        double *p = (double *)malloc((size_t)N * sizeof(double));
+        double *dp = (double *)malloc((size_t)N * sizeof(double));
+        if (!p || !dp) {
+#pragma omp atomic write
+            failed = 1;
+            free(p);
+            free(dp);
+            continue;
+        }
+        const int64_t qbase = bh * W * d, kbase = bh * N * d;
+        for (int64_t x = 0; x < N * d; ++x) { dk[kbase + x] = 0.0; dv[kbase + x] = 0.0; }
+        for (int64_t i = 0; i < W; ++i) {
+            /* probabilities of row i */
+            double m = -INFINITY;
+            for (int64_t j = 0; j < N; ++j) {
+                if (!tlin_ref_allowed(i, j, N, W, causal_window)) { p[j] = -INFINITY; continue; }
+                double s = 0.0;
+                for (int c = 0; c < d; ++c)
+                    s += widen(q, elem_type, qbase + i * d + c) * widen(k, elem_type, kbase + j * d + c);
+                p[j] = s * inv_sqrt_d;
+                if (p[j] > m) m = p[j];
+            }
+            double l = 0.0;
+            for (int64_t j = 0; j < N; ++j) {
+                p[j] = (p[j] == -INFINITY) ? 0.0 : exp(p[j] - m);
+                l += p[j];
+            }
+            double delta = 0.0;
+            for (int64_t j = 0; j < N; ++j) {
+                p[j] /= l;
+                double t = 0.0;
+                for (int c = 0; c < d; ++c)
+                    t += widen(dout, elem_type, qbase + i * d + c) * widen(v, elem_type, kbase + j * d + c);
+                dp[j] = t;
+                delta += p[j] * t;
+            }
+            for (int c = 0; c < d; ++c) dq[qbase + i * d + c] = 0.0;
+            for (int64_t j = 0; j < N; ++j) {
+                if (p[j] == 0.0) continue;
+                const double ds = p[j] * (dp[j] - delta) * inv_sqrt_d;
+                for (int c = 0; c < d; ++c) {
+                    dq[qbase + i * d + c] += ds * widen(k, elem_type, kbase + j * d + c);
+                    dk[kbase + j * d + c] += ds * widen(q, elem_type, qbase + i * d + c);
+                    dv[kbase + j * d + c] += p[j] * widen(dout, elem_type, qbase + i * d + c);
+                }
+            }
+        }
+        free(p);
+        free(dp);
+    }
+    return failed ? -2 : 0;
+}

@@ -361,3 +361,90 @@ def test_stored_oracle_rows_have_not_drifted():
         assert np.abs(out[b, h, i, :8] - vals[1:]).max() < 1e-9
         n += 1
     assert n == 4
+
+
+# ----------------------------------------------------------------------------- backward oracle
+# The gradient of the Section 3 attention formula.  None of these pins calls attn_backward for its expectation.
+def _rand_problem(seed, B, H, N, W, d):
+    rng = np.random.default_rng(seed)
+    mk = lambda *s: rng.standard_normal(s).astype(np.float32)
+    return mk(B, H, W, d), mk(B, H, N, d), mk(B, H, N, d), mk(B, H, W, d)
+
+
+@pytest.mark.parametrize("B,H,N,W,d,causal", [(1, 1, 6, 3, 4, 1), (1, 2, 7, 7, 3, 1), (2, 1, 5, 2, 2, 0), (1, 1, 4, 6, 4, 0)])
+def test_backward_matches_central_differences_of_the_forward(B, H, N, W, d, causal):
+    """dL/dx for L = sum(out * g), by central differences of the forward oracle (itself pinned above)."""
+    q, k, v, g = _rand_problem(40 + N, B, H, N, W, d)
+    dq, dk, dv = oracle.attn_backward(q, k, v, g, causal)
+
+    def loss(q_, k_, v_):
+        out, _ = oracle.attn_forward(q_, k_, v_, causal)
+        return float((out * g.astype(np.float64)).sum())
+
+    eps = 1e-3          # inputs are float32: the step has to survive the cast; the forward is smooth, error O(eps^2)
+    for name, x, grad in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        rng = np.random.default_rng(7)
+        for _ in range(12):
+            idx = tuple(int(rng.integers(0, n)) for n in x.shape)
+            xp, xm = x.copy(), x.copy()
+            xp[idx] += eps
+            xm[idx] -= eps
+            args_p = {"q": (xp, k, v), "k": (q, xp, v), "v": (q, k, xp)}[name]
+            args_m = {"q": (xm, k, v), "k": (q, xm, v), "v": (q, k, xm)}[name]
+            step = float(xp[idx]) - float(xm[idx])          # the step actually taken after rounding to float32
+            fd = (loss(*args_p) - loss(*args_m)) / step
+            assert abs(fd - grad[idx]) <= 2e-5 * max(1.0, abs(fd)), (name, idx, fd, grad[idx])
+
+
+@pytest.mark.parametrize("N,W,causal", [(9, 5, 1), (6, 6, 1), (8, 3, 0)])
+def test_backward_matches_autograd_of_the_textbook_formula(N, W, causal):
+    """torch autograd (fp64, CPU) through softmax(QK^T/sqrt(d) + mask)V written with library ops."""
+    B, H, d = 2, 2, 8
+    q, k, v, g = _rand_problem(50 + N, B, H, N, W, d)
+    tq, tk, tv = (torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in (q, k, v))
+    s = tq @ tk.transpose(-1, -2) / d ** 0.5
+    if causal:
+        keep = torch.arange(N)[None, :] <= (N - W) + torch.arange(W)[:, None]
+        s = s.masked_fill(~keep, float("-inf"))
+    (torch.softmax(s, -1) @ tv * torch.tensor(g, dtype=torch.float64)).sum().backward()
+    dq, dk, dv = oracle.attn_backward(q, k, v, g, causal)
+    assert np.abs(dq - tq.grad.numpy()).max() < 1e-12
+    assert np.abs(dk - tk.grad.numpy()).max() < 1e-12
+    assert np.abs(dv - tv.grad.numpy()).max() < 1e-12
+
+
+def test_backward_closed_forms():
+    """q = 0: uniform probabilities over the allowed keys, so dv_j = sum_i dout_i / n_i over the rows that see j,
+    and dk = 0 (ds multiplies q = 0); dq_i = sum_j ds_ij k_j / sqrt(d) with ds_ij = (dout_i.v_j - mean_j')/n_i."""
+    B, H, N, W, d = 1, 1, 6, 3, 4
+    _, k, v, g = _rand_problem(3, B, H, N, W, d)
+    q = np.zeros((B, H, W, d), dtype=np.float32)
+    dq, dk, dv = oracle.attn_backward(q, k, v, g, 1)
+    assert np.abs(dk).max() == 0.0
+    n_i = np.array([N - W + i + 1 for i in range(W)], dtype=np.float64)
+    exp_dv = np.zeros((N, d))
+    exp_dq = np.zeros((W, d))
+    for i in range(W):
+        n = int(n_i[i])
+        exp_dv[:n] += g[0, 0, i].astype(np.float64) / n
+        dp = v[0, 0, :n].astype(np.float64) @ g[0, 0, i].astype(np.float64)
+        ds = (dp - dp.mean()) / n
+        exp_dq[i] = ds @ k[0, 0, :n].astype(np.float64) / np.sqrt(d)
+    assert np.abs(dv[0, 0] - exp_dv).max() < 1e-13 and np.abs(dq[0, 0] - exp_dq).max() < 1e-13
+    # the rows of ds sum to zero: adding the same vector to every allowed key leaves dq's projection ... and
+    # a constant added to dout along v-directions: sum_j dv_j = sum_i dout_i (probabilities sum to one)
+    q2, k2, v2, g2 = _rand_problem(4, 1, 2, 7, 4, 3)
+    _, _, dv2 = oracle.attn_backward(q2, k2, v2, g2, 0)
+    assert np.abs(dv2.sum(axis=2) - g2.astype(np.float64).sum(axis=2)).max() < 1e-12
+
+
+def test_backward_respects_the_causal_window():
+    """Keys beyond a row's limit get no gradient from that row: with only the first window row carrying dout,
+    dk and dv vanish exactly for j > N - W, and dq of the other rows is zero."""
+    B, H, N, W, d = 1, 1, 8, 4, 4
+    q, k, v, g = _rand_problem(9, B, H, N, W, d)
+    g[:, :, 1:] = 0.0
+    dq, dk, dv = oracle.attn_backward(q, k, v, g, 1)
+    assert (dk[0, 0, N - W + 1:] == 0).all() and (dv[0, 0, N - W + 1:] == 0).all()
+    assert (dq[0, 0, 1:] == 0).all() and np.abs(dq[0, 0, 0]).max() > 0
+    assert np.abs(dv[0, 0, :N - W + 1]).min() > 0
