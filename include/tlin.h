@@ -126,6 +126,23 @@ int tlin_decode_step_static(const void* q_new, const void* k_new, const void* v_
                             int B, int H, int Ncap, int pos, int d, tlin_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Backward pass of tlin_attn_forward (bf16 in and out, fp32 arithmetic).  Training runs every layer
+ * as a full forward and backward pass ("cache miss" everywhere, Section 4.1); the paper states no
+ * gradient algorithm, so this is the chain rule applied to the Section 3 attention formula with the
+ * same window rule:  p = exp(q k^T / sqrt(d) - lse),  dv = p^T dout,  dp = dout v^T,
+ * ds = p * (dp - rowsum(dout * out)) / sqrt(d),  dq = ds k,  dk = ds^T q.
+ *   q, out, dout, dq [B,H,W,d]   k, v, dk, dv [B,H,N,d]   lse [B,H,W] fp32   (all DEVICE, 16-byte aligned)
+ * out and lse are what tlin_attn_forward returned for the same q, k, v and causal_window (lse is
+ * required here); dout is the loss gradient with respect to out; the loss must not depend on lse.
+ * dq, dk, dv are overwritten (keys that no query may use get zeros).  d in {64,128}.
+ * Needs a workspace of tlin_workspace_bytes_backward bytes (row sums and the fp32 dq accumulator).
+ * This first path runs on the CUDA cores.  Errors as for tlin_attn_forward.
+ */
+int tlin_attn_backward(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                       const void* dout, void* dq, void* dk, void* dv,
+                       int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------
  * Exact merge of two results over DISJOINT key sets for the same queries (not in the paper; it is
  * the split-K combine, exposed so that "history" and "window" attention may also be computed
  * separately and joined): lse = log(e^lse_a + e^lse_b), out = (e^lse_a out_a + e^lse_b out_b)/e^lse.
@@ -144,6 +161,7 @@ int tlin_merge_lse_f32(const float* out_a, const float* lse_a, const float* out_
  */
 size_t tlin_workspace_bytes_forward(int B, int H, int N, int W, int d, int causal_window);
 size_t tlin_workspace_bytes_decode(int B, int H, int Ncap, int d);
+size_t tlin_workspace_bytes_backward(int B, int H, int N, int W, int d);
 int tlin_set_workspace(void* dev_ptr, size_t bytes);
 
 /* ------------------------------------------------------------------------------------------

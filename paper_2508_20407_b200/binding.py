@@ -44,6 +44,7 @@ SIGNATURES = {
     "tlin_attn_forward": (_i, [_vp] * 5 + [_i] * 6 + [_vp]),
     "tlin_attn_forward_f32": (_i, [_vp] * 5 + [_i] * 6 + [_vp]),
     "tlin_attn_forward_host": (_i, [_vp] * 10 + [_i] * 6 + [_vp]),
+    "tlin_attn_backward": (_i, [_vp] * 9 + [_i] * 6 + [_vp]),
     "tlin_decode_step": (_i, [_vp] * 7 + [_i] * 5 + [_vp]),
     "tlin_decode_step_host": (_i, [_vp] * 12 + [_i] * 5 + [_vp]),
     "tlin_decode_step_static": (_i, [_vp] * 7 + [_i] * 5 + [_vp]),
@@ -52,6 +53,7 @@ SIGNATURES = {
     "tlin_merge_lse_f32": (_i, [_vp] * 6 + [_i64, _i, _vp]),
     "tlin_workspace_bytes_forward": (_sz, [_i] * 6),
     "tlin_workspace_bytes_decode": (_sz, [_i] * 4),
+    "tlin_workspace_bytes_backward": (_sz, [_i] * 5),
     "tlin_set_workspace": (_i, [_vp, _sz]),
     "tlin_plan_forward": (_i, [_i] * 8 + [ctypes.POINTER(FwdPlan)]),
     "tlin_plan_decode": (_i, [_i] * 5 + [ctypes.POINTER(DecodePlan)]),
@@ -122,6 +124,10 @@ def workspace_bytes_decode(B, H, Ncap, d) -> int:
     return int(lib().tlin_workspace_bytes_decode(B, H, Ncap, d))
 
 
+def workspace_bytes_backward(B, H, N, W, d) -> int:
+    return int(lib().tlin_workspace_bytes_backward(B, H, N, W, d))
+
+
 def set_workspace(t: torch.Tensor | None):
     """Registers a device buffer (any dtype) as split-K scratch; the tensor is kept alive here."""
     global _workspace_tensor
@@ -179,6 +185,28 @@ def tlin_attn_forward_f32(q, k, v, out=None, lse=None, causal_window=1, stream=N
     _check(lib().tlin_attn_forward_f32(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), B, H, N, W, d,
                                        int(causal_window), _stream(stream)), "tlin_attn_forward_f32")
     return out, lse
+
+
+def tlin_attn_backward(q, k, v, out, lse, dout, dq=None, dk=None, dv=None, causal_window=1, stream=None):
+    """bf16 backward of ``tlin_attn_forward``: (dq [B,H,W,d], dk, dv [B,H,N,d]) for the loss gradient ``dout``.
+
+    ``out`` and ``lse`` are the forward's results for the same q, k, v and causal_window."""
+    B, H, W, d = q.shape
+    N = k.shape[2]
+    for t, shape, name in ((q, (B, H, W, d), "q"), (k, (B, H, N, d), "k"), (v, (B, H, N, d), "v"),
+                           (out, (B, H, W, d), "out"), (dout, (B, H, W, d), "dout")):
+        _dev(t, torch.bfloat16, shape, name)
+    _dev(lse, torch.float32, (B, H, W), "lse")
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(v) if dv is None else dv
+    _dev(dq, torch.bfloat16, (B, H, W, d), "dq")
+    _dev(dk, torch.bfloat16, (B, H, N, d), "dk")
+    _dev(dv, torch.bfloat16, (B, H, N, d), "dv")
+    ensure_workspace(workspace_bytes_backward(B, H, N, W, d), q.device)
+    _check(lib().tlin_attn_backward(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk),
+                                    _ptr(dv), B, H, N, W, d, int(causal_window), _stream(stream)), "tlin_attn_backward")
+    return dq, dk, dv
 
 
 def tlin_attn_forward_host(q_h, k_h, v_h, out_h, lse_h, q_d, k_d, v_d, out_d, lse_d, causal_window=1, stream=None):

@@ -110,6 +110,33 @@ extern "C" int tlin_attn_forward_host(const void* q_h, const void* k_h, const vo
     return TLIN_OK;
 }
 
+extern "C" int tlin_attn_backward(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                                  const void* dout, void* dq, void* dk, void* dv,
+                                  int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream) {
+    t_launches = 0;
+    if (!q || !k || !v || !out || !lse || !dout || !dq || !dk || !dv) return TLIN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || N <= 0 || W <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    if (causal_window != 0 && causal_window != 1) return TLIN_ERR_INVALID_ARG;
+    if (causal_window && N < W) return TLIN_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(dout) ||
+        !aligned16(dq) || !aligned16(dk) || !aligned16(dv)) return TLIN_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(lse) & 3u) return TLIN_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return TLIN_ERR_UNSUPPORTED;
+    int sms = 0;
+    const int rc = device_info(&sms);
+    if (rc != TLIN_OK) return rc;
+    const Workspace w = workspace();
+    if (!w.ptr || w.bytes < bwd_workspace_bytes(B, H, W, d)) return TLIN_ERR_WORKSPACE;
+    return launch_bwd_simt(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, d, causal_window, (float*)w.ptr, sms,
+                           (cudaStream_t)stream);
+}
+
+extern "C" size_t tlin_workspace_bytes_backward(int B, int H, int N, int W, int d) {
+    (void)N;
+    if (B <= 0 || H <= 0 || W <= 0 || d <= 0) return 0;
+    return bwd_workspace_bytes(B, H, W, d);
+}
+
 extern "C" int tlin_decode_step(const void* q_new, const void* k_new, const void* v_new,
                                 void* k_cache, void* v_cache, void* out, float* lse,
                                 int B, int H, int Ncap, int pos, int d, tlin_stream_t stream) {

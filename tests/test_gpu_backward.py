@@ -1,0 +1,118 @@
+"""GPU parity of the backward entry point against the CPU oracle's fp64 chain rule, element by element on the
+same seeded bf16 inputs.  The forward results the backward needs (out, lse) come from the library's own forward,
+as they do in training.
+
+Gates (bf16 in, fp32 arithmetic, bf16 out): per gradient tensor, relative L2 error <= 2e-2 and
+max|err| <= 2e-2 * max|reference| -- the forward's absolute gates, scaled by the gradient's own magnitude, because a
+gradient has no natural unit scale (it is linear in dout).  Where the exact gradient is identically zero (a single
+visible key makes the softmax constant, so dq = dk = 0) the fp32 difference dp - delta leaves rounding noise of a few
+1e-7 on unit-scale inputs: an absolute floor of 1e-5 covers it."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import parity
+from paper_2508_20407_b200 import binding as tl
+from paper_2508_20407_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+REL_L2, REL_MAX, ABS_FLOOR = 2e-2, 2e-2, 1e-5
+
+
+def grads(q, k, v, dout, causal):
+    out, lse = tl.tlin_attn_forward(q, k, v, causal_window=causal)
+    dq, dk, dv = tl.tlin_attn_backward(q, k, v, out, lse, dout, causal_window=causal)
+    torch.cuda.synchronize()
+    assert tl.tlin_get_status() == 0
+    assert tl.tlin_last_launch_count() >= 3
+    return dq, dk, dv
+
+
+def compare(got, ref, what):
+    got = got.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all(), f"{what}: non-finite gradient"
+    e = parity.errors(got, ref)
+    scale = float(np.abs(ref).max())
+    if scale > 1e-3:
+        assert e["rel_l2"] <= REL_L2, f"{what}: rel L2 {e['rel_l2']:.3e}"
+    assert e["max_abs"] <= REL_MAX * scale + ABS_FLOOR, f"{what}: max|err| {e['max_abs']:.3e} vs max|ref| {scale:.3e}"
+    return e
+
+
+def run_case(B, H, N, W, d, causal, seed, peaky=False):
+    wl = synth.Workload("bwd", B, H, d, N, W, seed=seed, causal_window=causal)
+    q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
+    if peaky:
+        q = (q.float() * 6.0).to(torch.bfloat16)
+    g = torch.Generator(device="cpu").manual_seed(seed + 7)
+    dout = torch.randn(q.shape, generator=g, dtype=torch.float32).to(torch.bfloat16).to(DEV)
+    dq, dk, dv = grads(q, k, v, dout, causal)
+    rq, rk, rv = oracle.attn_backward(q.cpu(), k.cpu(), v.cpu(), dout.cpu(), causal)
+    tag = f"B{B} H{H} N{N} W{W} d{d} causal{causal}"
+    compare(dq, rq, tag + " dq")
+    compare(dk, rk, tag + " dk")
+    compare(dv, rv, tag + " dv")
+    return dq, dk, dv
+
+
+SHAPES = [  # B, H, N, W, d, causal: single elements, ragged tails on both axes, several key slices, both masks
+    (1, 1, 1, 1, 64, 1), (1, 2, 33, 1, 128, 1), (2, 1, 64, 64, 64, 1), (1, 2, 300, 300, 128, 1),
+    (1, 3, 1000, 77, 128, 1), (2, 2, 515, 130, 64, 0), (1, 2, 257, 255, 128, 0), (1, 1, 100, 300, 128, 0),
+    (1, 1, 4096, 96, 128, 1), (3, 2, 1111, 200, 64, 1), (1, 1, 2049, 31, 64, 0),
+]
+
+
+@pytest.mark.parametrize("B,H,N,W,d,causal", SHAPES)
+def test_backward_elementwise(B, H, N, W, d, causal):
+    run_case(B, H, N, W, d, causal, seed=300 + N + W)
+
+
+def test_backward_cfg1_tiny():
+    wl = synth.WORKLOADS["cfg1_tiny"]
+    run_case(wl.B, wl.H, wl.N, wl.W, wl.d, wl.causal_window, seed=wl.seed)
+
+
+def test_backward_peaked_softmax():
+    # scores large enough that most rows put nearly all weight on one key: exercises exp(s - lse) near 1 and near 0
+    run_case(1, 2, 700, 96, 128, 1, seed=11, peaky=True)
+
+
+def test_backward_keys_outside_every_window_get_zero_gradient():
+    # with the window rule the last key is visible to the last query only; a key count N == W makes key j invisible
+    # to queries i < j.  Zero dout rows for the queries that see the tail => exact zeros in dk, dv there.
+    B, H, N, W, d = 1, 2, 160, 160, 64
+    wl = synth.Workload("bwd", B, H, d, N, W, seed=5, causal_window=1)
+    q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
+    dout = torch.randn(q.shape, device=DEV).to(torch.bfloat16)
+    dout[:, :, 100:, :] = 0
+    _, dk, dv = grads(q, k, v, dout, 1)
+    assert float(dk[:, :, 100:, :].float().abs().max()) == 0.0
+    assert float(dv[:, :, 100:, :].float().abs().max()) == 0.0
+    assert float(dk[:, :, :100, :].float().abs().max()) > 0.0
+
+
+def test_backward_is_deterministic_up_to_the_dq_sum_order():
+    # dk, dv have one owner per element: bitwise repeatable.  dq is summed over key slices with atomics: equal within
+    # fp32 rounding, so the rounded bf16 values may differ in the last place only.
+    wl = synth.Workload("bwd", 1, 2, 128, 3000, 64, seed=9, causal_window=1)
+    q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
+    dout = torch.randn(q.shape, device=DEV).to(torch.bfloat16)
+    a = grads(q, k, v, dout, 1)
+    b = grads(q, k, v, dout, 1)
+    assert torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])
+    diff = (a[0].float() - b[0].float()).abs()
+    assert float((diff / (a[0].float().abs() + 1e-20)).max()) <= 2.0 ** -7
+
+
+def test_backward_argument_errors():
+    q = torch.zeros(1, 1, 32, 64, dtype=torch.bfloat16, device=DEV)
+    k = torch.zeros(1, 1, 16, 64, dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros(1, 1, 32, dtype=torch.float32, device=DEV)
+    with pytest.raises(tl.TlinError):        # N < W with the window rule
+        tl.tlin_attn_backward(q, k, k, q, lse, q, causal_window=1)
+    q96 = torch.zeros(1, 1, 8, 96, dtype=torch.bfloat16, device=DEV)
+    lse8 = torch.zeros(1, 1, 8, dtype=torch.float32, device=DEV)
+    with pytest.raises(tl.TlinError):        # head size outside {64, 128}
+        tl.tlin_attn_backward(q96, q96, q96, q96, lse8, q96, causal_window=0)
