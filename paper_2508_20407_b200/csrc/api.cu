@@ -123,18 +123,33 @@ extern "C" int tlin_attn_backward(const void* q, const void* k, const void* v, c
     if (reinterpret_cast<uintptr_t>(lse) & 3u) return TLIN_ERR_INVALID_ARG;
     if (d != 64 && d != 128) return TLIN_ERR_UNSUPPORTED;
     int sms = 0;
-    const int rc = device_info(&sms);
+    int rc = device_info(&sms);
     if (rc != TLIN_OK) return rc;
     const Workspace w = workspace();
-    if (!w.ptr || w.bytes < bwd_workspace_bytes(B, H, W, d)) return TLIN_ERR_WORKSPACE;
-    return launch_bwd_simt(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, d, causal_window, (float*)w.ptr, sms,
-                           (cudaStream_t)stream);
+    if (forward_impl() == 1) {
+        if (!w.ptr || w.bytes < bwd_workspace_bytes(B, H, W, d)) return TLIN_ERR_WORKSPACE;
+        return launch_bwd_simt(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, d, causal_window, (float*)w.ptr, sms,
+                               (cudaStream_t)stream);
+    }
+    tlin_fwd_plan plan;
+    rc = tlin_plan_forward(B, H, N, W, d, causal_window, 0, sms, &plan);   // the dQ kernel follows the forward's plan
+    if (rc != TLIN_OK) return rc;
+    if (!w.ptr || w.bytes < bwd_tc_workspace_bytes(B, H, W, d, plan)) return TLIN_ERR_WORKSPACE;
+    return launch_bwd_tc(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, d, causal_window, plan, (float*)w.ptr, sms,
+                         (cudaStream_t)stream);
 }
 
 extern "C" size_t tlin_workspace_bytes_backward(int B, int H, int N, int W, int d) {
-    (void)N;
-    if (B <= 0 || H <= 0 || W <= 0 || d <= 0) return 0;
-    return bwd_workspace_bytes(B, H, W, d);
+    if (B <= 0 || H <= 0 || N <= 0 || W <= 0 || d <= 0) return 0;
+    size_t need = bwd_workspace_bytes(B, H, W, d);                 // CUDA-core path
+    for (int causal = 0; causal < 2; ++causal) {
+        tlin_fwd_plan plan;
+        if (causal && N < W) continue;
+        if (tlin_plan_forward(B, H, N, W, d, causal, 0, 0, &plan) != TLIN_OK || !plan.tensor_path) continue;
+        const size_t t = bwd_tc_workspace_bytes(B, H, W, d, plan);
+        if (t > need) need = t;
+    }
+    return need;
 }
 
 extern "C" int tlin_decode_step(const void* q_new, const void* k_new, const void* v_new,

@@ -1,0 +1,915 @@
+// Tensor-core backward pass for sm_100a (bf16 in and out, fp32 accumulate): the chain rule of the Section 3
+// attention formula with the window rule j <= N-W+i.  Training runs every layer as forward + backward ("cache miss"
+// throughout, Section 4.1); the paper gives no gradient algorithm of its own.
+//
+//   p = exp(q k^T / sqrt(d) - lse)    dp = dout v^T    ds = p * (dp - delta) / sqrt(d),  delta_i = dout_i . out_i
+//   dv = p^T dout      dk = ds^T q      dq = ds k
+//
+// Two kernels, neither with atomics, both recomputing p from the saved lse:
+//
+// bwd_dkdv_tc_kernel   A CTA owns one 128-key tile of a (b,h) at a time and walks the 128-row query tiles that may
+//   see it.  Scores are computed TRANSPOSED (S^T = K Q^T, dP^T = V dout^T: TMEM lane = key, column = query) so that
+//   P^T and dS^T, written back to TMEM as bf16, are directly the A operands of dV += P^T dout and dK += dS^T Q, whose
+//   B operands are the dout / Q tiles already in shared memory (read MN-major).  dK and dV stay in TMEM for the whole
+//   key tile and are written once.  One TMEM region holds S^T and then dP^T of a step; 256 threads (key row x half
+//   of the query columns) do the elementwise work.
+//
+// bwd_dq_tc_kernel     The forward's structure: a CTA owns 256 query rows (two Q tiles, one warpgroup each, one
+//   thread per row) and streams 128-key tiles; per tile S = Q K^T -> p (kept in registers), then dP = dout V^T into
+//   the same TMEM columns -> dS (bf16, in place) -> dQ += dS K with K read MN-major.  The work is scheduled like the
+//   forward (groups that split the key range write fp32 partial dQ to the workspace; a small kernel adds them).
+//
+// A preparation kernel writes lse*log2(e) and delta per query row, padded to a multiple of 128 rows per (b,h) with
+// +inf / 0: a padded row then gives p = 0 without any test.
+//
+// Every wait is bounded: on expiry the CTA sets the library's error word, drains and exits.
+#include "tlin_internal.h"
+#include "sm100_ptx.cuh"
+#include "tc_common.cuh"
+#include <math_constants.h>
+
+namespace tlin {
+namespace {
+
+using namespace ptx;
+using namespace tc;
+
+constexpr int kProducerWarp = 8;
+constexpr int kMmaWarp = 9;
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct BwdParams {
+    const float* lse2;        // [B*H, Wpad]  lse * log2(e), +inf beyond W
+    const float* delta;       // [B*H, Wpad]  dout . out,   0 beyond W
+    void* dq;                 // [B*H, W, D] bf16
+    void* dk;                 // [B*H, N, D] bf16
+    void* dv;
+    float* ws;                // partial dQ slots of the dq kernel
+    int* status;
+    long long total_units;    // dk/dv kernel: B*H*key_tiles; dq kernel: the plan's units
+    int n_groups, q_tiles, key_tiles, schedule;   // dq kernel: the forward's plan fields
+    int q_tiles128;           // ceil(W / 128)
+    int N, W, Wpad, causal;
+    float scale_log2e, scale;
+};
+
+// ------------------------------------------------------------------------------------------ preparation
+template <int D>
+__global__ void __launch_bounds__(256)
+bwd_prep_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout, const float* __restrict__ lse,
+                float* __restrict__ lse2, float* __restrict__ delta, int W, int Wpad, long long rows_padded) {
+    const long long prow = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (prow >= rows_padded) return;
+    const int lane = threadIdx.x & 31;
+    const long long bh = prow / Wpad;
+    const int i = (int)(prow - bh * Wpad);
+    if (i >= W) {
+        if (lane == 0) {
+            lse2[prow] = CUDART_INF_F;
+            delta[prow] = 0.f;
+        }
+        return;
+    }
+    const long long row = bh * W + i;
+    float acc = 0.f;
+    for (int c = lane * 2; c < D; c += 64) {
+        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(out + row * D + c));
+        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(dout + row * D + c));
+        acc = fmaf(a.x, b.x, fmaf(a.y, b.y, acc));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) {
+        lse2[prow] = lse[row] * kLog2e;
+        delta[prow] = acc;
+    }
+}
+
+// ------------------------------------------------------------------------------------------ dK / dV
+template <int D>
+struct ACfg {
+    static constexpr int kTileBytes = kQTile * D * 2;          // one 128-row tile of Q, K, V or dout
+    static constexpr int kBoxes = D / 64;
+    // shared memory: K,V of two key tiles (current and prefetched), two Q tiles, one dout tile,
+    // per Q slot 128 lse2 + 128 delta
+    static constexpr int kOffKV = 0;
+    static constexpr int kOffQ = 4 * kTileBytes;
+    static constexpr int kOffDO = 6 * kTileBytes;
+    static constexpr int kOffStats = 7 * kTileBytes;
+    static constexpr int kOffBars = kOffStats + 2 * 256 * 4;
+    static constexpr int kNumBars = 18;
+    static constexpr int kSmemBytes = kOffBars + kNumBars * 8 + 16;
+    // TMEM columns: dK, dV (D each), R = S^T then dP^T (128), P^T then dS^T as bf16 (64)
+    static constexpr uint32_t kColDK = 0, kColDV = D, kColR = 2 * D, kColP = 2 * D + 128;
+    static constexpr int kThreads = 32 * 10;
+};
+
+// first 128-row query tile that may use a key of key tile t
+__device__ __forceinline__ int first_q_tile(const BwdParams& p, int t) {
+    if (!p.causal) return 0;
+    const long long f = (long long)t * kTileN - ((long long)p.N - p.W);
+    return f <= 0 ? 0 : (int)(f / kQTile);
+}
+
+template <int D>
+__global__ void __launch_bounds__(ACfg<D>::kThreads, 1)
+bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do, const BwdParams p) {
+    using C = ACfg<D>;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint8_t* sKV = smem + C::kOffKV;          // [buffer][K,V]
+    uint8_t* sQ = smem + C::kOffQ;            // [2]
+    uint8_t* sDO = smem + C::kOffDO;
+    float* sStats = reinterpret_cast<float*>(smem + C::kOffStats);   // [2][lse2 128 | delta 128]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kOffBars);
+    uint64_t* kv_full = bars + 0;     // [2]
+    uint64_t* kv_empty = bars + 2;    // [2]
+    uint64_t* q_full = bars + 4;      // [2]
+    uint64_t* q_empty = bars + 6;     // [2]
+    uint64_t* do_full = bars + 8;
+    uint64_t* do_empty = bars + 9;
+    uint64_t* s_full = bars + 10;     // S^T of a step is in R
+    uint64_t* p_full = bars + 11;     // all threads have read S^T and stored P^T
+    uint64_t* dp_full = bars + 12;    // dP^T is in R
+    uint64_t* r_free = bars + 13;     // all threads have read dP^T
+    uint64_t* dv_done = bars + 14;    // the dV MMAs have consumed P^T
+    uint64_t* ds_full = bars + 15;    // all threads have stored dS^T
+    uint64_t* acc_full = bars + 16;   // dK, dV of the key tile are complete
+    uint64_t* acc_empty = bars + 17;  // all threads have read them
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::kNumBars);
+    int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool base_ok = (smem_u32(smem) & 1023u) == 0;   // the swizzled tiles need 1024-byte alignment
+
+    if (threadIdx.x == 0) {
+        *abort_flag = base_ok ? 0 : 1;
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&kv_full[i], 1);
+            mbar_init(&kv_empty[i], 1);
+            mbar_init(&q_full[i], 1);
+            mbar_init(&q_empty[i], 1);
+        }
+        mbar_init(do_full, 1);
+        mbar_init(do_empty, 1);
+        mbar_init(s_full, 1);
+        mbar_init(p_full, 256);
+        mbar_init(dp_full, 1);
+        mbar_init(r_free, 256);
+        mbar_init(dv_done, 1);
+        mbar_init(ds_full, 256);
+        mbar_init(acc_full, 1);
+        mbar_init(acc_empty, 256);
+        fence_mbar_init();
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(tmem_slot, 512);
+        tmem_relinquish();
+    }
+    if (warp == kProducerWarp && lane == 0) {
+        prefetch_tensormap(&map_q);
+        prefetch_tensormap(&map_k);
+        prefetch_tensormap(&map_v);
+        prefetch_tensormap(&map_do);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    volatile int* abort_p = abort_flag;
+
+    const long long u_begin = (long long)(((unsigned long long)blockIdx.x * (unsigned long long)p.total_units) / gridDim.x);
+    const long long u_end = (long long)(((unsigned long long)(blockIdx.x + 1) * (unsigned long long)p.total_units) / gridDim.x);
+
+    if (warp == kProducerWarp) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            bool ok = base_ok;
+            uint32_t g = 0, n_kv = 0;          // steps issued, key tiles issued
+            auto load_kv = [&](long long u) {
+                const uint32_t b = n_kv & 1;
+                ok = mbar_wait(&kv_empty[b], ((n_kv >> 1) & 1) ^ 1, abort_p);
+                if (!ok) return;
+                const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
+                mbar_arrive_expect_tx(&kv_full[b], 2 * C::kTileBytes);
+                for (int x = 0; x < C::kBoxes; ++x) {
+                    tma_load_3d(sKV + (b * 2 + 0) * C::kTileBytes + x * (kQTile * 128), &map_k, &kv_full[b], x * 64, t * kTileN, bh);
+                    tma_load_3d(sKV + (b * 2 + 1) * C::kTileBytes + x * (kQTile * 128), &map_v, &kv_full[b], x * 64, t * kTileN, bh);
+                }
+                ++n_kv;
+            };
+            if (ok && u_begin < u_end) load_kv(u_begin);
+            for (long long u = u_begin; u < u_end && ok; ++u) {
+                const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
+                const int i_first = first_q_tile(p, t);
+                for (int i = i_first; i < p.q_tiles128 && ok; ++i, ++g) {
+                    const uint32_t qs = g & 1;
+                    ok = mbar_wait(&q_empty[qs], ((g >> 1) & 1) ^ 1, abort_p);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(&q_full[qs], C::kTileBytes + 1024);
+                    for (int x = 0; x < C::kBoxes; ++x)
+                        tma_load_3d(sQ + qs * C::kTileBytes + x * (kQTile * 128), &map_q, &q_full[qs], x * 64, i * kQTile, bh);
+                    bulk_load_1d(sStats + qs * 256, p.lse2 + (long long)bh * p.Wpad + i * kQTile, 512, &q_full[qs]);
+                    bulk_load_1d(sStats + qs * 256 + 128, p.delta + (long long)bh * p.Wpad + i * kQTile, 512, &q_full[qs]);
+                    ok = mbar_wait(do_empty, (g & 1) ^ 1, abort_p);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(do_full, C::kTileBytes);
+                    for (int x = 0; x < C::kBoxes; ++x)
+                        tma_load_3d(sDO + x * (kQTile * 128), &map_do, do_full, x * 64, i * kQTile, bh);
+                    if (i == i_first && u + 1 < u_end) load_kv(u + 1);     // next key tile's K, V arrive during this one
+                }
+            }
+            if (!ok && base_ok) {
+                // leave no copy in flight: the barriers armed last must complete (bounded)
+                int dummy = 0;
+                if (n_kv > 0) mbar_wait(&kv_full[(n_kv - 1) & 1], ((n_kv - 1) >> 1) & 1, &dummy, 200000000LL);
+                if (n_kv > 1) mbar_wait(&kv_full[(n_kv - 2) & 1], ((n_kv - 2) >> 1) & 1, &dummy, 200000000LL);
+                // q_full / do_full of step g may or may not have been armed; the steps before it were
+                if (g > 0) mbar_wait(&q_full[(g - 1) & 1], ((g - 1) >> 1) & 1, &dummy, 200000000LL);
+                if (g > 0) mbar_wait(do_full, (g - 1) & 1, &dummy, 200000000LL);
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------------ MMA issuer (all lanes walk, one issues)
+        const uint32_t idesc_st = make_idesc_bf16(kQTile, kTileN, 0, 0);     // S^T, dP^T: M = keys, N = queries
+        const uint32_t idesc_acc = make_idesc_bf16(kQTile, D, 0, 1);         // dV, dK: A in TMEM, B MN-major
+        const uint64_t kmaj = make_smem_desc_sw128(smem_u32(smem), 16, 1024);
+        const uint64_t mnmaj = make_smem_desc_sw128(smem_u32(smem), kQTile * 128, 1024);
+        const uint32_t desc_hi = (uint32_t)(kmaj >> 32);
+        const uint32_t kmaj_lo = (uint32_t)kmaj, mnmaj_lo = (uint32_t)mnmaj;
+        const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
+        const uint32_t tDK = tmem_u + C::kColDK, tDV = tmem_u + C::kColDV, tR = tmem_u + C::kColR, tP = tmem_u + C::kColP;
+        auto tile_off = [&](int byte_off) { return (uint32_t)(byte_off >> 4); };
+        auto issue_st = [&](uint32_t a_off, uint32_t b_off) {       // R = A B^T, both tiles K-major, contraction over d
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t off16 = ((kk >> 2) * (kQTile * 128) + (kk & 3) * 32) >> 4;
+                if (elect_one()) mma_ss_parts(tR, kmaj_lo + a_off + off16, kmaj_lo + b_off + off16, desc_hi, idesc_st, kk > 0);
+            }
+        };
+        auto issue_acc = [&](uint32_t d_tmem, uint32_t b_off, bool accumulate) {   // D += P^T(TMEM) B, contraction over queries
+#pragma unroll
+            for (int kk = 0; kk < kQTile / 16; ++kk)
+                if (elect_one()) mma_ts_parts(d_tmem, tP + kk * 8, mnmaj_lo + b_off + kk * (2048 >> 4), desc_hi, idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+        };
+        bool ok = base_ok;
+        uint32_t g = 0, n = 0;
+        for (long long u = u_begin; u < u_end && ok; ++u, ++n) {
+            const uint32_t b = n & 1;
+            const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
+            const int steps = p.q_tiles128 - first_q_tile(p, t);
+            const uint32_t k_off = tile_off(C::kOffKV + (b * 2 + 0) * C::kTileBytes), v_off = tile_off(C::kOffKV + (b * 2 + 1) * C::kTileBytes);
+            const uint32_t do_off = tile_off(C::kOffDO);
+            ok = __all_sync(0xffffffffu, mbar_wait(&kv_full[b], (n >> 1) & 1, abort_p));
+            if (!ok) break;
+            ok = __all_sync(0xffffffffu, mbar_wait(&q_full[g & 1], (g >> 1) & 1, abort_p));
+            if (!ok) break;
+            tc_fence_after();
+            issue_st(k_off, tile_off(C::kOffQ + (g & 1) * C::kTileBytes));
+            commit_elected(s_full);
+            for (int s = 0; s < steps && ok; ++s, ++g) {
+                const uint32_t q_off = tile_off(C::kOffQ + (g & 1) * C::kTileBytes);
+                ok = __all_sync(0xffffffffu, mbar_wait(p_full, g & 1, abort_p));
+                if (!ok) break;
+                ok = __all_sync(0xffffffffu, mbar_wait(do_full, g & 1, abort_p));
+                if (!ok) break;
+                if (s == 0 && n > 0) {          // the previous key tile's dK, dV must have been read out
+                    ok = __all_sync(0xffffffffu, mbar_wait(acc_empty, (n - 1) & 1, abort_p));
+                    if (!ok) break;
+                }
+                tc_fence_after();
+                issue_st(v_off, do_off);                    // dP^T over S^T: every thread has read S^T (p_full)
+                commit_elected(dp_full);
+                issue_acc(tDV, do_off, s > 0);
+                commit_elected(dv_done);
+                commit_elected(do_empty);
+                if (s + 1 < steps) {                        // next step's S^T as soon as dP^T has been read
+                    ok = __all_sync(0xffffffffu, mbar_wait(&q_full[(g + 1) & 1], ((g + 1) >> 1) & 1, abort_p));
+                    if (!ok) break;
+                    ok = __all_sync(0xffffffffu, mbar_wait(r_free, g & 1, abort_p));
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_st(k_off, tile_off(C::kOffQ + ((g + 1) & 1) * C::kTileBytes));
+                    commit_elected(s_full);
+                }
+                ok = __all_sync(0xffffffffu, mbar_wait(ds_full, g & 1, abort_p));
+                if (!ok) break;
+                tc_fence_after();
+                issue_acc(tDK, q_off, s > 0);
+                commit_elected(&q_empty[g & 1]);
+            }
+            if (!ok) break;
+            commit_elected(acc_full);
+            commit_elected(&kv_empty[b]);
+        }
+    } else {
+        // ------------------------------------------------------------------ elementwise threads
+        const int wg = warp >> 2;                              // which half of the query columns
+        const int r = (warp & 3) * 32 + lane;                  // key row inside the tile == TMEM lane
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tR = tmem_base + lane_addr + C::kColR + wg * 64;
+        const uint32_t tP = tmem_base + lane_addr + C::kColP + wg * 32;
+        bool ok = base_ok;
+        uint32_t g = 0, n = 0;
+        for (long long u = u_begin; u < u_end && ok; ++u, ++n) {
+            const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
+            const int key = t * kTileN + r;
+            const int i_first = first_q_tile(p, t);
+            const long long shift = (long long)p.N - p.W;       // query q may use key k iff q >= k - shift
+            const int q_min = p.causal ? (int)((long long)key - shift) : -0x7fffffff;
+            const int q_min_warp = p.causal ? (int)((long long)key - lane + 31 - shift) : -0x7fffffff;   // largest in the warp
+            for (int i = i_first; i < p.q_tiles128; ++i, ++g) {
+                const float* st = sStats + (g & 1) * 256 + wg * 64;
+                const int q0 = i * kQTile + wg * 64;              // first query of this thread's columns
+                ok = __all_sync(0xffffffffu, mbar_wait(s_full, g & 1, abort_p));
+                if (!ok) break;
+                // already complete (the S^T MMAs waited for it); observing it here orders the bulk-copied lse2 / delta
+                // before this thread's reads
+                ok = __all_sync(0xffffffffu, mbar_wait(&q_full[g & 1], (g >> 1) & 1, abort_p));
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t sv[2][32];
+                tmem_ld32_async(tR, sv[0]);
+                tmem_ld32_async(tR + 32, sv[1]);
+                tmem_wait_ld(sv[0]);
+                tmem_wait_ld(sv[1]);
+                const bool masked = q0 < q_min_warp;              // warp-uniform: some element of some lane is masked
+                float pf[64];
+#pragma unroll
+                for (int c = 0; c < 64; c += 4) {
+                    const float4 l4 = *reinterpret_cast<const float4*>(st + c);
+                    pf[c + 0] = ex2(fmaf(__uint_as_float(sv[c >> 5][(c + 0) & 31]), p.scale_log2e, -l4.x));
+                    pf[c + 1] = ex2(fmaf(__uint_as_float(sv[c >> 5][(c + 1) & 31]), p.scale_log2e, -l4.y));
+                    pf[c + 2] = ex2(fmaf(__uint_as_float(sv[c >> 5][(c + 2) & 31]), p.scale_log2e, -l4.z));
+                    pf[c + 3] = ex2(fmaf(__uint_as_float(sv[c >> 5][(c + 3) & 31]), p.scale_log2e, -l4.w));
+                }
+                if (masked) {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c)
+                        if (q0 + c < q_min) pf[c] = 0.f;
+                }
+                {
+                    uint32_t pk[32];
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) pk[c] = pack_bf16x2(pf[2 * c], pf[2 * c + 1]);
+                    tmem_st32(tP, pk);
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(p_full);
+                ok = __all_sync(0xffffffffu, mbar_wait(dp_full, g & 1, abort_p));
+                if (!ok) break;
+                tc_fence_after();
+                tmem_ld32_async(tR, sv[0]);
+                tmem_ld32_async(tR + 32, sv[1]);
+                tmem_wait_ld(sv[0]);
+                tmem_wait_ld(sv[1]);
+                tc_fence_before();
+                mbar_arrive(r_free);
+#pragma unroll
+                for (int c = 0; c < 64; c += 4) {
+                    const float4 d4 = *reinterpret_cast<const float4*>(st + 128 + c);
+                    pf[c + 0] *= __uint_as_float(sv[c >> 5][(c + 0) & 31]) - d4.x;
+                    pf[c + 1] *= __uint_as_float(sv[c >> 5][(c + 1) & 31]) - d4.y;
+                    pf[c + 2] *= __uint_as_float(sv[c >> 5][(c + 2) & 31]) - d4.z;
+                    pf[c + 3] *= __uint_as_float(sv[c >> 5][(c + 3) & 31]) - d4.w;
+                }
+                ok = __all_sync(0xffffffffu, mbar_wait(dv_done, g & 1, abort_p));    // P^T is no longer being read
+                if (!ok) break;
+                tc_fence_after();
+                {
+                    uint32_t pk[32];
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) pk[c] = pack_bf16x2(pf[2 * c], pf[2 * c + 1]);
+                    tmem_st32(tP, pk);
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(ds_full);
+            }
+            if (!ok) break;
+            // ---------------------------------------------------------------- dK, dV of this key tile
+            ok = __all_sync(0xffffffffu, mbar_wait(acc_full, n & 1, abort_p));
+            if (!ok) break;
+            tc_fence_after();
+            const bool store = key < p.N;
+#pragma unroll
+            for (int which = 0; which < 2; ++which) {
+                const uint32_t tA = tmem_base + lane_addr + (which == 0 ? C::kColDK : C::kColDV) + wg * (D / 2);
+                const float f = which == 0 ? p.scale : 1.f;
+                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(which == 0 ? p.dk : p.dv) +
+                                     ((long long)bh * p.N + key) * D + wg * (D / 2);
+#pragma unroll
+                for (int c = 0; c < D / 64; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tA + c * 32, o);
+                    if (store) {
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            uint4 w;
+                            w.x = pack_bf16x2(__uint_as_float(o[v4 * 8 + 0]) * f, __uint_as_float(o[v4 * 8 + 1]) * f);
+                            w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * f, __uint_as_float(o[v4 * 8 + 3]) * f);
+                            w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * f, __uint_as_float(o[v4 * 8 + 5]) * f);
+                            w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * f, __uint_as_float(o[v4 * 8 + 7]) * f);
+                            *reinterpret_cast<uint4*>(dst + c * 32 + v4 * 8) = w;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acc_empty);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, base_ok ? (int)TLIN_ERR_TIMEOUT : (int)TLIN_ERR_CUDA);
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ------------------------------------------------------------------------------------------ dQ
+template <int D>
+struct BCfg {
+    static constexpr int kTileBytes = kQTile * D * 2;
+    static constexpr int kBoxes = D / 64;
+    static constexpr int kKSlots = D == 128 ? 2 : 4;           // K tiles live for a whole step (S, then dQ)
+    static constexpr int kVSlots = D == 128 ? 1 : 2;           // V tiles only for the dP MMAs
+    static constexpr int kOffQ = 0;                            // 2 tiles
+    static constexpr int kOffDO = 2 * kTileBytes;              // 2 tiles
+    static constexpr int kOffK = 4 * kTileBytes;
+    static constexpr int kOffV = (4 + kKSlots) * kTileBytes;
+    static constexpr int kOffBars = (4 + kKSlots + kVSlots) * kTileBytes;
+    static constexpr int kNumBars = 11 + 2 * kKSlots + 2 * kVSlots;
+    static constexpr int kSmemBytes = kOffBars + kNumBars * 8 + 16;
+    // TMEM columns: R0, R1 (S, then dP, then dS as bf16; 128 each), dQ0, dQ1 (D each)
+    static constexpr uint32_t kColR = 0, kColDQ = 256;
+    static constexpr int kThreads = 32 * 12;                   // warps 10 and 11 only lend their registers
+    static constexpr int kComputeRegs = 216, kOtherRegs = 72;
+};
+
+template <int D>
+__global__ void __launch_bounds__(BCfg<D>::kThreads, 1)
+bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do, const BwdParams p) {
+    using C = BCfg<D>;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint8_t* sQ = smem + C::kOffQ;
+    uint8_t* sDO = smem + C::kOffDO;
+    uint8_t* sK = smem + C::kOffK;
+    uint8_t* sV = smem + C::kOffV;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kOffBars);
+    uint64_t* qdo_full = bars + 0;
+    uint64_t* qdo_empty = bars + 1;
+    uint64_t* dq_done = bars + 2;
+    uint64_t* s_full = bars + 3;      // [2]
+    uint64_t* p_ready = bars + 5;     // [2]  every thread of the tile has read S
+    uint64_t* dp_full = bars + 7;     // [2]
+    uint64_t* ds_full = bars + 9;     // [2]
+    uint64_t* k_full = bars + 11;
+    uint64_t* k_empty = k_full + C::kKSlots;
+    uint64_t* v_full = k_empty + C::kKSlots;
+    uint64_t* v_empty = v_full + C::kVSlots;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::kNumBars);
+    int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool base_ok = (smem_u32(smem) & 1023u) == 0;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = base_ok ? 0 : 1;
+        mbar_init(qdo_full, 1);
+        mbar_init(qdo_empty, 1);
+        mbar_init(dq_done, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&s_full[i], 1);
+            mbar_init(&p_ready[i], kQTile);
+            mbar_init(&dp_full[i], 1);
+            mbar_init(&ds_full[i], kQTile);
+        }
+        for (int s = 0; s < C::kKSlots; ++s) {
+            mbar_init(&k_full[s], 1);
+            mbar_init(&k_empty[s], 1);
+        }
+        for (int s = 0; s < C::kVSlots; ++s) {
+            mbar_init(&v_full[s], 1);
+            mbar_init(&v_empty[s], 1);
+        }
+        fence_mbar_init();
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(tmem_slot, 512);
+        tmem_relinquish();
+    }
+    if (warp == kProducerWarp && lane == 0) {
+        prefetch_tensormap(&map_q);
+        prefetch_tensormap(&map_k);
+        prefetch_tensormap(&map_v);
+        prefetch_tensormap(&map_do);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    volatile int* abort_p = abort_flag;
+
+    if (warp >= 8) {
+    setmaxnreg_dec<C::kOtherRegs>();
+    if (warp == kProducerWarp) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t kit = 0, vit = 0, seg_idx = 0;
+            bool ok = base_ok;
+            SegmentWalker walk(p);
+            Segment s;
+            while (ok && walk.next(s)) {
+                const int row0 = s.qt * kTileM;
+                const int c0 = seg_count(s, tiles_allowed(p, row0, 0)), c1 = seg_count(s, tiles_allowed(p, row0, 1));
+                const int cnt = c0 > c1 ? c0 : c1;
+                if (cnt == 0) continue;
+                if (seg_idx > 0) ok = mbar_wait(qdo_empty, (seg_idx - 1) & 1, abort_p);
+                if (!ok) break;
+                mbar_arrive_expect_tx(qdo_full, 4 * C::kTileBytes);
+                for (int i = 0; i < 2; ++i)
+                    for (int x = 0; x < C::kBoxes; ++x) {
+                        tma_load_3d(sQ + i * C::kTileBytes + x * (kQTile * 128), &map_q, qdo_full, x * 64, row0 + i * kQTile, s.bh);
+                        tma_load_3d(sDO + i * C::kTileBytes + x * (kQTile * 128), &map_do, qdo_full, x * 64, row0 + i * kQTile, s.bh);
+                    }
+                for (int j = 0; j < cnt && ok; ++j) {
+                    const int t = s.t_begin + j;
+                    {
+                        const uint32_t slot = kit % C::kKSlots, round = kit / C::kKSlots;
+                        ok = mbar_wait(&k_empty[slot], (round & 1) ^ 1, abort_p);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&k_full[slot], C::kTileBytes);
+                        for (int x = 0; x < C::kBoxes; ++x)
+                            tma_load_3d(sK + slot * C::kTileBytes + x * (kQTile * 128), &map_k, &k_full[slot], x * 64, t * kTileN, s.bh);
+                        ++kit;
+                    }
+                    {
+                        const uint32_t slot = vit % C::kVSlots, round = vit / C::kVSlots;
+                        ok = mbar_wait(&v_empty[slot], (round & 1) ^ 1, abort_p);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&v_full[slot], C::kTileBytes);
+                        for (int x = 0; x < C::kBoxes; ++x)
+                            tma_load_3d(sV + slot * C::kTileBytes + x * (kQTile * 128), &map_v, &v_full[slot], x * 64, t * kTileN, s.bh);
+                        ++vit;
+                    }
+                }
+                ++seg_idx;
+            }
+            if (!ok && base_ok) {
+                int dummy = 0;          // leave no copy in flight: what was armed last must land (bounded)
+                for (uint32_t back = 0; back < (uint32_t)C::kKSlots && back < kit; ++back) {
+                    const uint32_t id = kit - 1 - back;
+                    mbar_wait(&k_full[id % C::kKSlots], (id / C::kKSlots) & 1, &dummy, 200000000LL);
+                }
+                for (uint32_t back = 0; back < (uint32_t)C::kVSlots && back < vit; ++back) {
+                    const uint32_t id = vit - 1 - back;
+                    mbar_wait(&v_full[id % C::kVSlots], (id / C::kVSlots) & 1, &dummy, 200000000LL);
+                }
+                if (seg_idx > 0) mbar_wait(qdo_full, (seg_idx - 1) & 1, &dummy, 200000000LL);
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------------ MMA issuer (all lanes walk, one issues)
+        const uint32_t idesc_s = make_idesc_bf16(kQTile, kTileN, 0, 0);      // S, dP: M = queries, N = keys
+        const uint32_t idesc_dq = make_idesc_bf16(kQTile, D, 0, 1);          // dQ: A = dS in TMEM, B = K MN-major
+        const uint64_t kmaj = make_smem_desc_sw128(smem_u32(smem), 16, 1024);
+        const uint64_t mnmaj = make_smem_desc_sw128(smem_u32(smem), kQTile * 128, 1024);
+        const uint32_t desc_hi = (uint32_t)(kmaj >> 32);
+        const uint32_t kmaj_lo = (uint32_t)kmaj, mnmaj_lo = (uint32_t)mnmaj;
+        const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
+        auto issue_r = [&](int i, int a_byte_off, int b_byte_off) {        // R_i = A B^T (contraction over d)
+            const uint32_t a_lo = kmaj_lo + (uint32_t)(a_byte_off >> 4), b_lo = kmaj_lo + (uint32_t)(b_byte_off >> 4);
+            const uint32_t d = tmem_u + C::kColR + i * kTileN;
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t off16 = ((kk >> 2) * (kQTile * 128) + (kk & 3) * 32) >> 4;
+                if (elect_one()) mma_ss_parts(d, a_lo + off16, b_lo + off16, desc_hi, idesc_s, kk > 0);
+            }
+        };
+        auto issue_dq = [&](int i, int k_byte_off, bool accumulate) {       // dQ_i += dS_i K (contraction over keys)
+            const uint32_t b_lo = mnmaj_lo + (uint32_t)(k_byte_off >> 4);
+            const uint32_t d = tmem_u + C::kColDQ + i * D, a = tmem_u + C::kColR + i * kTileN;
+#pragma unroll
+            for (int kk = 0; kk < kTileN / 16; ++kk)
+                if (elect_one()) mma_ts_parts(d, a + kk * 8, b_lo + kk * (2048 >> 4), desc_hi, idesc_dq, (accumulate || kk > 0) ? 1u : 0u);
+        };
+        uint32_t kit = 0, vit = 0, seg_idx = 0;
+        uint32_t n_step[2] = {0, 0};
+        bool ok = base_ok;
+        SegmentWalker walk(p);
+        Segment s;
+        while (ok && walk.next(s)) {
+            const int row0 = s.qt * kTileM;
+            const int c0 = seg_count(s, tiles_allowed(p, row0, 0)), c1 = seg_count(s, tiles_allowed(p, row0, 1));
+            const int cnt = c0 > c1 ? c0 : c1;
+            if (cnt == 0) continue;
+            const int cq[2] = {c0, c1};
+            ok = __all_sync(0xffffffffu, mbar_wait(qdo_full, seg_idx & 1, abort_p));
+            if (!ok) break;
+            uint32_t ks = kit % C::kKSlots;
+            ok = __all_sync(0xffffffffu, mbar_wait(&k_full[ks], (kit / C::kKSlots) & 1, abort_p));
+            if (!ok) break;
+            tc_fence_after();
+            for (int i = 0; i < 2; ++i)
+                if (cq[i] > 0) {
+                    issue_r(i, C::kOffQ + i * C::kTileBytes, C::kOffK + ks * C::kTileBytes);
+                    commit_elected(&s_full[i]);
+                }
+            for (int j = 0; j < cnt && ok; ++j) {
+                const uint32_t vs = vit % C::kVSlots;
+                ok = __all_sync(0xffffffffu, mbar_wait(&v_full[vs], (vit / C::kVSlots) & 1, abort_p));
+                if (!ok) break;
+                ++vit;
+                for (int i = 0; i < 2 && ok; ++i) {
+                    if (j < cq[i]) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(&p_ready[i], n_step[i] & 1, abort_p));
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_r(i, C::kOffDO + i * C::kTileBytes, C::kOffV + vs * C::kTileBytes);   // dP over S
+                        commit_elected(&dp_full[i]);
+                    }
+                }
+                if (!ok) break;
+                commit_elected(&v_empty[vs]);
+                const bool have_next = j + 1 < cnt;
+                if (!have_next) commit_elected(qdo_empty);       // Q and dout of this segment have been read for the last time
+                uint32_t nks = 0;
+                if (have_next) {
+                    nks = (kit + 1) % C::kKSlots;
+                    ok = __all_sync(0xffffffffu, mbar_wait(&k_full[nks], ((kit + 1) / C::kKSlots) & 1, abort_p));
+                    if (!ok) break;
+                }
+                for (int i = 0; i < 2 && ok; ++i) {
+                    if (j < cq[i]) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(&ds_full[i], n_step[i] & 1, abort_p));
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_dq(i, C::kOffK + ks * C::kTileBytes, j > 0);
+                        ++n_step[i];
+                    }
+                    if (have_next && j + 1 < cq[i]) {
+                        tc_fence_after();
+                        issue_r(i, C::kOffQ + i * C::kTileBytes, C::kOffK + nks * C::kTileBytes);
+                        commit_elected(&s_full[i]);
+                    }
+                }
+                if (!ok) break;
+                commit_elected(&k_empty[ks]);
+                ++kit;
+                ks = nks;
+            }
+            if (!ok) break;
+            commit_elected(dq_done);
+            ++seg_idx;
+        }
+    }
+    } else {
+        // ------------------------------------------------------------------ elementwise warpgroups (one per Q tile)
+        setmaxnreg_inc<C::kComputeRegs>();
+        const int i = warp >> 2;
+        const int r = (warp & 3) * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tR = tmem_base + lane_addr + C::kColR + i * kTileN;
+        const uint32_t tDQ = tmem_base + lane_addr + C::kColDQ + i * D;
+        uint32_t n = 0, seg_idx = 0;
+        bool ok = base_ok;
+        SegmentWalker walk(p);
+        const int bh_first = (int)(walk.u / p.key_tiles);     // (b,h) of this CTA's first unit (used under schedule 0 only)
+        Segment s;
+        while (ok && walk.next(s)) {
+            const int row0 = s.qt * kTileM;
+            const int row = row0 + i * kQTile + r;
+            const int a0 = tiles_allowed(p, row0, 0), a1 = tiles_allowed(p, row0, 1);
+            const int c0 = seg_count(s, a0), c1 = seg_count(s, a1);
+            if ((c0 > c1 ? c0 : c1) == 0) continue;           // the MMA warp skips this segment too
+            const int allowed_i = i == 0 ? a0 : a1, cnt_i = i == 0 ? c0 : c1;
+            const long long lim_row_ll = p.causal ? (long long)p.N - p.W + row + 1 : (long long)p.N;
+            const int lim_row = (int)(lim_row_ll < p.N ? lim_row_ll : p.N);
+            const long long lim_warp_ll = p.causal ? (long long)p.N - p.W + (row - lane) + 1 : (long long)p.N;
+            const int lim_warp = (int)(lim_warp_ll < p.N ? lim_warp_ll : p.N);
+            const bool row_ok = row < p.W;
+            const float l2 = row_ok ? p.lse2[(long long)s.bh * p.Wpad + row] : CUDART_INF_F;
+            const float dl = row_ok ? p.delta[(long long)s.bh * p.Wpad + row] : 0.f;
+            for (int j = 0; j < cnt_i; ++j) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&s_full[i], n & 1, abort_p));
+                if (!ok) break;
+                tc_fence_after();
+                const int k0 = (s.t_begin + j) * kTileN;
+                const bool masked = k0 + kTileN > lim_warp;
+                const int nvalid = lim_row - k0;
+                uint32_t sv[kTileN / 32][32];
+#pragma unroll
+                for (int c = 0; c < kTileN / 32; ++c) tmem_ld32_async(tR + c * 32, sv[c]);
+#pragma unroll
+                for (int c = 0; c < kTileN / 32; ++c) tmem_wait_ld(sv[c]);
+                tc_fence_before();
+                mbar_arrive(&p_ready[i]);                      // S is in registers: dP may overwrite it
+                // p = 2^(s*scale*log2e - lse*log2e), kept as fp32 in the registers that held s
+#pragma unroll
+                for (int e = 0; e < kTileN; ++e) {
+                    float pe = ex2(fmaf(__uint_as_float(sv[e >> 5][e & 31]), p.scale_log2e, -l2));
+                    if (masked && e >= nvalid) pe = 0.f;
+                    sv[e >> 5][e & 31] = __float_as_uint(pe);
+                }
+                ok = __all_sync(0xffffffffu, mbar_wait(&dp_full[i], n & 1, abort_p));
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int c = 0; c < kTileN / 16; ++c) {
+                    uint32_t dp[16];
+                    tmem_ld16_async(tR + c * 16, dp);
+                    tmem_wait_ld16(dp);
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float d0 = __uint_as_float(sv[c >> 1][(c & 1) * 16 + 2 * e]) * (__uint_as_float(dp[2 * e]) - dl);
+                        const float d1 = __uint_as_float(sv[c >> 1][(c & 1) * 16 + 2 * e + 1]) * (__uint_as_float(dp[2 * e + 1]) - dl);
+                        pk[e] = pack_bf16x2(d0, d1);
+                    }
+                    tmem_st8(tR + c * 8, pk);                 // bf16 dS over columns of dP that are already in registers
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(&ds_full[i]);
+                ++n;
+            }
+            if (!ok) break;
+            const uint32_t my_seg = seg_idx++;
+            if (allowed_i == 0) continue;                      // this Q tile does not exist
+            // ---------------------------------------------------------------- dQ of the segment
+            if (cnt_i > 0) {
+                ok = __all_sync(0xffffffffu, mbar_wait(dq_done, my_seg & 1, abort_p));
+                if (!ok) break;
+                tc_fence_after();
+            }
+            const bool whole = s.t_begin == 0 && s.t_end == p.key_tiles;
+            if (whole) {
+                __nv_bfloat16* drow = reinterpret_cast<__nv_bfloat16*>(p.dq) + ((long long)s.bh * p.W + row) * D;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t o[32];
+                    if (cnt_i > 0) tmem_ld32(tDQ + c * 32, o);
+                    if (row_ok) {
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            uint4 w;
+                            w.x = pack_bf16x2(__uint_as_float(o[v4 * 8 + 0]) * p.scale, __uint_as_float(o[v4 * 8 + 1]) * p.scale);
+                            w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * p.scale, __uint_as_float(o[v4 * 8 + 3]) * p.scale);
+                            w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * p.scale, __uint_as_float(o[v4 * 8 + 5]) * p.scale);
+                            w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * p.scale, __uint_as_float(o[v4 * 8 + 7]) * p.scale);
+                            if (cnt_i == 0) w = make_uint4(0, 0, 0, 0);
+                            *reinterpret_cast<uint4*>(drow + c * 32 + v4 * 8) = w;
+                        }
+                    }
+                }
+            } else {
+                // partial sum -> workspace slot (0: first segment of this CTA's range, 1: a later one); unscaled fp32
+                const int slot = s.bh == bh_first ? 0 : 1;
+                float* orow = p.ws + ((long long)blockIdx.x * 2 + slot) * (long long)kTileM * D + (long long)(i * kQTile + r) * D;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t o[32];
+                    if (cnt_i > 0) tmem_ld32(tDQ + c * 32, o);
+#pragma unroll
+                    for (int v4 = 0; v4 < 8; ++v4) {
+                        float4 w;
+                        w.x = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 0]) : 0.f;
+                        w.y = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 1]) : 0.f;
+                        w.z = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 2]) : 0.f;
+                        w.w = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 3]) : 0.f;
+                        *reinterpret_cast<float4*>(orow + c * 32 + v4 * 4) = w;
+                    }
+                }
+            }
+            tc_fence_before();
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, base_ok ? (int)TLIN_ERR_TIMEOUT : (int)TLIN_ERR_CUDA);
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// Adds the partial dQ of every (b,h) whose key tiles were split between groups, scales and rounds to bf16.
+// One CTA per 8 query rows of a (b,h, 256-row tile): one warp per row.
+template <int D>
+__global__ void __launch_bounds__(256)
+bwd_dq_reduce_kernel(const BwdParams p) {
+    constexpr int CPL = D / 32;
+    const int blocks_per_tile = kTileM / 8;
+    const int part = blockIdx.x % blocks_per_tile;
+    const int tile_id = blockIdx.x / blocks_per_tile;       // bh * q_tiles + qt
+    const int bh = tile_id / p.q_tiles, qt = tile_id - bh * p.q_tiles;
+    const unsigned long long T = (unsigned long long)p.key_tiles, U = (unsigned long long)p.total_units, G = (unsigned)p.n_groups;
+    // groups holding the first and the last unit of this (b,h): largest g with floor(g*U/G) <= x
+    const unsigned long long x0 = (unsigned long long)bh * T, x1 = x0 + T - 1;
+    const int g_lo = (int)(((x0 + 1) * G - 1) / U), g_hi = (int)(((x1 + 1) * G - 1) / U);
+    if (g_hi == g_lo) return;                               // written directly by the dQ kernel
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rr = part * 8 + warp;
+    const int row = qt * kTileM + rr;
+    if (row >= p.W) return;
+    float acc[CPL];
+#pragma unroll
+    for (int e = 0; e < CPL; ++e) acc[e] = 0.f;
+    for (int g = g_lo; g <= g_hi; ++g) {
+        const int cta = g * p.q_tiles + qt;
+        const int slot = bh == (int)((((unsigned long long)g * U) / G) / T) ? 0 : 1;
+        const float* src = p.ws + ((long long)cta * 2 + slot) * (long long)kTileM * D + (long long)rr * D + lane * CPL;
+#pragma unroll
+        for (int e = 0; e < CPL; ++e) acc[e] += src[e];
+    }
+    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.dq) + ((long long)bh * p.W + row) * D + lane * CPL;
+#pragma unroll
+    for (int e = 0; e < CPL; e += 2)
+        *reinterpret_cast<uint32_t*>(dst + e) = pack_bf16x2(acc[e] * p.scale, acc[e + 1] * p.scale);
+}
+
+// ------------------------------------------------------------------------------------------ host side
+template <int D>
+int launch_d(const void* q, const void* k, const void* v, const void* out, const float* lse, const void* dout,
+             void* dq, void* dk, void* dv, int B, int H, int N, int W, int causal, const tlin_fwd_plan& plan,
+             float* ws, int num_sms, cudaStream_t st) {
+    const long long bh = (long long)B * H;
+    const int Wpad = (W + kQTile - 1) / kQTile * kQTile;
+    CUtensorMap mq, mk, mv, mdo;
+    int rc = make_map(&mq, q, D, W, bh);
+    if (rc == TLIN_OK) rc = make_map(&mk, k, D, N, bh);
+    if (rc == TLIN_OK) rc = make_map(&mv, v, D, N, bh);
+    if (rc == TLIN_OK) rc = make_map(&mdo, dout, D, W, bh);
+    if (rc != TLIN_OK) return rc;
+    BwdParams p;
+    float* lse2 = ws;
+    float* delta = ws + bh * Wpad;
+    p.lse2 = lse2; p.delta = delta; p.dq = dq; p.dk = dk; p.dv = dv;
+    p.ws = ws + 2 * bh * Wpad;
+    p.status = status_word();
+    if (!p.status) return TLIN_ERR_CUDA;
+    p.key_tiles = (N + kTileN - 1) / kTileN;
+    p.q_tiles128 = Wpad / kQTile;
+    p.N = N; p.W = W; p.Wpad = Wpad; p.causal = causal;
+    p.scale = 1.f / sqrtf((float)D);
+    p.scale_log2e = kLog2e * p.scale;
+    static std::once_flag attr_once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(attr_once, [] {
+        attr_err = cudaFuncSetAttribute(bwd_dkdv_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, ACfg<D>::kSmemBytes);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(bwd_dq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, BCfg<D>::kSmemBytes);
+    });
+    TLIN_CUDA_CHECK(attr_err);
+    const long long rows_padded = bh * Wpad;
+    bwd_prep_kernel<D><<<(unsigned)((rows_padded + 7) / 8), 256, 0, st>>>(
+        (const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse, lse2, delta, W, Wpad, rows_padded);
+    TLIN_CUDA_CHECK(cudaGetLastError());
+    // dK, dV: the units are (b,h,key tile); a CTA takes a contiguous run of them
+    BwdParams pa = p;
+    pa.total_units = bh * p.key_tiles;
+    pa.n_groups = 0; pa.q_tiles = 0; pa.schedule = 0;
+    const long long ctas_a = pa.total_units < num_sms ? pa.total_units : num_sms;
+    bwd_dkdv_tc_kernel<D><<<(unsigned)ctas_a, ACfg<D>::kThreads, ACfg<D>::kSmemBytes, st>>>(mq, mk, mv, mdo, pa);
+    TLIN_CUDA_CHECK(cudaGetLastError());
+    // dQ: the forward's plan
+    BwdParams pb = p;
+    pb.total_units = plan.total_units; pb.n_groups = plan.n_groups; pb.q_tiles = plan.q_tiles; pb.schedule = plan.schedule;
+    bwd_dq_tc_kernel<D><<<plan.n_ctas, BCfg<D>::kThreads, BCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mdo, pb);
+    TLIN_CUDA_CHECK(cudaGetLastError());
+    count_launch(3);
+    if (plan.uses_workspace) {
+        bwd_dq_reduce_kernel<D><<<(unsigned)(bh * plan.q_tiles * (kTileM / 8)), 256, 0, st>>>(pb);
+        TLIN_CUDA_CHECK(cudaGetLastError());
+        count_launch();
+    }
+    return TLIN_OK;
+}
+
+}  // namespace
+
+// row statistics (lse2, delta, padded) + the dQ kernel's partial slots
+size_t bwd_tc_workspace_bytes(long long B, long long H, long long W, int d, const tlin_fwd_plan& plan) {
+    const long long bh = B * H, Wpad = (W + tc::kQTile - 1) / tc::kQTile * tc::kQTile;
+    long long floats = 2 * bh * Wpad;
+    if (plan.uses_workspace) floats += (long long)plan.n_ctas * 2 * tc::kTileM * d;
+    return (size_t)floats * sizeof(float);
+}
+
+int launch_bwd_tc(const void* q, const void* k, const void* v, const void* out, const float* lse, const void* dout,
+                  void* dq, void* dk, void* dv, int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& plan,
+                  float* ws, int num_sms, cudaStream_t st) {
+    if (plan.tile_m != tc::kTileM || plan.tile_n != kTileN || !plan.tensor_path) return TLIN_ERR_UNSUPPORTED;
+    if ((long long)B * H * W > 0x7fffffffLL || (long long)B * H > 0x7fffffffLL) return TLIN_ERR_UNSUPPORTED;
+    if (d == 128) return launch_d<128>(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, causal, plan, ws, num_sms, st);
+    if (d == 64) return launch_d<64>(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, causal, plan, ws, num_sms, st);
+    return TLIN_ERR_UNSUPPORTED;
+}
+
+}  // namespace tlin

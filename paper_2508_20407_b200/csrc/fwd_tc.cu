@@ -19,6 +19,7 @@
 // Every wait is bounded: on expiry the CTA sets the library's error word, drains and exits.
 #include "tlin_internal.h"
 #include "sm100_ptx.cuh"
+#include "tc_common.cuh"
 #include <math_constants.h>
 #include <mutex>
 
@@ -26,9 +27,8 @@ namespace tlin {
 namespace {
 
 using namespace ptx;
+using namespace tc;
 
-constexpr int kQTile = 128;                 // rows per Q tile (one TMEM lane per row)
-constexpr int kTileM = 2 * kQTile;          // rows per CTA
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr int kThreads = 32 * 12;          // warps 10 and 11 only lend their registers
@@ -84,58 +84,6 @@ struct Params {
     int schedule;         // 0: groups of q_tiles CTAs stream key ranges; 1: every CTA walks whole (b,h,q-tile) problems
     float scale_log2e;
 };
-
-// Work of one CTA as a list of segments: a (b,h), a pair of Q tiles (256 query rows) and a range of key tiles.
-// Schedule 0: CTA = (group, q-tile pair); the group's unit range [u, u1) over (b,h,key tile) is cut at the (b,h)
-// borders.  Schedule 1: the units are whole (b,h,q-tile pair) problems and a CTA takes a contiguous run of them.
-struct Segment { int bh, qt, t_begin, t_end; };
-
-struct SegmentWalker {
-    long long u, u1;
-    int T, q_tiles, qt_fixed, schedule;
-    __device__ SegmentWalker(const Params& p) : T(p.key_tiles), q_tiles(p.q_tiles), schedule(p.schedule) {
-        const int g = schedule == 0 ? (int)(blockIdx.x / p.q_tiles) : (int)blockIdx.x;
-        qt_fixed = schedule == 0 ? (int)(blockIdx.x - g * p.q_tiles) : 0;
-        u = (long long)(((unsigned long long)g * (unsigned long long)p.total_units) / (unsigned)p.n_groups);
-        u1 = (long long)(((unsigned long long)(g + 1) * (unsigned long long)p.total_units) / (unsigned)p.n_groups);
-    }
-    __device__ bool next(Segment& s) {
-        if (u >= u1) return false;
-        if (schedule != 0) {
-            s.bh = (int)(u / q_tiles);
-            s.qt = (int)(u - (long long)s.bh * q_tiles);
-            s.t_begin = 0;
-            s.t_end = T;
-            ++u;
-            return true;
-        }
-        s.qt = qt_fixed;
-        s.bh = (int)(u / T);
-        s.t_begin = (int)(u - (long long)s.bh * T);
-        const long long left = u1 - u;
-        s.t_end = (int)((long long)s.t_begin + left < (long long)T ? (long long)s.t_begin + left : (long long)T);
-        u += s.t_end - s.t_begin;
-        return true;
-    }
-};
-
-__device__ __forceinline__ void commit_elected(uint64_t* bar) {
-    if (elect_one()) tc_commit(bar);
-}
-
-// Number of key tiles Q tile `i` of this CTA may use at all (0 if the tile lies beyond W).
-__device__ __forceinline__ int tiles_allowed(const Params& p, int row0, int i) {
-    const int r_first = row0 + i * kQTile;
-    if (r_first >= p.W) return 0;
-    if (!p.causal) return p.key_tiles;
-    const long long r_end = r_first + kQTile < p.W ? r_first + kQTile : p.W;     // one past the last row
-    const long long keys = (long long)p.N - p.W + r_end;                        // keys visible to the last row
-    return (int)((keys + kTileN - 1) / kTileN);
-}
-__device__ __forceinline__ int seg_count(const Segment& s, int allowed) {
-    const int e = s.t_end < allowed ? s.t_end : allowed;
-    return e > s.t_begin ? e - s.t_begin : 0;
-}
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -617,42 +565,6 @@ fwd_merge_kernel(const Params p) {
             if (p.lse != nullptr && lane == 0) p.lse[(long long)bh * p.W + row] = m + logf(z);
         }
     }
-}
-
-// ---------------------------------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        void* f = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(f);
-    });
-    return fn;
-}
-
-// [BH, rows, D] bf16, box = 64 elements x 128 rows x 1, 128-byte swizzle, zero fill outside.
-int make_map(CUtensorMap* m, const void* ptr, int D, long long rows, long long bh) {
-    EncodeTiledFn enc = encode_fn();
-    if (!enc) return TLIN_ERR_CUDA;
-    cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)bh};
-    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)rows * D * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)kQTile, 1};
-    cuuint32_t es[3] = {1, 1, 1};
-    const CUresult rc = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (rc != CUDA_SUCCESS) {
-        fprintf(stderr, "libtlin: cuTensorMapEncodeTiled failed (%d)\n", (int)rc);
-        return TLIN_ERR_CUDA;
-    }
-    return TLIN_OK;
 }
 
 template <int D>

@@ -21,12 +21,19 @@ DEV = "cuda"
 REL_L2, REL_MAX, ABS_FLOOR = 2e-2, 2e-2, 1e-5
 
 
-def grads(q, k, v, dout, causal):
+IMPLS = [0, 1]      # 0: tensor-core kernels, 1: CUDA-core kernels (the same switch as the forward's)
+
+
+def grads(q, k, v, dout, causal, impl=0):
     out, lse = tl.tlin_attn_forward(q, k, v, causal_window=causal)
-    dq, dk, dv = tl.tlin_attn_backward(q, k, v, out, lse, dout, causal_window=causal)
-    torch.cuda.synchronize()
-    assert tl.tlin_get_status() == 0
-    assert tl.tlin_last_launch_count() >= 3
+    prev = tl.tlin_set_forward_impl(impl)
+    try:
+        dq, dk, dv = tl.tlin_attn_backward(q, k, v, out, lse, dout, causal_window=causal)
+        torch.cuda.synchronize()
+        assert tl.tlin_get_status() == 0
+        assert tl.tlin_last_launch_count() >= 3
+    finally:
+        tl.tlin_set_forward_impl(prev)
     return dq, dk, dv
 
 
@@ -41,16 +48,16 @@ def compare(got, ref, what):
     return e
 
 
-def run_case(B, H, N, W, d, causal, seed, peaky=False):
+def run_case(B, H, N, W, d, causal, seed, peaky=False, impl=0):
     wl = synth.Workload("bwd", B, H, d, N, W, seed=seed, causal_window=causal)
     q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
     if peaky:
         q = (q.float() * 6.0).to(torch.bfloat16)
     g = torch.Generator(device="cpu").manual_seed(seed + 7)
     dout = torch.randn(q.shape, generator=g, dtype=torch.float32).to(torch.bfloat16).to(DEV)
-    dq, dk, dv = grads(q, k, v, dout, causal)
+    dq, dk, dv = grads(q, k, v, dout, causal, impl)
     rq, rk, rv = oracle.attn_backward(q.cpu(), k.cpu(), v.cpu(), dout.cpu(), causal)
-    tag = f"B{B} H{H} N{N} W{W} d{d} causal{causal}"
+    tag = f"B{B} H{H} N{N} W{W} d{d} causal{causal} impl{impl}"
     compare(dq, rq, tag + " dq")
     compare(dk, rk, tag + " dk")
     compare(dv, rv, tag + " dv")
@@ -64,22 +71,37 @@ SHAPES = [  # B, H, N, W, d, causal: single elements, ragged tails on both axes,
 ]
 
 
+@pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("B,H,N,W,d,causal", SHAPES)
-def test_backward_elementwise(B, H, N, W, d, causal):
-    run_case(B, H, N, W, d, causal, seed=300 + N + W)
+def test_backward_elementwise(B, H, N, W, d, causal, impl):
+    run_case(B, H, N, W, d, causal, seed=300 + N + W, impl=impl)
 
 
-def test_backward_cfg1_tiny():
+@pytest.mark.parametrize("impl", IMPLS)
+def test_backward_cfg1_tiny(impl):
     wl = synth.WORKLOADS["cfg1_tiny"]
-    run_case(wl.B, wl.H, wl.N, wl.W, wl.d, wl.causal_window, seed=wl.seed)
+    run_case(wl.B, wl.H, wl.N, wl.W, wl.d, wl.causal_window, seed=wl.seed, impl=impl)
 
 
-def test_backward_peaked_softmax():
+@pytest.mark.parametrize("impl", IMPLS)
+def test_backward_peaked_softmax(impl):
     # scores large enough that most rows put nearly all weight on one key: exercises exp(s - lse) near 1 and near 0
-    run_case(1, 2, 700, 96, 128, 1, seed=11, peaky=True)
+    run_case(1, 2, 700, 96, 128, 1, seed=11, peaky=True, impl=impl)
 
 
-def test_backward_keys_outside_every_window_get_zero_gradient():
+# many CTAs per (b,h) on the dQ side (key range split between groups, partial sums added by the reduce kernel), several
+# key tiles per CTA on the dK/dV side, both schedules of the plan
+BIG = [(1, 2, 40000, 300, 128, 1), (2, 3, 20000, 520, 64, 1), (1, 160, 384, 512, 64, 0), (6, 16, 1024, 1000, 64, 1),
+       (1, 1, 30000, 1024, 128, 0)]
+
+
+@pytest.mark.parametrize("B,H,N,W,d,causal", BIG)
+def test_backward_tensor_core_schedules(B, H, N, W, d, causal):
+    run_case(B, H, N, W, d, causal, seed=500 + N + W, impl=0)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_backward_keys_outside_every_window_get_zero_gradient(impl):
     # with the window rule the last key is visible to the last query only; a key count N == W makes key j invisible
     # to queries i < j.  Zero dout rows for the queries that see the tail => exact zeros in dk, dv there.
     B, H, N, W, d = 1, 2, 160, 160, 64
@@ -87,20 +109,29 @@ def test_backward_keys_outside_every_window_get_zero_gradient():
     q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
     dout = torch.randn(q.shape, device=DEV).to(torch.bfloat16)
     dout[:, :, 100:, :] = 0
-    _, dk, dv = grads(q, k, v, dout, 1)
+    _, dk, dv = grads(q, k, v, dout, 1, impl)
     assert float(dk[:, :, 100:, :].float().abs().max()) == 0.0
     assert float(dv[:, :, 100:, :].float().abs().max()) == 0.0
     assert float(dk[:, :, :100, :].float().abs().max()) > 0.0
 
 
-def test_backward_is_deterministic_up_to_the_dq_sum_order():
+def test_backward_tensor_core_path_is_bitwise_repeatable():
+    wl = synth.Workload("bwd", 1, 2, 128, 30000, 300, seed=9, causal_window=1)
+    q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
+    dout = torch.randn(q.shape, device=DEV).to(torch.bfloat16)
+    a = grads(q, k, v, dout, 1, 0)
+    b = grads(q, k, v, dout, 1, 0)
+    assert all(torch.equal(x, y) for x, y in zip(a, b))
+
+
+def test_backward_cuda_core_path_is_deterministic_up_to_the_dq_sum_order():
     # dk, dv have one owner per element: bitwise repeatable.  dq is summed over key slices with atomics: equal within
     # fp32 rounding, so the rounded bf16 values may differ in the last place only.
     wl = synth.Workload("bwd", 1, 2, 128, 3000, 64, seed=9, causal_window=1)
     q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
     dout = torch.randn(q.shape, device=DEV).to(torch.bfloat16)
-    a = grads(q, k, v, dout, 1)
-    b = grads(q, k, v, dout, 1)
+    a = grads(q, k, v, dout, 1, 1)
+    b = grads(q, k, v, dout, 1, 1)
     assert torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])
     diff = (a[0].float() - b[0].float()).abs()
     assert float((diff / (a[0].float().abs() + 1e-20)).max()) <= 2.0 ** -7
