@@ -11,8 +11,9 @@
 //   see it.  Scores are computed TRANSPOSED (S^T = K Q^T, dP^T = V dout^T: TMEM lane = key, column = query) so that
 //   P^T and dS^T, written back to TMEM as bf16, are directly the A operands of dV += P^T dout and dK += dS^T Q, whose
 //   B operands are the dout / Q tiles already in shared memory (read MN-major).  dK and dV stay in TMEM for the whole
-//   key tile and are written once.  One TMEM region holds S^T and then dP^T of a step; 256 threads (key row x half
-//   of the query columns) do the elementwise work.
+//   key tile and are written once.  Each 128-query tile is worked on as two independent chains of 64 queries, one per
+//   warpgroup (thread = key row): S^T_x -> P^T_x, then dP^T_x over the same TMEM columns -> dS^T_x; while one chain does
+//   its elementwise work the tensor pipe serves the other.
 //
 // bwd_dq_tc_kernel     The forward's structure: a CTA owns 256 query rows (two Q tiles, one warpgroup each, one
 //   thread per row) and streams 128-key tiles; per tile S = Q K^T -> p (kept in registers), then dP = dout V^T into
@@ -97,10 +98,11 @@ struct ACfg {
     static constexpr int kOffDO = 6 * kTileBytes;
     static constexpr int kOffStats = 7 * kTileBytes;
     static constexpr int kOffBars = kOffStats + 2 * 256 * 4;
-    static constexpr int kNumBars = 18;
+    static constexpr int kNumBars = 22;
     static constexpr int kSmemBytes = kOffBars + kNumBars * 8 + 16;
-    // TMEM columns: dK, dV (D each), R = S^T then dP^T (128), P^T then dS^T as bf16 (64)
-    static constexpr uint32_t kColDK = 0, kColDV = D, kColR = 2 * D, kColP = 2 * D + 128;
+    // TMEM columns: dK, dV (D each); per chain x (64 queries of the tile): R_x = S^T then dP^T (64 fp32 columns),
+    // P^T_x and dS^T_x as bf16 (32 columns each)
+    static constexpr uint32_t kColDK = 0, kColDV = D, kColR = 2 * D, kColP = 2 * D + 128, kColDS = 2 * D + 192;
     static constexpr int kThreads = 32 * 10;
 };
 
@@ -128,14 +130,13 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     uint64_t* q_empty = bars + 6;     // [2]
     uint64_t* do_full = bars + 8;
     uint64_t* do_empty = bars + 9;
-    uint64_t* s_full = bars + 10;     // S^T of a step is in R
-    uint64_t* p_full = bars + 11;     // all threads have read S^T and stored P^T
-    uint64_t* dp_full = bars + 12;    // dP^T is in R
-    uint64_t* r_free = bars + 13;     // all threads have read dP^T
-    uint64_t* dv_done = bars + 14;    // the dV MMAs have consumed P^T
-    uint64_t* ds_full = bars + 15;    // all threads have stored dS^T
-    uint64_t* acc_full = bars + 16;   // dK, dV of the key tile are complete
-    uint64_t* acc_empty = bars + 17;  // all threads have read them
+    uint64_t* s_full = bars + 10;     // [2] S^T of chain x is in R_x
+    uint64_t* p_full = bars + 12;     // [2] the chain's threads have read S^T and stored P^T
+    uint64_t* dp_full = bars + 14;    // [2] dP^T is in R_x
+    uint64_t* r_free = bars + 16;     // [2] the chain's threads have read dP^T
+    uint64_t* ds_full = bars + 18;    // [2] the chain's threads have stored dS^T
+    uint64_t* acc_full = bars + 20;   // dK, dV of the key tile are complete
+    uint64_t* acc_empty = bars + 21;  // all threads have read them
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::kNumBars);
     int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
 
@@ -152,12 +153,13 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
         mbar_init(do_full, 1);
         mbar_init(do_empty, 1);
-        mbar_init(s_full, 1);
-        mbar_init(p_full, 256);
-        mbar_init(dp_full, 1);
-        mbar_init(r_free, 256);
-        mbar_init(dv_done, 1);
-        mbar_init(ds_full, 256);
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(&s_full[x], 1);
+            mbar_init(&p_full[x], 128);
+            mbar_init(&dp_full[x], 1);
+            mbar_init(&r_free[x], 128);
+            mbar_init(&ds_full[x], 128);
+        }
         mbar_init(acc_full, 1);
         mbar_init(acc_empty, 256);
         fence_mbar_init();
@@ -231,26 +233,30 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issuer (all lanes walk, one issues)
-        const uint32_t idesc_st = make_idesc_bf16(kQTile, kTileN, 0, 0);     // S^T, dP^T: M = keys, N = queries
+        const uint32_t idesc_st = make_idesc_bf16(kQTile, 64, 0, 0);         // S^T, dP^T of a chain: M = keys, N = 64 queries
         const uint32_t idesc_acc = make_idesc_bf16(kQTile, D, 0, 1);         // dV, dK: A in TMEM, B MN-major
         const uint64_t kmaj = make_smem_desc_sw128(smem_u32(smem), 16, 1024);
         const uint64_t mnmaj = make_smem_desc_sw128(smem_u32(smem), kQTile * 128, 1024);
         const uint32_t desc_hi = (uint32_t)(kmaj >> 32);
         const uint32_t kmaj_lo = (uint32_t)kmaj, mnmaj_lo = (uint32_t)mnmaj;
         const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
-        const uint32_t tDK = tmem_u + C::kColDK, tDV = tmem_u + C::kColDV, tR = tmem_u + C::kColR, tP = tmem_u + C::kColP;
+        const uint32_t tDK = tmem_u + C::kColDK, tDV = tmem_u + C::kColDV;
         auto tile_off = [&](int byte_off) { return (uint32_t)(byte_off >> 4); };
-        auto issue_st = [&](uint32_t a_off, uint32_t b_off) {       // R = A B^T, both tiles K-major, contraction over d
+        // R_x = A B_x^T: A a whole K-major tile (K or V), B_x rows [64x, 64x+64) of a K-major tile (Q or dout)
+        auto issue_st = [&](int x, uint32_t a_off, uint32_t b_off) {
+            const uint32_t d = tmem_u + C::kColR + x * 64, b_rows = (uint32_t)(x * 64 * 128) >> 4;
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
                 const uint32_t off16 = ((kk >> 2) * (kQTile * 128) + (kk & 3) * 32) >> 4;
-                if (elect_one()) mma_ss_parts(tR, kmaj_lo + a_off + off16, kmaj_lo + b_off + off16, desc_hi, idesc_st, kk > 0);
+                if (elect_one()) mma_ss_parts(d, kmaj_lo + a_off + off16, kmaj_lo + b_off + b_rows + off16, desc_hi, idesc_st, kk > 0);
             }
         };
-        auto issue_acc = [&](uint32_t d_tmem, uint32_t b_off, bool accumulate) {   // D += P^T(TMEM) B, contraction over queries
+        // D += A_x B_x: A_x = P^T or dS^T of the chain (TMEM, 64 queries), B_x rows [64x, 64x+64) of an MN-major tile
+        auto issue_acc = [&](int x, uint32_t d_tmem, uint32_t a_col, uint32_t b_off, bool accumulate) {
+            const uint32_t a = tmem_u + a_col + x * 32;
 #pragma unroll
-            for (int kk = 0; kk < kQTile / 16; ++kk)
-                if (elect_one()) mma_ts_parts(d_tmem, tP + kk * 8, mnmaj_lo + b_off + kk * (2048 >> 4), desc_hi, idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+            for (int kk = 0; kk < 4; ++kk)
+                if (elect_one()) mma_ts_parts(d_tmem, a + kk * 8, mnmaj_lo + b_off + (x * 4 + kk) * (2048 >> 4), desc_hi, idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
         };
         bool ok = base_ok;
         uint32_t g = 0, n = 0;
@@ -265,37 +271,49 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             ok = __all_sync(0xffffffffu, mbar_wait(&q_full[g & 1], (g >> 1) & 1, abort_p));
             if (!ok) break;
             tc_fence_after();
-            issue_st(k_off, tile_off(C::kOffQ + (g & 1) * C::kTileBytes));
-            commit_elected(s_full);
+            for (int x = 0; x < 2; ++x) {
+                issue_st(x, k_off, tile_off(C::kOffQ + (g & 1) * C::kTileBytes));
+                commit_elected(&s_full[x]);
+            }
             for (int s = 0; s < steps && ok; ++s, ++g) {
                 const uint32_t q_off = tile_off(C::kOffQ + (g & 1) * C::kTileBytes);
-                ok = __all_sync(0xffffffffu, mbar_wait(p_full, g & 1, abort_p));
-                if (!ok) break;
-                ok = __all_sync(0xffffffffu, mbar_wait(do_full, g & 1, abort_p));
-                if (!ok) break;
-                if (s == 0 && n > 0) {          // the previous key tile's dK, dV must have been read out
-                    ok = __all_sync(0xffffffffu, mbar_wait(acc_empty, (n - 1) & 1, abort_p));
+                for (int x = 0; x < 2 && ok; ++x) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&p_full[x], g & 1, abort_p));
                     if (!ok) break;
+                    if (x == 0) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(do_full, g & 1, abort_p));
+                        if (!ok) break;
+                        if (s == 0 && n > 0) {      // the previous key tile's dK, dV must have been read out
+                            ok = __all_sync(0xffffffffu, mbar_wait(acc_empty, (n - 1) & 1, abort_p));
+                            if (!ok) break;
+                        }
+                    }
+                    tc_fence_after();
+                    issue_st(x, v_off, do_off);                 // dP^T over S^T: the chain's threads have read S^T (p_full)
+                    commit_elected(&dp_full[x]);
+                    issue_acc(x, tDV, C::kColP, do_off, s > 0 || x > 0);
                 }
-                tc_fence_after();
-                issue_st(v_off, do_off);                    // dP^T over S^T: every thread has read S^T (p_full)
-                commit_elected(dp_full);
-                issue_acc(tDV, do_off, s > 0);
-                commit_elected(dv_done);
+                if (!ok) break;
                 commit_elected(do_empty);
-                if (s + 1 < steps) {                        // next step's S^T as soon as dP^T has been read
+                const bool have_next = s + 1 < steps;
+                if (have_next) {
                     ok = __all_sync(0xffffffffu, mbar_wait(&q_full[(g + 1) & 1], ((g + 1) >> 1) & 1, abort_p));
                     if (!ok) break;
-                    ok = __all_sync(0xffffffffu, mbar_wait(r_free, g & 1, abort_p));
+                }
+                for (int x = 0; x < 2 && ok; ++x) {
+                    if (have_next) {                            // next step's S^T as soon as dP^T has been read
+                        ok = __all_sync(0xffffffffu, mbar_wait(&r_free[x], g & 1, abort_p));
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_st(x, k_off, tile_off(C::kOffQ + ((g + 1) & 1) * C::kTileBytes));
+                        commit_elected(&s_full[x]);
+                    }
+                    ok = __all_sync(0xffffffffu, mbar_wait(&ds_full[x], g & 1, abort_p));
                     if (!ok) break;
                     tc_fence_after();
-                    issue_st(k_off, tile_off(C::kOffQ + ((g + 1) & 1) * C::kTileBytes));
-                    commit_elected(s_full);
+                    issue_acc(x, tDK, C::kColDS, q_off, s > 0 || x > 0);
                 }
-                ok = __all_sync(0xffffffffu, mbar_wait(ds_full, g & 1, abort_p));
                 if (!ok) break;
-                tc_fence_after();
-                issue_acc(tDK, q_off, s > 0);
                 commit_elected(&q_empty[g & 1]);
             }
             if (!ok) break;
@@ -304,11 +322,12 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
     } else {
         // ------------------------------------------------------------------ elementwise threads
-        const int wg = warp >> 2;                              // which half of the query columns
+        const int wg = warp >> 2;                              // chain: which 64 queries of every tile
         const int r = (warp & 3) * 32 + lane;                  // key row inside the tile == TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tR = tmem_base + lane_addr + C::kColR + wg * 64;
         const uint32_t tP = tmem_base + lane_addr + C::kColP + wg * 32;
+        const uint32_t tDS = tmem_base + lane_addr + C::kColDS + wg * 32;
         bool ok = base_ok;
         uint32_t g = 0, n = 0;
         for (long long u = u_begin; u < u_end && ok; ++u, ++n) {
@@ -321,7 +340,7 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             for (int i = i_first; i < p.q_tiles128; ++i, ++g) {
                 const float* st = sStats + (g & 1) * 256 + wg * 64;
                 const int q0 = i * kQTile + wg * 64;              // first query of this thread's columns
-                ok = __all_sync(0xffffffffu, mbar_wait(s_full, g & 1, abort_p));
+                ok = __all_sync(0xffffffffu, mbar_wait(&s_full[wg], g & 1, abort_p));
                 if (!ok) break;
                 // already complete (the S^T MMAs waited for it); observing it here orders the bulk-copied lse2 / delta
                 // before this thread's reads
@@ -356,8 +375,8 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
                 tc_wait_st();
                 tc_fence_before();
-                mbar_arrive(p_full);
-                ok = __all_sync(0xffffffffu, mbar_wait(dp_full, g & 1, abort_p));
+                mbar_arrive(&p_full[wg]);
+                ok = __all_sync(0xffffffffu, mbar_wait(&dp_full[wg], g & 1, abort_p));
                 if (!ok) break;
                 tc_fence_after();
                 tmem_ld32_async(tR, sv[0]);
@@ -365,7 +384,7 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 tmem_wait_ld(sv[0]);
                 tmem_wait_ld(sv[1]);
                 tc_fence_before();
-                mbar_arrive(r_free);
+                mbar_arrive(&r_free[wg]);
 #pragma unroll
                 for (int c = 0; c < 64; c += 4) {
                     const float4 d4 = *reinterpret_cast<const float4*>(st + 128 + c);
@@ -374,18 +393,17 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     pf[c + 2] *= __uint_as_float(sv[c >> 5][(c + 2) & 31]) - d4.z;
                     pf[c + 3] *= __uint_as_float(sv[c >> 5][(c + 3) & 31]) - d4.w;
                 }
-                ok = __all_sync(0xffffffffu, mbar_wait(dv_done, g & 1, abort_p));    // P^T is no longer being read
-                if (!ok) break;
-                tc_fence_after();
                 {
+                    // dS^T has columns of its own: the dK MMAs of the previous step, which read them, were issued before
+                    // the dP^T MMAs whose completion this thread has just observed
                     uint32_t pk[32];
 #pragma unroll
                     for (int c = 0; c < 32; ++c) pk[c] = pack_bf16x2(pf[2 * c], pf[2 * c + 1]);
-                    tmem_st32(tP, pk);
+                    tmem_st32(tDS, pk);
                 }
                 tc_wait_st();
                 tc_fence_before();
-                mbar_arrive(ds_full);
+                mbar_arrive(&ds_full[wg]);
             }
             if (!ok) break;
             // ---------------------------------------------------------------- dK, dV of this key tile
