@@ -12,8 +12,8 @@
 //   P^T and dS^T, written back to TMEM as bf16, are directly the A operands of dV += P^T dout and dK += dS^T Q, whose
 //   B operands are the dout / Q tiles already in shared memory (read MN-major).  dK and dV stay in TMEM for the whole
 //   key tile and are written once.  Each 128-query tile is worked on as two independent chains of 64 queries, one per
-//   warpgroup (thread = key row): S^T_x -> P^T_x, then dP^T_x over the same TMEM columns -> dS^T_x; while one chain does
-//   its elementwise work the tensor pipe serves the other.
+//   warpgroup (thread = key row): [S^T_x | dP^T_x] by the tensor pipe, then P^T_x and dS^T_x written over them in
+//   place, then the two accumulating MMAs; while one chain does its elementwise work the tensor pipe serves the other.
 //
 // bwd_dq_tc_kernel     The forward's structure: a CTA owns 256 query rows (two Q tiles, one warpgroup each, one
 //   thread per row) and streams 128-key tiles; per tile S = Q K^T -> p (kept in registers), then dP = dout V^T into
@@ -89,20 +89,20 @@ bwd_prep_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __re
 // ------------------------------------------------------------------------------------------ dK / dV
 template <int D>
 struct ACfg {
-    static constexpr int kTileBytes = kQTile * D * 2;          // one 128-row tile of Q, K, V or dout
+    static constexpr int kTileBytes = kQTile * D * 2;          // one 128-row tile (K or V)
+    static constexpr int kHalfBytes = 64 * D * 2;              // one 64-row tile (Q or dout of a chain step)
     static constexpr int kBoxes = D / 64;
-    // shared memory: K,V of two key tiles (current and prefetched), two Q tiles, one dout tile,
-    // per Q slot 128 lse2 + 128 delta
+    static constexpr int kSlots = D == 128 ? 5 : 8;            // ring of chain steps: Q (64 rows), dout (64 rows), 64 lse2 + 64 delta
+    static constexpr int kSlotBytes = 2 * kHalfBytes;
     static constexpr int kOffKV = 0;
-    static constexpr int kOffQ = 4 * kTileBytes;
-    static constexpr int kOffDO = 6 * kTileBytes;
-    static constexpr int kOffStats = 7 * kTileBytes;
-    static constexpr int kOffBars = kOffStats + 2 * 256 * 4;
-    static constexpr int kNumBars = 22;
+    static constexpr int kOffRing = 2 * kTileBytes;
+    static constexpr int kOffStats = kOffRing + kSlots * kSlotBytes;
+    static constexpr int kOffBars = kOffStats + kSlots * 512;
+    static constexpr int kNumBars = 8 + 2 * kSlots;
     static constexpr int kSmemBytes = kOffBars + kNumBars * 8 + 16;
-    // TMEM columns: dK, dV (D each); per chain x (64 queries of the tile): R_x = S^T then dP^T (64 fp32 columns),
-    // P^T_x and dS^T_x as bf16 (32 columns each)
-    static constexpr uint32_t kColDK = 0, kColDV = D, kColR = 2 * D, kColP = 2 * D + 128, kColDS = 2 * D + 192;
+    // TMEM columns: dK, dV (D each); per chain x (64 queries of the tile) 128 columns: S^T_x (64 fp32) and dP^T_x
+    // (64 fp32); P^T_x and dS^T_x (bf16, 32 columns each) are written over the first half of S^T_x and dP^T_x
+    static constexpr uint32_t kColDK = 0, kColDV = D, kColR = 2 * D;
     static constexpr int kThreads = 32 * 10;
 };
 
@@ -119,24 +119,18 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do, const BwdParams p) {
     using C = ACfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
-    uint8_t* sKV = smem + C::kOffKV;          // [buffer][K,V]
-    uint8_t* sQ = smem + C::kOffQ;            // [2]
-    uint8_t* sDO = smem + C::kOffDO;
-    float* sStats = reinterpret_cast<float*>(smem + C::kOffStats);   // [2][lse2 128 | delta 128]
+    uint8_t* sKV = smem + C::kOffKV;          // K, V
+    uint8_t* sRing = smem + C::kOffRing;      // [kSlots][Q 64 rows | dout 64 rows]
+    float* sStats = reinterpret_cast<float*>(smem + C::kOffStats);   // [kSlots][lse2 64 | delta 64]
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kOffBars);
-    uint64_t* kv_full = bars + 0;     // [2]
-    uint64_t* kv_empty = bars + 2;    // [2]
-    uint64_t* q_full = bars + 4;      // [2]
-    uint64_t* q_empty = bars + 6;     // [2]
-    uint64_t* do_full = bars + 8;
-    uint64_t* do_empty = bars + 9;
-    uint64_t* s_full = bars + 10;     // [2] S^T of chain x is in R_x
-    uint64_t* p_full = bars + 12;     // [2] the chain's threads have read S^T and stored P^T
-    uint64_t* dp_full = bars + 14;    // [2] dP^T is in R_x
-    uint64_t* r_free = bars + 16;     // [2] the chain's threads have read dP^T
-    uint64_t* ds_full = bars + 18;    // [2] the chain's threads have stored dS^T
-    uint64_t* acc_full = bars + 20;   // dK, dV of the key tile are complete
-    uint64_t* acc_empty = bars + 21;  // all threads have read them
+    uint64_t* kv_full = bars + 0;
+    uint64_t* kv_empty = bars + 1;
+    uint64_t* sdp_full = bars + 2;    // [2] S^T_x and dP^T_x of a step are in TMEM
+    uint64_t* pds_full = bars + 4;    // [2] the chain's threads have stored P^T_x and dS^T_x
+    uint64_t* acc_full = bars + 6;    // dK, dV of the key tile are complete
+    uint64_t* acc_empty = bars + 7;   // all threads have read them
+    uint64_t* slot_full = bars + 8;   // [kSlots]
+    uint64_t* slot_empty = slot_full + C::kSlots;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::kNumBars);
     int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
 
@@ -145,20 +139,15 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
     if (threadIdx.x == 0) {
         *abort_flag = base_ok ? 0 : 1;
+        mbar_init(kv_full, 1);
+        mbar_init(kv_empty, 1);
         for (int i = 0; i < 2; ++i) {
-            mbar_init(&kv_full[i], 1);
-            mbar_init(&kv_empty[i], 1);
-            mbar_init(&q_full[i], 1);
-            mbar_init(&q_empty[i], 1);
+            mbar_init(&sdp_full[i], 1);
+            mbar_init(&pds_full[i], 128);
         }
-        mbar_init(do_full, 1);
-        mbar_init(do_empty, 1);
-        for (int x = 0; x < 2; ++x) {
-            mbar_init(&s_full[x], 1);
-            mbar_init(&p_full[x], 128);
-            mbar_init(&dp_full[x], 1);
-            mbar_init(&r_free[x], 128);
-            mbar_init(&ds_full[x], 128);
+        for (int i = 0; i < C::kSlots; ++i) {
+            mbar_init(&slot_full[i], 1);
+            mbar_init(&slot_empty[i], 1);
         }
         mbar_init(acc_full, 1);
         mbar_init(acc_empty, 256);
@@ -187,48 +176,46 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             bool ok = base_ok;
-            uint32_t g = 0, n_kv = 0;          // steps issued, key tiles issued
-            auto load_kv = [&](long long u) {
-                const uint32_t b = n_kv & 1;
-                ok = mbar_wait(&kv_empty[b], ((n_kv >> 1) & 1) ^ 1, abort_p);
-                if (!ok) return;
+            uint32_t hh = 0, n = 0;         // chain steps (64 queries each) issued, key tiles issued
+            for (long long u = u_begin; u < u_end && ok; ++u, ++n) {
                 const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
-                mbar_arrive_expect_tx(&kv_full[b], 2 * C::kTileBytes);
+                ok = mbar_wait(kv_empty, (n & 1) ^ 1, abort_p);
+                if (!ok) break;
+                mbar_arrive_expect_tx(kv_full, 2 * C::kTileBytes);
                 for (int x = 0; x < C::kBoxes; ++x) {
-                    tma_load_3d(sKV + (b * 2 + 0) * C::kTileBytes + x * (kQTile * 128), &map_k, &kv_full[b], x * 64, t * kTileN, bh);
-                    tma_load_3d(sKV + (b * 2 + 1) * C::kTileBytes + x * (kQTile * 128), &map_v, &kv_full[b], x * 64, t * kTileN, bh);
+                    tma_load_3d(sKV + x * (kQTile * 128), &map_k, kv_full, x * 64, t * kTileN, bh);
+                    tma_load_3d(sKV + C::kTileBytes + x * (kQTile * 128), &map_v, kv_full, x * 64, t * kTileN, bh);
                 }
-                ++n_kv;
-            };
-            if (ok && u_begin < u_end) load_kv(u_begin);
-            for (long long u = u_begin; u < u_end && ok; ++u) {
-                const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
-                const int i_first = first_q_tile(p, t);
-                for (int i = i_first; i < p.q_tiles128 && ok; ++i, ++g) {
-                    const uint32_t qs = g & 1;
-                    ok = mbar_wait(&q_empty[qs], ((g >> 1) & 1) ^ 1, abort_p);
+                if (u + 1 < u_end) {        // K, V have one buffer: the next tile's rows come as far as L2 meanwhile
+                    const int bh_n = (int)((u + 1) / p.key_tiles), t_n = (int)(u + 1 - (long long)bh_n * p.key_tiles);
+                    for (int x = 0; x < C::kBoxes; ++x) {
+                        tma_prefetch_l2_3d(&map_k, x * 64, t_n * kTileN, bh_n);
+                        tma_prefetch_l2_3d(&map_v, x * 64, t_n * kTileN, bh_n);
+                    }
+                }
+                const int row_first = first_q_tile(p, t) * kQTile, row_end = p.q_tiles128 * kQTile;
+                for (int row = row_first; row < row_end && ok; row += 64, ++hh) {
+                    const uint32_t slot = hh % C::kSlots, round = hh / C::kSlots;
+                    ok = mbar_wait(&slot_empty[slot], (round & 1) ^ 1, abort_p);
                     if (!ok) break;
-                    mbar_arrive_expect_tx(&q_full[qs], C::kTileBytes + 1024);
-                    for (int x = 0; x < C::kBoxes; ++x)
-                        tma_load_3d(sQ + qs * C::kTileBytes + x * (kQTile * 128), &map_q, &q_full[qs], x * 64, i * kQTile, bh);
-                    bulk_load_1d(sStats + qs * 256, p.lse2 + (long long)bh * p.Wpad + i * kQTile, 512, &q_full[qs]);
-                    bulk_load_1d(sStats + qs * 256 + 128, p.delta + (long long)bh * p.Wpad + i * kQTile, 512, &q_full[qs]);
-                    ok = mbar_wait(do_empty, (g & 1) ^ 1, abort_p);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(do_full, C::kTileBytes);
-                    for (int x = 0; x < C::kBoxes; ++x)
-                        tma_load_3d(sDO + x * (kQTile * 128), &map_do, do_full, x * 64, i * kQTile, bh);
-                    if (i == i_first && u + 1 < u_end) load_kv(u + 1);     // next key tile's K, V arrive during this one
+                    uint8_t* dst = sRing + slot * C::kSlotBytes;
+                    mbar_arrive_expect_tx(&slot_full[slot], C::kSlotBytes + 512);
+                    for (int x = 0; x < C::kBoxes; ++x) {
+                        tma_load_3d(dst + x * (64 * 128), &map_q, &slot_full[slot], x * 64, row, bh);
+                        tma_load_3d(dst + C::kHalfBytes + x * (64 * 128), &map_do, &slot_full[slot], x * 64, row, bh);
+                    }
+                    bulk_load_1d(sStats + slot * 128, p.lse2 + (long long)bh * p.Wpad + row, 256, &slot_full[slot]);
+                    bulk_load_1d(sStats + slot * 128 + 64, p.delta + (long long)bh * p.Wpad + row, 256, &slot_full[slot]);
                 }
             }
             if (!ok && base_ok) {
                 // leave no copy in flight: the barriers armed last must complete (bounded)
                 int dummy = 0;
-                if (n_kv > 0) mbar_wait(&kv_full[(n_kv - 1) & 1], ((n_kv - 1) >> 1) & 1, &dummy, 200000000LL);
-                if (n_kv > 1) mbar_wait(&kv_full[(n_kv - 2) & 1], ((n_kv - 2) >> 1) & 1, &dummy, 200000000LL);
-                // q_full / do_full of step g may or may not have been armed; the steps before it were
-                if (g > 0) mbar_wait(&q_full[(g - 1) & 1], ((g - 1) >> 1) & 1, &dummy, 200000000LL);
-                if (g > 0) mbar_wait(do_full, (g - 1) & 1, &dummy, 200000000LL);
+                if (n > 0) mbar_wait(kv_full, (n - 1) & 1, &dummy, 200000000LL);
+                for (uint32_t back = 1; back <= (uint32_t)C::kSlots && back <= hh; ++back) {
+                    const uint32_t id = hh - back;
+                    mbar_wait(&slot_full[id % C::kSlots], (id / C::kSlots) & 1, &dummy, 200000000LL);
+                }
             }
         }
     } else if (warp == kMmaWarp) {
@@ -236,174 +223,144 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const uint32_t idesc_st = make_idesc_bf16(kQTile, 64, 0, 0);         // S^T, dP^T of a chain: M = keys, N = 64 queries
         const uint32_t idesc_acc = make_idesc_bf16(kQTile, D, 0, 1);         // dV, dK: A in TMEM, B MN-major
         const uint64_t kmaj = make_smem_desc_sw128(smem_u32(smem), 16, 1024);
-        const uint64_t mnmaj = make_smem_desc_sw128(smem_u32(smem), kQTile * 128, 1024);
+        const uint64_t mnmaj = make_smem_desc_sw128(smem_u32(smem), 64 * 128, 1024);   // 64-row tiles: 8 KB between column blocks
         const uint32_t desc_hi = (uint32_t)(kmaj >> 32);
         const uint32_t kmaj_lo = (uint32_t)kmaj, mnmaj_lo = (uint32_t)mnmaj;
         const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
         const uint32_t tDK = tmem_u + C::kColDK, tDV = tmem_u + C::kColDV;
-        auto tile_off = [&](int byte_off) { return (uint32_t)(byte_off >> 4); };
-        // R_x = A B_x^T: A a whole K-major tile (K or V), B_x rows [64x, 64x+64) of a K-major tile (Q or dout)
-        auto issue_st = [&](int x, uint32_t a_off, uint32_t b_off) {
-            const uint32_t d = tmem_u + C::kColR + x * 64, b_rows = (uint32_t)(x * 64 * 128) >> 4;
+        const uint32_t k_off = (uint32_t)(C::kOffKV >> 4), v_off = (uint32_t)((C::kOffKV + C::kTileBytes) >> 4);
+        // [S^T_x | dP^T_x] = [K Q_x^T | V dout_x^T]: A a 128-row K-major tile, B the 64-row K-major tile of the slot
+        auto issue_sdp = [&](int x, uint32_t slot) {
+            const uint32_t q_off = (uint32_t)((C::kOffRing + slot * C::kSlotBytes) >> 4), do_off = q_off + (uint32_t)(C::kHalfBytes >> 4);
+            const uint32_t d = tmem_u + C::kColR + x * 128;
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
-                const uint32_t off16 = ((kk >> 2) * (kQTile * 128) + (kk & 3) * 32) >> 4;
-                if (elect_one()) mma_ss_parts(d, kmaj_lo + a_off + off16, kmaj_lo + b_off + b_rows + off16, desc_hi, idesc_st, kk > 0);
+                const uint32_t a16 = ((kk >> 2) * (kQTile * 128) + (kk & 3) * 32) >> 4, b16 = ((kk >> 2) * (64 * 128) + (kk & 3) * 32) >> 4;
+                if (elect_one()) mma_ss_parts(d, kmaj_lo + k_off + a16, kmaj_lo + q_off + b16, desc_hi, idesc_st, kk > 0);
             }
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t a16 = ((kk >> 2) * (kQTile * 128) + (kk & 3) * 32) >> 4, b16 = ((kk >> 2) * (64 * 128) + (kk & 3) * 32) >> 4;
+                if (elect_one()) mma_ss_parts(d + 64, kmaj_lo + v_off + a16, kmaj_lo + do_off + b16, desc_hi, idesc_st, kk > 0);
+            }
+            commit_elected(&sdp_full[x]);
         };
-        // D += A_x B_x: A_x = P^T or dS^T of the chain (TMEM, 64 queries), B_x rows [64x, 64x+64) of an MN-major tile
-        auto issue_acc = [&](int x, uint32_t d_tmem, uint32_t a_col, uint32_t b_off, bool accumulate) {
-            const uint32_t a = tmem_u + a_col + x * 32;
+        // dV += P^T_x dout_x, dK += dS^T_x Q_x: A in TMEM (64 queries = 32 columns), B the slot's 64-row tile read MN-major
+        auto issue_acc = [&](int x, uint32_t slot, bool accumulate) {
+            const uint32_t q_off = (uint32_t)((C::kOffRing + slot * C::kSlotBytes) >> 4), do_off = q_off + (uint32_t)(C::kHalfBytes >> 4);
+            const uint32_t a = tmem_u + C::kColR + x * 128;
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-                if (elect_one()) mma_ts_parts(d_tmem, a + kk * 8, mnmaj_lo + b_off + (x * 4 + kk) * (2048 >> 4), desc_hi, idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+                if (elect_one()) mma_ts_parts(tDV, a + kk * 8, mnmaj_lo + do_off + kk * (2048 >> 4), desc_hi, idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                if (elect_one()) mma_ts_parts(tDK, a + 64 + kk * 8, mnmaj_lo + q_off + kk * (2048 >> 4), desc_hi, idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+            commit_elected(&slot_empty[slot]);
         };
         bool ok = base_ok;
-        uint32_t g = 0, n = 0;
-        for (long long u = u_begin; u < u_end && ok; ++u, ++n) {
-            const uint32_t b = n & 1;
-            const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
+        uint32_t g = 0, n = 0;              // 128-query steps done, key tiles done; chain x of step g uses ring entry 2g + x
+        int t = (int)(u_begin % p.key_tiles);
+        for (long long u = u_begin; u < u_end && ok; ++u, ++n, t = t + 1 == p.key_tiles ? 0 : t + 1) {
             const int steps = p.q_tiles128 - first_q_tile(p, t);
-            const uint32_t k_off = tile_off(C::kOffKV + (b * 2 + 0) * C::kTileBytes), v_off = tile_off(C::kOffKV + (b * 2 + 1) * C::kTileBytes);
-            const uint32_t do_off = tile_off(C::kOffDO);
-            ok = __all_sync(0xffffffffu, mbar_wait(&kv_full[b], (n >> 1) & 1, abort_p));
+            ok = __all_sync(0xffffffffu, mbar_wait(kv_full, n & 1, abort_p));
             if (!ok) break;
-            ok = __all_sync(0xffffffffu, mbar_wait(&q_full[g & 1], (g >> 1) & 1, abort_p));
-            if (!ok) break;
-            tc_fence_after();
-            for (int x = 0; x < 2; ++x) {
-                issue_st(x, k_off, tile_off(C::kOffQ + (g & 1) * C::kTileBytes));
-                commit_elected(&s_full[x]);
+            for (int x = 0; x < 2 && ok; ++x) {
+                const uint32_t hh = 2 * g + x;
+                ok = __all_sync(0xffffffffu, mbar_wait(&slot_full[hh % C::kSlots], (hh / C::kSlots) & 1, abort_p));
+                if (!ok) break;
+                issue_sdp(x, hh % C::kSlots);
             }
+            if (!ok) break;
+            if (steps == 1) commit_elected(kv_empty);       // K, V have been read for the last time: the next tile's may load
             for (int s = 0; s < steps && ok; ++s, ++g) {
-                const uint32_t q_off = tile_off(C::kOffQ + (g & 1) * C::kTileBytes);
-                for (int x = 0; x < 2 && ok; ++x) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(&p_full[x], g & 1, abort_p));
-                    if (!ok) break;
-                    if (x == 0) {
-                        ok = __all_sync(0xffffffffu, mbar_wait(do_full, g & 1, abort_p));
-                        if (!ok) break;
-                        if (s == 0 && n > 0) {      // the previous key tile's dK, dV must have been read out
-                            ok = __all_sync(0xffffffffu, mbar_wait(acc_empty, (n - 1) & 1, abort_p));
-                            if (!ok) break;
-                        }
-                    }
-                    tc_fence_after();
-                    issue_st(x, v_off, do_off);                 // dP^T over S^T: the chain's threads have read S^T (p_full)
-                    commit_elected(&dp_full[x]);
-                    issue_acc(x, tDV, C::kColP, do_off, s > 0 || x > 0);
-                }
-                if (!ok) break;
-                commit_elected(do_empty);
                 const bool have_next = s + 1 < steps;
-                if (have_next) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(&q_full[(g + 1) & 1], ((g + 1) >> 1) & 1, abort_p));
-                    if (!ok) break;
-                }
                 for (int x = 0; x < 2 && ok; ++x) {
-                    if (have_next) {                            // next step's S^T as soon as dP^T has been read
-                        ok = __all_sync(0xffffffffu, mbar_wait(&r_free[x], g & 1, abort_p));
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_st(x, k_off, tile_off(C::kOffQ + ((g + 1) & 1) * C::kTileBytes));
-                        commit_elected(&s_full[x]);
-                    }
-                    ok = __all_sync(0xffffffffu, mbar_wait(&ds_full[x], g & 1, abort_p));
+                    const uint32_t hh = 2 * g + x;
+                    ok = __all_sync(0xffffffffu, mbar_wait(&pds_full[x], g & 1, abort_p));
                     if (!ok) break;
+                    if (s == 0 && x == 0 && n > 0) {        // the previous key tile's dK, dV must have been read out
+                        ok = __all_sync(0xffffffffu, mbar_wait(acc_empty, (n - 1) & 1, abort_p));
+                        if (!ok) break;
+                    }
                     tc_fence_after();
-                    issue_acc(x, tDK, C::kColDS, q_off, s > 0 || x > 0);
+                    issue_acc(x, hh % C::kSlots, s > 0 || x > 0);
+                    if (have_next) {
+                        const uint32_t hn = hh + 2;
+                        ok = __all_sync(0xffffffffu, mbar_wait(&slot_full[hn % C::kSlots], (hn / C::kSlots) & 1, abort_p));
+                        if (!ok) break;
+                        issue_sdp(x, hn % C::kSlots);
+                    }
                 }
                 if (!ok) break;
-                commit_elected(&q_empty[g & 1]);
+                if (have_next && s + 2 == steps) commit_elected(kv_empty);
             }
             if (!ok) break;
             commit_elected(acc_full);
-            commit_elected(&kv_empty[b]);
         }
     } else {
         // ------------------------------------------------------------------ elementwise threads
         const int wg = warp >> 2;                              // chain: which 64 queries of every tile
         const int r = (warp & 3) * 32 + lane;                  // key row inside the tile == TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tR = tmem_base + lane_addr + C::kColR + wg * 64;
-        const uint32_t tP = tmem_base + lane_addr + C::kColP + wg * 32;
-        const uint32_t tDS = tmem_base + lane_addr + C::kColDS + wg * 32;
+        const uint32_t tS = tmem_base + lane_addr + C::kColR + wg * 128;
+        const uint32_t tDP = tS + 64;
         bool ok = base_ok;
         uint32_t g = 0, n = 0;
-        for (long long u = u_begin; u < u_end && ok; ++u, ++n) {
-            const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
+        int bh = (int)(u_begin / p.key_tiles), t = (int)(u_begin - (long long)bh * p.key_tiles);
+        for (long long u = u_begin; u < u_end && ok; ++u, ++n, ++t) {
+            if (t == p.key_tiles) {
+                t = 0;
+                ++bh;
+            }
             const int key = t * kTileN + r;
             const int i_first = first_q_tile(p, t);
             const long long shift = (long long)p.N - p.W;       // query q may use key k iff q >= k - shift
             const int q_min = p.causal ? (int)((long long)key - shift) : -0x7fffffff;
             const int q_min_warp = p.causal ? (int)((long long)key - lane + 31 - shift) : -0x7fffffff;   // largest in the warp
             for (int i = i_first; i < p.q_tiles128; ++i, ++g) {
-                const float* st = sStats + (g & 1) * 256 + wg * 64;
+                const uint32_t hh = 2 * g + wg, slot = hh % C::kSlots;
+                const float* st = sStats + slot * 128;
                 const int q0 = i * kQTile + wg * 64;              // first query of this thread's columns
-                ok = __all_sync(0xffffffffu, mbar_wait(&s_full[wg], g & 1, abort_p));
+                ok = __all_sync(0xffffffffu, mbar_wait(&sdp_full[wg], g & 1, abort_p));
                 if (!ok) break;
-                // already complete (the S^T MMAs waited for it); observing it here orders the bulk-copied lse2 / delta
+                // already complete (the MMAs waited for it); observing it here orders the bulk-copied lse2 / delta
                 // before this thread's reads
-                ok = __all_sync(0xffffffffu, mbar_wait(&q_full[g & 1], (g >> 1) & 1, abort_p));
+                ok = __all_sync(0xffffffffu, mbar_wait(&slot_full[slot], (hh / C::kSlots) & 1, abort_p));
                 if (!ok) break;
                 tc_fence_after();
-                uint32_t sv[2][32];
-                tmem_ld32_async(tR, sv[0]);
-                tmem_ld32_async(tR + 32, sv[1]);
-                tmem_wait_ld(sv[0]);
-                tmem_wait_ld(sv[1]);
                 const bool masked = q0 < q_min_warp;              // warp-uniform: some element of some lane is masked
-                float pf[64];
 #pragma unroll
-                for (int c = 0; c < 64; c += 4) {
-                    const float4 l4 = *reinterpret_cast<const float4*>(st + c);
-                    pf[c + 0] = ex2(fmaf(__uint_as_float(sv[c >> 5][(c + 0) & 31]), p.scale_log2e, -l4.x));
-                    pf[c + 1] = ex2(fmaf(__uint_as_float(sv[c >> 5][(c + 1) & 31]), p.scale_log2e, -l4.y));
-                    pf[c + 2] = ex2(fmaf(__uint_as_float(sv[c >> 5][(c + 2) & 31]), p.scale_log2e, -l4.z));
-                    pf[c + 3] = ex2(fmaf(__uint_as_float(sv[c >> 5][(c + 3) & 31]), p.scale_log2e, -l4.w));
-                }
-                if (masked) {
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t sv[32], dv_[32];
+                    tmem_ld32_async(tS + h * 32, sv);
+                    tmem_ld32_async(tDP + h * 32, dv_);
+                    tmem_wait_ld(sv);
+                    tmem_wait_ld(dv_);
+                    uint32_t pk[16], dk_[16];
 #pragma unroll
-                    for (int c = 0; c < 64; ++c)
-                        if (q0 + c < q_min) pf[c] = 0.f;
-                }
-                {
-                    uint32_t pk[32];
+                    for (int c = 0; c < 32; c += 4) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(st + h * 32 + c);
+                        const float4 d4 = *reinterpret_cast<const float4*>(st + 64 + h * 32 + c);
+                        const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dlv[4] = {d4.x, d4.y, d4.z, d4.w};
+                        float pe[4], de[4];
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) pk[c] = pack_bf16x2(pf[2 * c], pf[2 * c + 1]);
-                    tmem_st32(tP, pk);
-                }
-                tc_wait_st();
-                tc_fence_before();
-                mbar_arrive(&p_full[wg]);
-                ok = __all_sync(0xffffffffu, mbar_wait(&dp_full[wg], g & 1, abort_p));
-                if (!ok) break;
-                tc_fence_after();
-                tmem_ld32_async(tR, sv[0]);
-                tmem_ld32_async(tR + 32, sv[1]);
-                tmem_wait_ld(sv[0]);
-                tmem_wait_ld(sv[1]);
-                tc_fence_before();
-                mbar_arrive(&r_free[wg]);
-#pragma unroll
-                for (int c = 0; c < 64; c += 4) {
-                    const float4 d4 = *reinterpret_cast<const float4*>(st + 128 + c);
-                    pf[c + 0] *= __uint_as_float(sv[c >> 5][(c + 0) & 31]) - d4.x;
-                    pf[c + 1] *= __uint_as_float(sv[c >> 5][(c + 1) & 31]) - d4.y;
-                    pf[c + 2] *= __uint_as_float(sv[c >> 5][(c + 2) & 31]) - d4.z;
-                    pf[c + 3] *= __uint_as_float(sv[c >> 5][(c + 3) & 31]) - d4.w;
-                }
-                {
-                    // dS^T has columns of its own: the dK MMAs of the previous step, which read them, were issued before
-                    // the dP^T MMAs whose completion this thread has just observed
-                    uint32_t pk[32];
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) pk[c] = pack_bf16x2(pf[2 * c], pf[2 * c + 1]);
-                    tmem_st32(tDS, pk);
+                        for (int e = 0; e < 4; ++e) {
+                            pe[e] = ex2(fmaf(__uint_as_float(sv[c + e]), p.scale_log2e, -lv[e]));
+                            if (masked && q0 + h * 32 + c + e < q_min) pe[e] = 0.f;
+                            de[e] = pe[e] * (__uint_as_float(dv_[c + e]) - dlv[e]);
+                        }
+                        pk[c / 2] = pack_bf16x2(pe[0], pe[1]);
+                        pk[c / 2 + 1] = pack_bf16x2(pe[2], pe[3]);
+                        dk_[c / 2] = pack_bf16x2(de[0], de[1]);
+                        dk_[c / 2 + 1] = pack_bf16x2(de[2], de[3]);
+                    }
+                    // bf16 P^T over columns of S^T, dS^T over columns of dP^T, that are already in registers
+                    tmem_st16(tS + h * 16, pk);
+                    tmem_st16(tDP + h * 16, dk_);
                 }
                 tc_wait_st();
                 tc_fence_before();
-                mbar_arrive(&ds_full[wg]);
+                mbar_arrive(&pds_full[wg]);
             }
             if (!ok) break;
             // ---------------------------------------------------------------- dK, dV of this key tile
@@ -859,11 +816,13 @@ int launch_d(const void* q, const void* k, const void* v, const void* out, const
              float* ws, int num_sms, cudaStream_t st) {
     const long long bh = (long long)B * H;
     const int Wpad = (W + kQTile - 1) / kQTile * kQTile;
-    CUtensorMap mq, mk, mv, mdo;
+    CUtensorMap mq, mk, mv, mdo, mq64, mdo64;
     int rc = make_map(&mq, q, D, W, bh);
     if (rc == TLIN_OK) rc = make_map(&mk, k, D, N, bh);
     if (rc == TLIN_OK) rc = make_map(&mv, v, D, N, bh);
     if (rc == TLIN_OK) rc = make_map(&mdo, dout, D, W, bh);
+    if (rc == TLIN_OK) rc = make_map(&mq64, q, D, W, bh, 64);
+    if (rc == TLIN_OK) rc = make_map(&mdo64, dout, D, W, bh, 64);
     if (rc != TLIN_OK) return rc;
     BwdParams p;
     float* lse2 = ws;
@@ -894,7 +853,7 @@ int launch_d(const void* q, const void* k, const void* v, const void* out, const
     pa.total_units = bh * p.key_tiles;
     pa.n_groups = 0; pa.q_tiles = 0; pa.schedule = 0;
     const long long ctas_a = pa.total_units < num_sms ? pa.total_units : num_sms;
-    bwd_dkdv_tc_kernel<D><<<(unsigned)ctas_a, ACfg<D>::kThreads, ACfg<D>::kSmemBytes, st>>>(mq, mk, mv, mdo, pa);
+    bwd_dkdv_tc_kernel<D><<<(unsigned)ctas_a, ACfg<D>::kThreads, ACfg<D>::kSmemBytes, st>>>(mq64, mk, mv, mdo64, pa);
     TLIN_CUDA_CHECK(cudaGetLastError());
     // dQ: the forward's plan
     BwdParams pb = p;

@@ -86,13 +86,13 @@ inline EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// [BH, rows, D] bf16, box = 64 elements x 128 rows x 1, 128-byte swizzle, zero fill outside.
-inline int make_map(CUtensorMap* m, const void* ptr, int D, long long rows, long long bh) {
+// [BH, rows, D] bf16, box = 64 elements x box_rows rows x 1, 128-byte swizzle, zero fill outside.
+inline int make_map(CUtensorMap* m, const void* ptr, int D, long long rows, long long bh, int box_rows = kQTile) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return TLIN_ERR_CUDA;
     cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)bh};
     cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)rows * D * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)kQTile, 1};
+    cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     cuuint32_t es[3] = {1, 1, 1};
     const CUresult rc = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
