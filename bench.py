@@ -34,7 +34,9 @@ import torch  # noqa: E402
 from paper_2508_20407_b200 import synth  # noqa: E402
 
 WORKLOADS = {"fwd128k": "cfg4_vlong", "fwd32k": "cfg3_long", "fwd8k": "cfg2_mid", "decode": "cfg5_decode",
-             "restore": "restore_vlong", "inner_self": "inner_self", "inner_gen": "inner_gen"}
+             "restore": "restore_vlong", "inner_self": "inner_self", "inner_gen": "inner_gen",
+             "bwd_chunk": "train_chunk", "bwd32k": "cfg3_long"}
+BACKWARD = ("bwd_chunk", "bwd32k")      # legs that time tlin_attn_backward on the named shape
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -313,6 +315,43 @@ def run_forward(wl, args, rank, world, device, peaks, with_cpu):
     return res
 
 
+def run_backward(wl, args, rank, world, device, peaks):
+    """Backward pass alone (out and lse come from one untimed forward).  FLOPs counted: the five matrix products of the
+    chain rule (2.5 x the forward); the two kernels execute seven (both recompute the scores)."""
+    from paper_2508_20407_b200 import binding as tl
+    q, k, v = synth.forward_inputs(wl, device=device)
+    g = torch.Generator(device="cpu").manual_seed(wl.seed + 99)
+    dout = torch.randn(q.shape, generator=g, dtype=torch.float32).to(torch.bfloat16).to(device)
+    out, lse = tl.tlin_attn_forward(q, k, v, causal_window=wl.causal_window)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    tl.ensure_workspace(tl.workspace_bytes_backward(wl.B, wl.H, wl.N, wl.W, wl.d), device)
+    launches = []
+
+    def step(_):
+        tl.tlin_attn_backward(q, k, v, out, lse, dout, dq, dk, dv, wl.causal_window)
+        launches.append(tl.tlin_last_launch_count())
+
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    nbytes = 2 * (4 * wl.B * wl.H * wl.N * wl.d + 4 * wl.B * wl.H * wl.W * wl.d)      # q,k,v,out,dout in; dq,dk,dv out
+    flush = torch.empty(int(2.5 * L2_BYTES), dtype=torch.uint8, device=device) if nbytes < 2 * L2_BYTES else None
+    ms, clocks = time_steps(step, args.steps, args.warmup, world, device, sampler, flush)
+    ms_step = ms / args.steps
+    flop = 10.0 * wl.B * wl.H * wl.W * wl.N * wl.d
+    tflops = flop / (ms_step * 1e-3) / 1e12
+    roof = dict(bound="tensor", achieved=tflops, peak=peaks["bf16_tflops"], unit="TFLOP/s", frac=tflops / peaks["bf16_tflops"],
+                traffic=None, algorithmic_bytes=nbytes, peak_source=peaks["source"] + " (burst)",
+                kernel="backward (row statistics, dK/dV kernel, dQ kernel, dQ partial sums)",
+                executed_over_counted_flops=1.4, roofline_ms=flop / (peaks["bf16_tflops"] * 1e12) * 1e3)
+    if "bf16_tflops_sustained" in peaks:
+        roof["frac_of_sustained_peak"] = tflops / peaks["bf16_tflops_sustained"]
+    l2_note = ("inputs+outputs %.0f MB > 2 x L2 (126 MB): back-to-back calls, no flush" % (nbytes / 1e6) if flush is None else
+               "inputs+outputs %.0f MB: a %.0f MB buffer is overwritten before every timed call (L2 flush), calls timed one by one"
+               % (nbytes / 1e6, flush.numel() / 1e6))
+    return dict(workload=wl.name + " backward", shape=dict(B=wl.B, H=wl.H, N=wl.N, W=wl.W, d=wl.d, causal_window=wl.causal_window),
+                l2=l2_note, ms_per_step=ms_step, tflops=tflops, roofline=roof, e2e=None, clocks=clocks,
+                gpu_launches=int(sum(launches[args.warmup:])), launches_per_step=launches[-1] if launches else 0)
+
+
 def run_decode(wl, args, rank, world, device, peaks, with_cpu):
     from paper_2508_20407_b200 import binding as tl
     (kc, vc), (qn, kn, vn) = synth.decode_inputs(wl, device=device)
@@ -460,11 +499,14 @@ def main():
         wl = synth.Workload("custom_" + args.shape.replace(",", "_"), v[0], v[1], v[4], v[2], v[3], seed=9,
                             causal_window=v[5] if len(v) > 5 else 1, decode=args.workload == "decode")
     with_cpu = (not args.no_cpu) and world == 1
-    runner = run_decode if wl.decode else run_forward
-    main_res = runner(wl, args, rank, world, device, peaks, with_cpu)
+    if args.workload in BACKWARD:
+        main_res = run_backward(wl, args, rank, world, device, peaks)
+    else:
+        runner = run_decode if wl.decode else run_forward
+        main_res = runner(wl, args, rank, world, device, peaks, with_cpu)
     also = []
     if not args.only and world == 1:
-        for name in ("fwd32k", "decode", "restore", "inner_self", "inner_gen"):
+        for name in ("fwd32k", "decode", "restore", "inner_self", "inner_gen", "bwd_chunk", "bwd32k"):
             if name == args.workload:
                 continue
             torch.cuda.empty_cache()
@@ -472,10 +514,15 @@ def main():
             w2 = synth.WORKLOADS[WORKLOADS[name]]
             a2 = argparse.Namespace(**vars(args))
             a2.no_e2e = args.no_e2e or name not in ("fwd32k", "decode")     # host-buffer legs only where they are cheap to set up
-            also.append((run_decode if w2.decode else run_forward)(w2, a2, rank, world, device, peaks, False))
+            if name in BACKWARD:
+                also.append(run_backward(w2, a2, rank, world, device, peaks))
+            else:
+                also.append((run_decode if w2.decode else run_forward)(w2, a2, rank, world, device, peaks, False))
 
     if rank == 0:
-        if wl.decode:
+        if args.workload in BACKWARD:
+            metric, unit, value = "attention_backward_TFLOP_per_s", "TFLOP/s", world * main_res["tflops"]
+        elif wl.decode:
             metric, unit, value = "decode_kv_GB_per_s", "GB/s", main_res["gb_per_s"]
         else:
             metric, unit, value = "context_tokens_per_s", "context tokens/s", main_res["tokens_per_s"]

@@ -37,6 +37,7 @@ using namespace tc;
 
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
+constexpr int kKvWarp = 10;                 // dK/dV kernel only
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct BwdParams {
@@ -103,7 +104,7 @@ struct ACfg {
     // TMEM columns: dK, dV (D each); per chain x (64 queries of the tile) 128 columns: S^T_x (64 fp32) and dP^T_x
     // (64 fp32); P^T_x and dS^T_x (bf16, 32 columns each) are written over the first half of S^T_x and dP^T_x
     static constexpr uint32_t kColDK = 0, kColDV = D, kColR = 2 * D;
-    static constexpr int kThreads = 32 * 10;
+    static constexpr int kThreads = 32 * 11;
 };
 
 // first 128-row query tile that may use a key of key tile t
@@ -173,26 +174,14 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const long long u_end = (long long)(((unsigned long long)(blockIdx.x + 1) * (unsigned long long)p.total_units) / gridDim.x);
 
     if (warp == kProducerWarp) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ TMA producer: Q / dout / row statistics ring
+        // The ring runs ahead of the key tiles: the first chain steps of the next key tile are loaded while the
+        // current one is still being worked on.
         if (lane == 0) {
             bool ok = base_ok;
-            uint32_t hh = 0, n = 0;         // chain steps (64 queries each) issued, key tiles issued
-            for (long long u = u_begin; u < u_end && ok; ++u, ++n) {
+            uint32_t hh = 0;                // chain steps (64 queries each) issued
+            for (long long u = u_begin; u < u_end && ok; ++u) {
                 const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
-                ok = mbar_wait(kv_empty, (n & 1) ^ 1, abort_p);
-                if (!ok) break;
-                mbar_arrive_expect_tx(kv_full, 2 * C::kTileBytes);
-                for (int x = 0; x < C::kBoxes; ++x) {
-                    tma_load_3d(sKV + x * (kQTile * 128), &map_k, kv_full, x * 64, t * kTileN, bh);
-                    tma_load_3d(sKV + C::kTileBytes + x * (kQTile * 128), &map_v, kv_full, x * 64, t * kTileN, bh);
-                }
-                if (u + 1 < u_end) {        // K, V have one buffer: the next tile's rows come as far as L2 meanwhile
-                    const int bh_n = (int)((u + 1) / p.key_tiles), t_n = (int)(u + 1 - (long long)bh_n * p.key_tiles);
-                    for (int x = 0; x < C::kBoxes; ++x) {
-                        tma_prefetch_l2_3d(&map_k, x * 64, t_n * kTileN, bh_n);
-                        tma_prefetch_l2_3d(&map_v, x * 64, t_n * kTileN, bh_n);
-                    }
-                }
                 const int row_first = first_q_tile(p, t) * kQTile, row_end = p.q_tiles128 * kQTile;
                 for (int row = row_first; row < row_end && ok; row += 64, ++hh) {
                     const uint32_t slot = hh % C::kSlots, round = hh / C::kSlots;
@@ -209,13 +198,38 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
             }
             if (!ok && base_ok) {
-                // leave no copy in flight: the barriers armed last must complete (bounded)
-                int dummy = 0;
-                if (n > 0) mbar_wait(kv_full, (n - 1) & 1, &dummy, 200000000LL);
+                int dummy = 0;              // leave no copy in flight: the barriers armed last must complete (bounded)
                 for (uint32_t back = 1; back <= (uint32_t)C::kSlots && back <= hh; ++back) {
                     const uint32_t id = hh - back;
                     mbar_wait(&slot_full[id % C::kSlots], (id / C::kSlots) & 1, &dummy, 200000000LL);
                 }
+            }
+        }
+    } else if (warp == kKvWarp) {
+        // ------------------------------------------------------------------ TMA producer: K, V of the key tiles
+        if (lane == 0) {
+            bool ok = base_ok;
+            uint32_t n = 0;
+            for (long long u = u_begin; u < u_end && ok; ++u, ++n) {
+                const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
+                if (u + 1 < u_end) {        // K, V have one buffer: the next tile's rows come as far as L2 meanwhile
+                    const int bh_n = (int)((u + 1) / p.key_tiles), t_n = (int)(u + 1 - (long long)bh_n * p.key_tiles);
+                    for (int x = 0; x < C::kBoxes; ++x) {
+                        tma_prefetch_l2_3d(&map_k, x * 64, t_n * kTileN, bh_n);
+                        tma_prefetch_l2_3d(&map_v, x * 64, t_n * kTileN, bh_n);
+                    }
+                }
+                ok = mbar_wait(kv_empty, (n & 1) ^ 1, abort_p);
+                if (!ok) break;
+                mbar_arrive_expect_tx(kv_full, 2 * C::kTileBytes);
+                for (int x = 0; x < C::kBoxes; ++x) {
+                    tma_load_3d(sKV + x * (kQTile * 128), &map_k, kv_full, x * 64, t * kTileN, bh);
+                    tma_load_3d(sKV + C::kTileBytes + x * (kQTile * 128), &map_v, kv_full, x * 64, t * kTileN, bh);
+                }
+            }
+            if (!ok && base_ok && n > 0) {
+                int dummy = 0;
+                mbar_wait(kv_full, (n - 1) & 1, &dummy, 200000000LL);
             }
         }
     } else if (warp == kMmaWarp) {
@@ -297,7 +311,7 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (!ok) break;
             commit_elected(acc_full);
         }
-    } else {
+    } else if (warp < 8) {
         // ------------------------------------------------------------------ elementwise threads
         const int wg = warp >> 2;                              // chain: which 64 queries of every tile
         const int r = (warp & 3) * 32 + lane;                  // key row inside the tile == TMEM lane

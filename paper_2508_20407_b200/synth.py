@@ -155,6 +155,9 @@ WORKLOADS = {
     "inner_self": _w("inner_self", 1, 32, 128, 1024, 1024, 6, causal_window=0),
     # inner generation layer: W_og window queries over [summary tokens; window], causal inside the window
     "inner_gen": _w("inner_gen", 1, 32, 128, 2048, 1024, 7, causal_window=1),
+    # --- training (forward + backward): the last of the 8 windows of a sliding-window pass (stride W_og = 1024) over
+    # sequences of 8192 tokens: W_og window queries over the whole sequence so far, causal inside the window
+    "train_chunk": _w("train_chunk", 4, 32, 128, 8192, 1024, 8, causal_window=1),
 }
 
 Q_ID, K_ID, V_ID, QNEW_ID, KNEW_ID, VNEW_ID = 0, 1, 2, 3, 4, 5
