@@ -178,3 +178,23 @@ def test_decode_plan_balances_the_benchmark_shape():
     waves = -(-p.n_ctas // 296)
     ideal = 65537 * 256 / 296
     assert waves * p.keys_per_split <= 1.05 * ideal
+
+
+def test_backward_workspace_covers_row_statistics_and_partial_sums():
+    # host arithmetic only: 2 floats per padded query row (lse*log2e, delta) plus, when the key range of a (b,h) is split
+    # between groups, two 256 x d fp32 slots per CTA of the dQ kernel; never less than the CUDA-core path's needs
+    # (one float per row + an fp32 dQ accumulator)
+    for B, H, N, W, d in [(1, 32, 131072, 1024, 128), (4, 32, 8192, 1024, 128), (4, 16, 8192, 256, 64), (1, 1, 1, 1, 64), (2, 3, 1000, 300, 128)]:
+        got = tl.workspace_bytes_backward(B, H, N, W, d)
+        rows = B * H * W
+        simt = 4 * ((rows + 3) // 4 * 4 + rows * d)
+        wpad = (W + 127) // 128 * 128
+        need = simt
+        for causal in (0, 1):
+            if causal and N < W:
+                continue
+            plan = tl.tlin_plan_forward(B, H, N, W, d, causal)
+            tc = 4 * (2 * B * H * wpad + (plan.n_ctas * 2 * 256 * d if plan.uses_workspace else 0))
+            need = max(need, tc)
+        assert got == need, (B, H, N, W, d, got, need)
+    assert tl.workspace_bytes_backward(0, 1, 1, 1, 64) == 0
