@@ -134,13 +134,19 @@ int tlin_decode_step_static(const void* q_new, const void* k_new, const void* v_
  *   q, out, dout, dq [B,H,W,d]   k, v, dk, dv [B,H,N,d]   lse [B,H,W] fp32   (all DEVICE, 16-byte aligned)
  * out and lse are what tlin_attn_forward returned for the same q, k, v and causal_window (lse is
  * required here); dout is the loss gradient with respect to out; the loss must not depend on lse.
- * dq, dk, dv are overwritten (keys that no query may use get zeros).  d in {64,128}.
- * Needs a workspace of tlin_workspace_bytes_backward bytes (row sums and the fp32 dq accumulator).
- * This first path runs on the CUDA cores.  Errors as for tlin_attn_forward.
+ * dq, dk, dv are overwritten (keys that no query may use get zeros).
+ * bf16: d in {64,128} runs on the tensor cores (two kernels that recompute p, no atomics, bitwise repeatable); any other
+ * d that is a multiple of 8 up to 256 runs on the CUDA-core kernels (dq summed with fp32 atomics).  f32: d a multiple
+ * of 4 up to 256 (covers the paper's d = 36), CUDA-core kernels.
+ * Needs a workspace of tlin_workspace_bytes_backward bytes (row sums, partial or accumulated dq in fp32).
+ * Errors as for tlin_attn_forward.
  */
 int tlin_attn_backward(const void* q, const void* k, const void* v, const void* out, const float* lse,
                        const void* dout, void* dq, void* dk, void* dv,
                        int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream);
+int tlin_attn_backward_f32(const float* q, const float* k, const float* v, const float* out, const float* lse,
+                           const float* dout, float* dq, float* dk, float* dv,
+                           int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------
  * Exact merge of two results over DISJOINT key sets for the same queries (not in the paper; it is

@@ -45,6 +45,7 @@ SIGNATURES = {
     "tlin_attn_forward_f32": (_i, [_vp] * 5 + [_i] * 6 + [_vp]),
     "tlin_attn_forward_host": (_i, [_vp] * 10 + [_i] * 6 + [_vp]),
     "tlin_attn_backward": (_i, [_vp] * 9 + [_i] * 6 + [_vp]),
+    "tlin_attn_backward_f32": (_i, [_vp] * 9 + [_i] * 6 + [_vp]),
     "tlin_decode_step": (_i, [_vp] * 7 + [_i] * 5 + [_vp]),
     "tlin_decode_step_host": (_i, [_vp] * 12 + [_i] * 5 + [_vp]),
     "tlin_decode_step_static": (_i, [_vp] * 7 + [_i] * 5 + [_vp]),
@@ -187,26 +188,35 @@ def tlin_attn_forward_f32(q, k, v, out=None, lse=None, causal_window=1, stream=N
     return out, lse
 
 
-def tlin_attn_backward(q, k, v, out, lse, dout, dq=None, dk=None, dv=None, causal_window=1, stream=None):
-    """bf16 backward of ``tlin_attn_forward``: (dq [B,H,W,d], dk, dv [B,H,N,d]) for the loss gradient ``dout``.
-
-    ``out`` and ``lse`` are the forward's results for the same q, k, v and causal_window."""
+def _backward(fn_name, dtype, q, k, v, out, lse, dout, dq, dk, dv, causal_window, stream):
     B, H, W, d = q.shape
     N = k.shape[2]
     for t, shape, name in ((q, (B, H, W, d), "q"), (k, (B, H, N, d), "k"), (v, (B, H, N, d), "v"),
                            (out, (B, H, W, d), "out"), (dout, (B, H, W, d), "dout")):
-        _dev(t, torch.bfloat16, shape, name)
+        _dev(t, dtype, shape, name)
     _dev(lse, torch.float32, (B, H, W), "lse")
     dq = torch.empty_like(q) if dq is None else dq
     dk = torch.empty_like(k) if dk is None else dk
     dv = torch.empty_like(v) if dv is None else dv
-    _dev(dq, torch.bfloat16, (B, H, W, d), "dq")
-    _dev(dk, torch.bfloat16, (B, H, N, d), "dk")
-    _dev(dv, torch.bfloat16, (B, H, N, d), "dv")
+    _dev(dq, dtype, (B, H, W, d), "dq")
+    _dev(dk, dtype, (B, H, N, d), "dk")
+    _dev(dv, dtype, (B, H, N, d), "dv")
     ensure_workspace(workspace_bytes_backward(B, H, N, W, d), q.device)
-    _check(lib().tlin_attn_backward(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk),
-                                    _ptr(dv), B, H, N, W, d, int(causal_window), _stream(stream)), "tlin_attn_backward")
+    _check(getattr(lib(), fn_name)(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk),
+                                   _ptr(dv), B, H, N, W, d, int(causal_window), _stream(stream)), fn_name)
     return dq, dk, dv
+
+
+def tlin_attn_backward(q, k, v, out, lse, dout, dq=None, dk=None, dv=None, causal_window=1, stream=None):
+    """bf16 backward of ``tlin_attn_forward``: (dq [B,H,W,d], dk, dv [B,H,N,d]) for the loss gradient ``dout``.
+
+    ``out`` and ``lse`` are the forward's results for the same q, k, v and causal_window."""
+    return _backward("tlin_attn_backward", torch.bfloat16, q, k, v, out, lse, dout, dq, dk, dv, causal_window, stream)
+
+
+def tlin_attn_backward_f32(q, k, v, out, lse, dout, dq=None, dk=None, dv=None, causal_window=1, stream=None):
+    """fp32 backward of ``tlin_attn_forward_f32`` (CUDA-core kernels)."""
+    return _backward("tlin_attn_backward_f32", torch.float32, q, k, v, out, lse, dout, dq, dk, dv, causal_window, stream)
 
 
 def tlin_attn_forward_host(q_h, k_h, v_h, out_h, lse_h, q_d, k_d, v_d, out_d, lse_d, causal_window=1, stream=None):

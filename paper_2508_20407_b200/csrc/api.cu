@@ -110,9 +110,9 @@ extern "C" int tlin_attn_forward_host(const void* q_h, const void* k_h, const vo
     return TLIN_OK;
 }
 
-extern "C" int tlin_attn_backward(const void* q, const void* k, const void* v, const void* out, const float* lse,
-                                  const void* dout, void* dq, void* dk, void* dv,
-                                  int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream) {
+static int backward_common(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                           const void* dout, void* dq, void* dk, void* dv,
+                           int B, int H, int N, int W, int d, int causal_window, int is_f32, cudaStream_t st) {
     t_launches = 0;
     if (!q || !k || !v || !out || !lse || !dout || !dq || !dk || !dv) return TLIN_ERR_INVALID_ARG;
     if (B <= 0 || H <= 0 || N <= 0 || W <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
@@ -121,22 +121,33 @@ extern "C" int tlin_attn_backward(const void* q, const void* k, const void* v, c
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(dout) ||
         !aligned16(dq) || !aligned16(dk) || !aligned16(dv)) return TLIN_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(lse) & 3u) return TLIN_ERR_INVALID_ARG;
-    if (d != 64 && d != 128) return TLIN_ERR_UNSUPPORTED;
+    if (is_f32 ? (d % 4 != 0 || d > 256) : (d % 8 != 0 || d > 256)) return TLIN_ERR_UNSUPPORTED;
     int sms = 0;
     int rc = device_info(&sms);
     if (rc != TLIN_OK) return rc;
     const Workspace w = workspace();
-    if (forward_impl() == 1) {
+    const bool tc = !is_f32 && (d == 64 || d == 128) && forward_impl() != 1;
+    if (!tc) {
         if (!w.ptr || w.bytes < bwd_workspace_bytes(B, H, W, d)) return TLIN_ERR_WORKSPACE;
-        return launch_bwd_simt(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, d, causal_window, (float*)w.ptr, sms,
-                               (cudaStream_t)stream);
+        return launch_bwd_simt(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, d, causal_window, is_f32, (float*)w.ptr, sms, st);
     }
     tlin_fwd_plan plan;
     rc = tlin_plan_forward(B, H, N, W, d, causal_window, 0, sms, &plan);   // the dQ kernel follows the forward's plan
     if (rc != TLIN_OK) return rc;
     if (!w.ptr || w.bytes < bwd_tc_workspace_bytes(B, H, W, d, plan)) return TLIN_ERR_WORKSPACE;
-    return launch_bwd_tc(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, d, causal_window, plan, (float*)w.ptr, sms,
-                         (cudaStream_t)stream);
+    return launch_bwd_tc(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, d, causal_window, plan, (float*)w.ptr, sms, st);
+}
+
+extern "C" int tlin_attn_backward(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                                  const void* dout, void* dq, void* dk, void* dv,
+                                  int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream) {
+    return backward_common(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, d, causal_window, 0, (cudaStream_t)stream);
+}
+
+extern "C" int tlin_attn_backward_f32(const float* q, const float* k, const float* v, const float* out, const float* lse,
+                                      const float* dout, float* dq, float* dk, float* dv,
+                                      int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream) {
+    return backward_common(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, d, causal_window, 1, (cudaStream_t)stream);
 }
 
 extern "C" size_t tlin_workspace_bytes_backward(int B, int H, int N, int W, int d) {

@@ -44,8 +44,8 @@ int launch_decode(const void* q_new, const void* k_new, const void* v_new, void*
                   void* out, float* lse, int B, int H, int Ncap, int pos, const int* pos_per_seq, int d,
                   const tlin_decode_plan& plan, float* ws, cudaStream_t st);
 int launch_bwd_simt(const void* q, const void* k, const void* v, const void* out, const float* lse, const void* dout,
-                    void* dq, void* dk, void* dv, int B, int H, int N, int W, int d, int causal, float* ws, int num_sms,
-                    cudaStream_t st);
+                    void* dq, void* dk, void* dv, int B, int H, int N, int W, int d, int causal, int is_f32, float* ws,
+                    int num_sms, cudaStream_t st);
 size_t bwd_workspace_bytes(long long B, long long H, long long W, int d);
 int launch_bwd_tc(const void* q, const void* k, const void* v, const void* out, const float* lse, const void* dout,
                   void* dq, void* dk, void* dv, int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& plan,

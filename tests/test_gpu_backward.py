@@ -126,7 +126,7 @@ def test_backward_tensor_core_path_is_bitwise_repeatable():
 
 def test_backward_cuda_core_path_is_deterministic_up_to_the_dq_sum_order():
     # dk, dv have one owner per element: bitwise repeatable.  dq is summed over key slices with atomics: equal within
-    # fp32 rounding, so the rounded bf16 values may differ in the last place only.
+    # fp32 rounding, so the rounded bf16 values differ by at most a last place of the largest elements.
     wl = synth.Workload("bwd", 1, 2, 128, 3000, 64, seed=9, causal_window=1)
     q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
     dout = torch.randn(q.shape, device=DEV).to(torch.bfloat16)
@@ -134,7 +134,7 @@ def test_backward_cuda_core_path_is_deterministic_up_to_the_dq_sum_order():
     b = grads(q, k, v, dout, 1, 1)
     assert torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])
     diff = (a[0].float() - b[0].float()).abs()
-    assert float((diff / (a[0].float().abs() + 1e-20)).max()) <= 2.0 ** -7
+    assert float(diff.max()) <= 2.0 ** -7 * float(a[0].float().abs().max())
 
 
 def test_backward_argument_errors():
@@ -143,7 +143,40 @@ def test_backward_argument_errors():
     lse = torch.zeros(1, 1, 32, dtype=torch.float32, device=DEV)
     with pytest.raises(tl.TlinError):        # N < W with the window rule
         tl.tlin_attn_backward(q, k, k, q, lse, q, causal_window=1)
-    q96 = torch.zeros(1, 1, 8, 96, dtype=torch.bfloat16, device=DEV)
+    q100 = torch.zeros(1, 1, 8, 100, dtype=torch.bfloat16, device=DEV)
     lse8 = torch.zeros(1, 1, 8, dtype=torch.float32, device=DEV)
-    with pytest.raises(tl.TlinError):        # head size outside {64, 128}
-        tl.tlin_attn_backward(q96, q96, q96, q96, lse8, q96, causal_window=0)
+    with pytest.raises(tl.TlinError):        # bf16 head sizes are multiples of 8
+        tl.tlin_attn_backward(q100, q100, q100, q100, lse8, q100, causal_window=0)
+
+
+ODD = [(1, 2, 300, 77, 40, 1), (2, 1, 515, 130, 96, 0), (1, 1, 200, 64, 256, 1), (1, 2, 129, 33, 8, 1)]
+
+
+@pytest.mark.parametrize("B,H,N,W,d,causal", ODD)
+def test_backward_other_head_sizes_bf16(B, H, N, W, d, causal):
+    # head sizes outside {64, 128} are served by the CUDA-core kernels whatever the switch says
+    run_case(B, H, N, W, d, causal, seed=700 + N + d, impl=0)
+
+
+F32 = [(1, 2, 300, 77, 36, 1), (2, 1, 515, 130, 64, 0), (1, 1, 1000, 200, 128, 1), (1, 3, 97, 97, 100, 1), (1, 1, 1, 1, 4, 1)]
+
+
+@pytest.mark.parametrize("B,H,N,W,d,causal", F32)
+def test_backward_f32(B, H, N, W, d, causal):
+    # fp32 tensors, fp32 arithmetic (the paper's own model has d = 36): gates of the fp32 forward, relative to the
+    # gradient's magnitude
+    wl = synth.Workload("bwd32", B, H, d, N, W, seed=900 + N + d, causal_window=causal)
+    q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.float32)
+    g = torch.Generator(device="cpu").manual_seed(3)
+    dout = torch.randn(q.shape, generator=g, dtype=torch.float32).to(DEV)
+    out, lse = tl.tlin_attn_forward_f32(q, k, v, causal_window=causal)
+    dq, dk, dv = tl.tlin_attn_backward_f32(q, k, v, out, lse, dout, causal_window=causal)
+    torch.cuda.synchronize()
+    assert tl.tlin_get_status() == 0
+    refs = oracle.attn_backward(q.cpu(), k.cpu(), v.cpu(), dout.cpu(), causal)
+    for got, ref, name in zip((dq, dk, dv), refs, ("dq", "dk", "dv")):
+        e = parity.errors(got.cpu().numpy(), ref)
+        scale = float(np.abs(ref).max())
+        assert e["max_abs"] <= 1e-4 * scale + 1e-6, f"{name}: max|err| {e['max_abs']:.3e} vs max|ref| {scale:.3e}"
+        if scale > 1e-3:
+            assert e["rel_l2"] <= 1e-4, f"{name}: rel L2 {e['rel_l2']:.3e}"
