@@ -436,7 +436,10 @@ struct BCfg {
     // TMEM columns: R0, R1 (S, then dP, then dS as bf16; 128 each), dQ0, dQ1 (D each)
     static constexpr uint32_t kColR = 0, kColDQ = 256;
     static constexpr int kThreads = 32 * 12;                   // warps 10 and 11 only lend their registers
-    static constexpr int kComputeRegs = 216, kOtherRegs = 72;
+    // setmaxnreg moves registers between warpgroups; the CTA starts with 168 per thread (65536 / 384, rounded down to a
+    // multiple of 8), and an increase beyond what the other warpgroup released would wait for ever
+    static constexpr int kComputeRegs = 200, kOtherRegs = 104;
+    static_assert(256 * kComputeRegs + 128 * kOtherRegs <= kThreads * 168, "register budget of the CTA exceeded");
 };
 
 template <int D>
@@ -737,42 +740,36 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 tc_fence_after();
             }
             const bool whole = s.t_begin == 0 && s.t_end == p.key_tiles;
-            if (whole) {
-                __nv_bfloat16* drow = reinterpret_cast<__nv_bfloat16*>(p.dq) + ((long long)s.bh * p.W + row) * D;
+            __nv_bfloat16* drow = reinterpret_cast<__nv_bfloat16*>(p.dq) + ((long long)s.bh * p.W + row) * D;
+            // partial sum -> workspace slot (0: first segment of this CTA's range, 1: a later one); unscaled fp32
+            float* prow = p.ws + ((long long)blockIdx.x * 2 + (s.bh == bh_first ? 0 : 1)) * (long long)kTileM * D + (long long)(i * kQTile + r) * D;
+            const float f = whole ? p.scale : 1.f;
+#pragma unroll 1
+            for (int c = 0; c < D / 16; ++c) {
+                uint32_t o[16];
+                if (cnt_i > 0) {
+                    tmem_ld16_async(tDQ + c * 16, o);
+                    tmem_wait_ld16(o);
+                } else {
 #pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t o[32];
-                    if (cnt_i > 0) tmem_ld32(tDQ + c * 32, o);
+                    for (int e = 0; e < 16; ++e) o[e] = 0u;
+                }
+                if (whole) {
                     if (row_ok) {
 #pragma unroll
-                        for (int v4 = 0; v4 < 4; ++v4) {
+                        for (int v4 = 0; v4 < 2; ++v4) {
                             uint4 w;
-                            w.x = pack_bf16x2(__uint_as_float(o[v4 * 8 + 0]) * p.scale, __uint_as_float(o[v4 * 8 + 1]) * p.scale);
-                            w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * p.scale, __uint_as_float(o[v4 * 8 + 3]) * p.scale);
-                            w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * p.scale, __uint_as_float(o[v4 * 8 + 5]) * p.scale);
-                            w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * p.scale, __uint_as_float(o[v4 * 8 + 7]) * p.scale);
-                            if (cnt_i == 0) w = make_uint4(0, 0, 0, 0);
-                            *reinterpret_cast<uint4*>(drow + c * 32 + v4 * 8) = w;
+                            w.x = pack_bf16x2(__uint_as_float(o[v4 * 8 + 0]) * f, __uint_as_float(o[v4 * 8 + 1]) * f);
+                            w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * f, __uint_as_float(o[v4 * 8 + 3]) * f);
+                            w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * f, __uint_as_float(o[v4 * 8 + 5]) * f);
+                            w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * f, __uint_as_float(o[v4 * 8 + 7]) * f);
+                            *reinterpret_cast<uint4*>(drow + c * 16 + v4 * 8) = w;
                         }
                     }
-                }
-            } else {
-                // partial sum -> workspace slot (0: first segment of this CTA's range, 1: a later one); unscaled fp32
-                const int slot = s.bh == bh_first ? 0 : 1;
-                float* orow = p.ws + ((long long)blockIdx.x * 2 + slot) * (long long)kTileM * D + (long long)(i * kQTile + r) * D;
+                } else {
 #pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t o[32];
-                    if (cnt_i > 0) tmem_ld32(tDQ + c * 32, o);
-#pragma unroll
-                    for (int v4 = 0; v4 < 8; ++v4) {
-                        float4 w;
-                        w.x = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 0]) : 0.f;
-                        w.y = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 1]) : 0.f;
-                        w.z = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 2]) : 0.f;
-                        w.w = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 3]) : 0.f;
-                        *reinterpret_cast<float4*>(orow + c * 32 + v4 * 4) = w;
-                    }
+                    for (int v4 = 0; v4 < 4; ++v4)
+                        *reinterpret_cast<uint4*>(prow + c * 16 + v4 * 4) = make_uint4(o[v4 * 4], o[v4 * 4 + 1], o[v4 * 4 + 2], o[v4 * 4 + 3]);
                 }
             }
             tc_fence_before();

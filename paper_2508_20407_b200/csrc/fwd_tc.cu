@@ -33,6 +33,8 @@ constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr int kThreads = 32 * 12;          // warps 10 and 11 only lend their registers
 constexpr int kSoftmaxRegs = 216, kOtherRegs = 72;   // 256*224 + 128*56 = 384*168 registers
+// an increase beyond what the other warpgroup released would wait for ever
+static_assert(256 * kSoftmaxRegs + 128 * kOtherRegs <= kThreads * 168, "register budget of the CTA exceeded");
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kPolyPairs = 5;                // of every 16 column pairs, this many get 2^x from the polynomial
