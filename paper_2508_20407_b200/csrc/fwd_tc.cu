@@ -298,6 +298,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         uint32_t n = 0;     // tiles processed by this warpgroup (phase counter of s_full/p_full/pv_done)
         bool ok = true;
         SegmentWalker walk(p);
+        const int bh_first = (int)(walk.u / p.key_tiles);  // (b,h) of this CTA's first unit (used under schedule 0 only)
         Segment s;
         while (ok && walk.next(s)) {
             const int row0 = s.qt * kTileM;
@@ -422,47 +423,48 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             const float inv_l = l > 0.f ? 1.f / l : 0.f;
             const float lse_val = l > 0.f ? (m_ref + log2f(l)) * kLn2 : -CUDART_INF_F;
             const bool store = row < p.W;
-            if (whole) {
-                __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + ((long long)s.bh * p.W + row) * D;
+            __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + ((long long)s.bh * p.W + row) * D;
+            // partial result -> workspace slot (0: first segment of this CTA's range, 1: a later one)
+            float* pbase = p.ws + ((long long)blockIdx.x * 2 + (s.bh == bh_first ? 0 : 1)) * (long long)kTileM * (D + 1);
+            float* prow = pbase + (long long)(i * kQTile + r) * D;
 #pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t o[32];
-                    if (cnt_i > 0) tmem_ld32(tO + c * 32, o);
+            for (int c = 0; c < D / 16; ++c) {
+                uint32_t o[16];
+                if (cnt_i > 0) {
+                    tmem_ld16_async(tO + c * 16, o);
+                    tmem_wait_ld16(o);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) o[e] = 0u;
+                }
+                if (whole) {
                     if (store) {
 #pragma unroll
-                        for (int v4 = 0; v4 < 4; ++v4) {
+                        for (int v4 = 0; v4 < 2; ++v4) {
                             uint4 w;
                             w.x = pack_bf16x2(__uint_as_float(o[v4 * 8 + 0]) * inv_l, __uint_as_float(o[v4 * 8 + 1]) * inv_l);
                             w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * inv_l, __uint_as_float(o[v4 * 8 + 3]) * inv_l);
                             w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * inv_l, __uint_as_float(o[v4 * 8 + 5]) * inv_l);
                             w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * inv_l, __uint_as_float(o[v4 * 8 + 7]) * inv_l);
-                            *reinterpret_cast<uint4*>(orow + c * 32 + v4 * 8) = w;
+                            *reinterpret_cast<uint4*>(orow + c * 16 + v4 * 8) = w;
                         }
                     }
-                }
-                if (store && p.lse != nullptr) p.lse[(long long)s.bh * p.W + row] = lse_val;
-            } else {
-                // partial result -> workspace slot (0: first segment of this CTA's range, 1: a later one)
-                const int g = (int)(blockIdx.x / p.q_tiles);          // partial segments exist only under schedule 0
-                const long long u_first = (long long)(((unsigned long long)g * (unsigned long long)p.total_units) / (unsigned)p.n_groups);
-                const int slot = s.bh == (int)(u_first / p.key_tiles) ? 0 : 1;
-                float* base = p.ws + ((long long)blockIdx.x * 2 + slot) * (long long)kTileM * (D + 1);
-                float* orow = base + (long long)(i * kQTile + r) * D;
+                } else {
 #pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t o[32];
-                    if (cnt_i > 0) tmem_ld32(tO + c * 32, o);
-#pragma unroll
-                    for (int v4 = 0; v4 < 8; ++v4) {
+                    for (int v4 = 0; v4 < 4; ++v4) {
                         float4 w;
-                        w.x = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 0]) * inv_l : 0.f;
-                        w.y = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 1]) * inv_l : 0.f;
-                        w.z = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 2]) * inv_l : 0.f;
-                        w.w = cnt_i > 0 ? __uint_as_float(o[v4 * 4 + 3]) * inv_l : 0.f;
-                        *reinterpret_cast<float4*>(orow + c * 32 + v4 * 4) = w;
+                        w.x = __uint_as_float(o[v4 * 4 + 0]) * inv_l;
+                        w.y = __uint_as_float(o[v4 * 4 + 1]) * inv_l;
+                        w.z = __uint_as_float(o[v4 * 4 + 2]) * inv_l;
+                        w.w = __uint_as_float(o[v4 * 4 + 3]) * inv_l;
+                        *reinterpret_cast<float4*>(prow + c * 16 + v4 * 4) = w;
                     }
                 }
-                base[(long long)kTileM * D + i * kQTile + r] = lse_val;
+            }
+            if (whole) {
+                if (store && p.lse != nullptr) p.lse[(long long)s.bh * p.W + row] = lse_val;
+            } else {
+                pbase[(long long)kTileM * D + i * kQTile + r] = lse_val;
             }
             tc_fence_before();      // TMEM reads of O are complete before the next segment's arrive lets PV overwrite it
         }
