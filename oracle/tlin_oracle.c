@@ -20,6 +20,10 @@
  *     keys, unmasked (causal_window = 0).
  *   - Appendix A, "Cache Hit": in a cached step only the newest token takes
  *     part; it attends to every cached row including its own.
+ *   - Section 4.1: training is a forward and a backward pass through every
+ *     layer.  The paper states no gradient algorithm; tlin_ref_attn_backward
+ *     is the chain rule of the formula above written out row by row (pinned by
+ *     central differences of the forward, a library autograd and closed forms).
  *
  * Every function is pinned by tests that do not call it to produce their
  * expectation (closed forms, brute force with an explicit probability matrix,

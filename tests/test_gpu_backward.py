@@ -180,3 +180,19 @@ def test_backward_f32(B, H, N, W, d, causal):
         assert e["max_abs"] <= 1e-4 * scale + 1e-6, f"{name}: max|err| {e['max_abs']:.3e} vs max|ref| {scale:.3e}"
         if scale > 1e-3:
             assert e["rel_l2"] <= 1e-4, f"{name}: rel L2 {e['rel_l2']:.3e}"
+
+
+def test_backward_at_the_benchmarked_training_shape_on_two_heads():
+    # the full train_chunk workload (B4 H32 N8192 W1024 d128, the launch configuration bench.py times); the oracle
+    # recomputes two (b,h) pairs of it, which are independent problems
+    wl = synth.WORKLOADS["train_chunk"]
+    q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
+    g = torch.Generator(device="cpu").manual_seed(wl.seed + 99)
+    dout = torch.randn(q.shape, generator=g, dtype=torch.float32).to(torch.bfloat16).to(DEV)
+    dq, dk, dv = grads(q, k, v, dout, wl.causal_window, 0)
+    for b, h in ((0, 0), (3, 17)):
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        rq, rk, rv = oracle.attn_backward(q[sl].cpu(), k[sl].cpu(), v[sl].cpu(), dout[sl].cpu(), wl.causal_window)
+        compare(dq[sl], rq, f"train_chunk b{b} h{h} dq")
+        compare(dk[sl], rk, f"train_chunk b{b} h{h} dk")
+        compare(dv[sl], rv, f"train_chunk b{b} h{h} dv")
