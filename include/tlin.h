@@ -64,6 +64,19 @@ int tlin_attn_forward(const void* q, const void* k, const void* v, void* out, fl
 int tlin_attn_forward_f32(const float* q, const float* k, const float* v, float* out, float* lse,
                           int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream);
 
+/* Chunk-scheduled forward for sliding-window training (Section 5.1: the window slides by W_og and every chunk attends to
+ * all the chunks before it): C problems over ONE key/value tensor, problem c using its first n_keys[c] rows.
+ *   q   [C,B,H,W,d]   the W queries of each chunk        k,v [B,H,L,d]   shared; n_keys[c] <= L (HOST array of C ints)
+ *   out [C,B,H,W,d]   lse [C,B,H,W] (may be NULL)
+ * causal_window as in tlin_attn_forward, applied per chunk with N = n_keys[c] (with n_keys[c] = (c+1)*W and
+ * causal_window = 1 chunk c is the c-th window of the training pass).  The chunks are issued as C launches of the forward
+ * kernel on `stream`, each with its own plan, reading k and v in place through a strided tensor map; nothing is copied.
+ * bf16, d in {64,128} (tensor-core path) only; other shapes return TLIN_ERR_UNSUPPORTED.  Workspace:
+ * tlin_workspace_bytes_forward_prefixes (the largest of the chunks' needs). */
+int tlin_attn_forward_prefixes(const void* q, const void* k, const void* v, void* out, float* lse,
+                               int B, int H, int L, int W, int d, int C, const int32_t* n_keys,
+                               int causal_window, tlin_stream_t stream);
+
 /* Same as tlin_attn_forward with HOST input/output buffers (ideally pinned).  *_h are HOST
  * pointers; *_d are DEVICE staging buffers of the same shapes, supplied by the caller.  Copies
  * q,k,v host->device, runs the forward, copies out (and lse if lse_h != NULL) device->host, all on
@@ -167,6 +180,7 @@ int tlin_merge_lse_f32(const float* out_a, const float* lse_a, const float* out_
  */
 size_t tlin_workspace_bytes_forward(int B, int H, int N, int W, int d, int causal_window);
 size_t tlin_workspace_bytes_decode(int B, int H, int Ncap, int d);
+size_t tlin_workspace_bytes_forward_prefixes(int B, int H, int W, int d, int C, const int32_t* n_keys, int causal_window);
 size_t tlin_workspace_bytes_backward(int B, int H, int N, int W, int d);
 int tlin_set_workspace(void* dev_ptr, size_t bytes);
 

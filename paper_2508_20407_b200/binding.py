@@ -43,6 +43,7 @@ _vp, _i, _i64, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_siz
 SIGNATURES = {
     "tlin_attn_forward": (_i, [_vp] * 5 + [_i] * 6 + [_vp]),
     "tlin_attn_forward_f32": (_i, [_vp] * 5 + [_i] * 6 + [_vp]),
+    "tlin_attn_forward_prefixes": (_i, [_vp] * 5 + [_i] * 6 + [_vp, _i, _vp]),
     "tlin_attn_forward_host": (_i, [_vp] * 10 + [_i] * 6 + [_vp]),
     "tlin_attn_backward": (_i, [_vp] * 9 + [_i] * 6 + [_vp]),
     "tlin_attn_backward_f32": (_i, [_vp] * 9 + [_i] * 6 + [_vp]),
@@ -54,6 +55,7 @@ SIGNATURES = {
     "tlin_merge_lse_f32": (_i, [_vp] * 6 + [_i64, _i, _vp]),
     "tlin_workspace_bytes_forward": (_sz, [_i] * 6),
     "tlin_workspace_bytes_decode": (_sz, [_i] * 4),
+    "tlin_workspace_bytes_forward_prefixes": (_sz, [_i] * 5 + [_vp, _i]),
     "tlin_workspace_bytes_backward": (_sz, [_i] * 5),
     "tlin_set_workspace": (_i, [_vp, _sz]),
     "tlin_plan_forward": (_i, [_i] * 8 + [ctypes.POINTER(FwdPlan)]),
@@ -167,6 +169,31 @@ def tlin_attn_forward(q, k, v, out=None, lse=None, causal_window=1, stream=None)
     ensure_workspace(workspace_bytes_forward(B, H, N, W, d, causal_window), q.device)
     _check(lib().tlin_attn_forward(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), B, H, N, W, d,
                                    int(causal_window), _stream(stream)), "tlin_attn_forward")
+    return out, lse
+
+
+def tlin_attn_forward_prefixes(q, k, v, n_keys, out=None, lse=None, causal_window=1, stream=None):
+    """Chunk-scheduled forward: q [C,B,H,W,d], shared k,v [B,H,L,d], chunk c uses the first n_keys[c] key rows.
+
+    Returns (out [C,B,H,W,d] bf16, lse [C,B,H,W] fp32)."""
+    C, B, H, W, d = q.shape
+    L = k.shape[2]
+    n_keys = [int(x) for x in n_keys]
+    if len(n_keys) != C:
+        raise ValueError("one key count per chunk")
+    _dev(q, torch.bfloat16, (C, B, H, W, d), "q")
+    _dev(k, torch.bfloat16, (B, H, L, d), "k")
+    _dev(v, torch.bfloat16, (B, H, L, d), "v")
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((C, B, H, W), dtype=torch.float32, device=q.device)
+    _dev(out, torch.bfloat16, (C, B, H, W, d), "out")
+    _dev(lse, torch.float32, (C, B, H, W), "lse")
+    arr = (ctypes.c_int32 * C)(*n_keys)
+    ensure_workspace(int(lib().tlin_workspace_bytes_forward_prefixes(B, H, W, d, C, arr, int(causal_window))), q.device)
+    _check(lib().tlin_attn_forward_prefixes(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), B, H, L, W, d, C, arr,
+                                            int(causal_window), _stream(stream)), "tlin_attn_forward_prefixes")
     return out, lse
 
 

@@ -52,7 +52,8 @@ int forward_impl() { return g_impl.load(); }
 using namespace tlin;
 
 static int forward_common(const void* q, const void* k, const void* v, void* out, float* lse,
-                          int B, int H, int N, int W, int d, int causal_window, int is_f32, cudaStream_t st) {
+                          int B, int H, int N, int W, int d, int causal_window, int is_f32, cudaStream_t st,
+                          long long kv_rows_alloc = 0) {
     t_launches = 0;
     if (!q || !k || !v || !out) return TLIN_ERR_INVALID_ARG;
     if (B <= 0 || H <= 0 || N <= 0 || W <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
@@ -69,6 +70,7 @@ static int forward_common(const void* q, const void* k, const void* v, void* out
     if (rc != TLIN_OK) return rc;
     rc = tlin_plan_forward(B, H, N, W, d, causal_window, is_f32, sms, &plan);
     if (rc != TLIN_OK) return rc;
+    if (kv_rows_alloc > 0 && (is_f32 || !plan.tensor_path)) return TLIN_ERR_UNSUPPORTED;   // strided k, v: tensor path only
     if (is_f32)
         return launch_fwd_simt_f32((const float*)q, (const float*)k, (const float*)v, (float*)out, lse, B, H, N, W, d, causal_window, st);
     if (!plan.tensor_path)
@@ -79,12 +81,41 @@ static int forward_common(const void* q, const void* k, const void* v, void* out
         if (!w.ptr || w.bytes < (size_t)plan.workspace_bytes) return TLIN_ERR_WORKSPACE;
         ws = (float*)w.ptr;
     }
-    return launch_fwd_tc(q, k, v, out, lse, B, H, N, W, d, causal_window, plan, ws, st);
+    return launch_fwd_tc(q, k, v, out, lse, B, H, N, W, d, causal_window, plan, ws, kv_rows_alloc, st);
 }
 
 extern "C" int tlin_attn_forward(const void* q, const void* k, const void* v, void* out, float* lse,
                                  int B, int H, int N, int W, int d, int causal_window, tlin_stream_t stream) {
     return forward_common(q, k, v, out, lse, B, H, N, W, d, causal_window, 0, (cudaStream_t)stream);
+}
+
+extern "C" int tlin_attn_forward_prefixes(const void* q, const void* k, const void* v, void* out, float* lse,
+                                          int B, int H, int L, int W, int d, int C, const int32_t* n_keys,
+                                          int causal_window, tlin_stream_t stream) {
+    if (!n_keys || C <= 0 || L <= 0 || B <= 0 || H <= 0 || W <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    for (int c = 0; c < C; ++c)
+        if (n_keys[c] <= 0 || n_keys[c] > L) return TLIN_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return TLIN_ERR_UNSUPPORTED;
+    const size_t q_chunk = (size_t)B * H * W * d * 2, lse_chunk = (size_t)B * H * W;
+    int total = 0;                 // a chunked call counts the launches of all its chunks
+    for (int c = 0; c < C; ++c) {
+        const int rc = forward_common((const char*)q + c * q_chunk, k, v, (char*)out + c * q_chunk, lse ? lse + c * lse_chunk : nullptr,
+                                      B, H, n_keys[c], W, d, causal_window, 0, (cudaStream_t)stream, L);
+        if (rc != TLIN_OK) return rc;
+        total += t_launches;
+    }
+    t_launches = total;
+    return TLIN_OK;
+}
+
+extern "C" size_t tlin_workspace_bytes_forward_prefixes(int B, int H, int W, int d, int C, const int32_t* n_keys, int causal_window) {
+    size_t need = 0;
+    if (!n_keys) return 0;
+    for (int c = 0; c < C; ++c) {
+        const size_t b = tlin_workspace_bytes_forward(B, H, n_keys[c], W, d, causal_window);
+        if (b > need) need = b;
+    }
+    return need;
 }
 
 extern "C" int tlin_attn_forward_f32(const float* q, const float* k, const float* v, float* out, float* lse,

@@ -573,13 +573,13 @@ fwd_merge_kernel(const Params p) {
 
 template <int D>
 int launch_d(const void* q, const void* k, const void* v, void* out, float* lse, int B, int H, int N, int W,
-             int causal, const tlin_fwd_plan& plan, float* ws, cudaStream_t st) {
+             int causal, const tlin_fwd_plan& plan, float* ws, long long kv_rows_alloc, cudaStream_t st) {
     using C = Cfg<D>;
     const long long bh = (long long)B * H;
     CUtensorMap mq, mk, mv;
     int rc = make_map(&mq, q, D, W, bh);
-    if (rc == TLIN_OK) rc = make_map(&mk, k, D, N, bh);
-    if (rc == TLIN_OK) rc = make_map(&mv, v, D, N, bh);
+    if (rc == TLIN_OK) rc = make_map(&mk, k, D, N, bh, kQTile, kv_rows_alloc);
+    if (rc == TLIN_OK) rc = make_map(&mv, v, D, N, bh, kQTile, kv_rows_alloc);
     if (rc != TLIN_OK) return rc;
     Params p;
     p.out = out; p.lse = lse; p.ws = ws; p.status = status_word();
@@ -608,11 +608,11 @@ int launch_d(const void* q, const void* k, const void* v, void* out, float* lse,
 
 int launch_fwd_tc(const void* q, const void* k, const void* v, void* out, float* lse,
                   int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& plan,
-                  float* ws, cudaStream_t st) {
+                  float* ws, long long kv_rows_alloc, cudaStream_t st) {
     if (plan.tile_m != kTileM || plan.tile_n != kTileN) return TLIN_ERR_UNSUPPORTED;
     if ((long long)B * H * W > 0x7fffffffLL) return TLIN_ERR_UNSUPPORTED;
-    if (d == 128) return launch_d<128>(q, k, v, out, lse, B, H, N, W, causal, plan, ws, st);
-    if (d == 64) return launch_d<64>(q, k, v, out, lse, B, H, N, W, causal, plan, ws, st);
+    if (d == 128) return launch_d<128>(q, k, v, out, lse, B, H, N, W, causal, plan, ws, kv_rows_alloc, st);
+    if (d == 64) return launch_d<64>(q, k, v, out, lse, B, H, N, W, causal, plan, ws, kv_rows_alloc, st);
     return TLIN_ERR_UNSUPPORTED;
 }
 

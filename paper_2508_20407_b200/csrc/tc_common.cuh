@@ -86,12 +86,13 @@ inline EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// [BH, rows, D] bf16, box = 64 elements x box_rows rows x 1, 128-byte swizzle, zero fill outside.
-inline int make_map(CUtensorMap* m, const void* ptr, int D, long long rows, long long bh, int box_rows = kQTile) {
+// [BH, rows, D] bf16, box = 64 elements x box_rows rows x 1, 128-byte swizzle, zero fill outside.  rows_alloc > rows: only
+// the first `rows` rows of every (b,h) block of rows_alloc rows are visible (the rest reads as zero fill).
+inline int make_map(CUtensorMap* m, const void* ptr, int D, long long rows, long long bh, int box_rows = kQTile, long long rows_alloc = 0) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return TLIN_ERR_CUDA;
     cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)bh};
-    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)rows * D * 2};
+    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)(rows_alloc > 0 ? rows_alloc : rows) * D * 2};
     cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     cuuint32_t es[3] = {1, 1, 1};
     const CUresult rc = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,

@@ -39,7 +39,7 @@ int launch_fwd_simt_f32(const float* q, const float* k, const float* v, float* o
                         int B, int H, int N, int W, int d, int causal, cudaStream_t st);
 int launch_fwd_tc(const void* q, const void* k, const void* v, void* out, float* lse,
                   int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& plan,
-                  float* ws, cudaStream_t st);
+                  float* ws, long long kv_rows_alloc, cudaStream_t st);   // kv_rows_alloc: rows per (b,h) of k, v (0 = N)
 int launch_decode(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                   void* out, float* lse, int B, int H, int Ncap, int pos, const int* pos_per_seq, int d,
                   const tlin_decode_plan& plan, float* ws, cudaStream_t st);

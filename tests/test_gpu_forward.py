@@ -215,3 +215,46 @@ def test_full_size_sampled_rows(name, causal):
     wl = synth.WORKLOADS[name]
     impl = 2 if TC_AVAILABLE else 1
     sampled_rows_compare(wl, impl, 6, [(0, 0), (0, wl.H // 2), (0, wl.H - 1)], causal)
+
+
+def test_chunk_scheduled_forward_equals_per_chunk_calls_and_full_causal_attention():
+    # Sliding-window training (Section 5.1): C windows of W tokens, window c attends to everything up to its own end.
+    # One call over shared k, v; each chunk must equal the oracle on the key prefix, and the chunks laid end to end are
+    # the rows of plain causal attention over the whole sequence.
+    if not TC_AVAILABLE:
+        pytest.skip("tensor path not built")
+    C, B, H, W, d = 5, 2, 2, 96, 128
+    L = C * W
+    wl = synth.Workload("chunks", B, H, d, L, L, seed=41, causal_window=1)
+    q_all, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)          # q_all [B,H,L,d]
+    q = q_all.view(B, H, C, W, d).permute(2, 0, 1, 3, 4).contiguous()                 # [C,B,H,W,d]
+    n_keys = [(c + 1) * W for c in range(C)]
+    out, lse = tl.tlin_attn_forward_prefixes(q, k, v, n_keys, causal_window=1)
+    torch.cuda.synchronize()
+    assert tl.tlin_get_status() == 0 and tl.tlin_last_launch_count() >= C
+    for c in range(C):
+        ref, ref_lse = oracle.attn_forward(q[c].cpu(), k[:, :, :n_keys[c]].contiguous().cpu(), v[:, :, :n_keys[c]].contiguous().cpu(), 1)
+        parity.check(out[c].float().cpu().numpy(), lse[c].cpu().numpy(), ref, ref_lse, "bf16", f"chunk {c}")
+    full, full_lse = tl.tlin_attn_forward(q_all, k, v, causal_window=1)
+    stitched = out.permute(1, 2, 0, 3, 4).reshape(B, H, L, d)
+    assert float((stitched.float() - full.float()).abs().max()) <= 2e-2
+    assert float((lse.permute(1, 2, 0, 3).reshape(B, H, L) - full_lse).abs().max()) <= 1e-3
+
+
+def test_chunk_scheduled_forward_ragged_prefixes_without_mask():
+    # focused attention of every chunk over its own history: W summary queries, unmasked, arbitrary prefix lengths
+    if not TC_AVAILABLE:
+        pytest.skip("tensor path not built")
+    C, B, H, W, d, L = 3, 1, 3, 40, 64, 1000
+    wl = synth.Workload("prefixes", B, H, d, L, C * W, seed=43, causal_window=0)
+    q_all, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
+    q = q_all.view(B, H, C, W, d).permute(2, 0, 1, 3, 4).contiguous()
+    n_keys = [100, 333, 1000]
+    out, lse = tl.tlin_attn_forward_prefixes(q, k, v, n_keys, causal_window=0)
+    torch.cuda.synchronize()
+    assert tl.tlin_get_status() == 0
+    for c in range(C):
+        ref, ref_lse = oracle.attn_forward(q[c].cpu(), k[:, :, :n_keys[c]].contiguous().cpu(), v[:, :, :n_keys[c]].contiguous().cpu(), 0)
+        parity.check(out[c].float().cpu().numpy(), lse[c].cpu().numpy(), ref, ref_lse, "bf16", f"prefix {n_keys[c]}")
+    with pytest.raises(tl.TlinError):
+        tl.tlin_attn_forward_prefixes(q, k, v, [100, 333, 1001], causal_window=0)      # beyond the key tensor
