@@ -93,12 +93,13 @@ struct ACfg {
     static constexpr int kTileBytes = kQTile * D * 2;          // one 128-row tile (K or V)
     static constexpr int kHalfBytes = 64 * D * 2;              // one 64-row tile (Q or dout of a chain step)
     static constexpr int kBoxes = D / 64;
-    static constexpr int kSlots = D == 128 ? 5 : 8;            // ring of chain steps: Q (64 rows), dout (64 rows), 64 lse2 + 64 delta
+    static constexpr int kSlots = D == 128 ? 4 : 8;            // ring of chain steps: Q (64 rows), dout (64 rows), 64 lse2 + 64 delta
     static constexpr int kSlotBytes = 2 * kHalfBytes;
     static constexpr int kOffKV = 0;
     static constexpr int kOffRing = 2 * kTileBytes;
     static constexpr int kOffStats = kOffRing + kSlots * kSlotBytes;
-    static constexpr int kOffBars = kOffStats + kSlots * 512;
+    static constexpr int kOffStage = kOffStats + kSlots * 512;  // per compute warp 32 rows x D bytes: dK / dV rows on their way out
+    static constexpr int kOffBars = kOffStage + 8 * 32 * D;
     static constexpr int kNumBars = 8 + 2 * kSlots;
     static constexpr int kSmemBytes = kOffBars + kNumBars * 8 + 16;
     // TMEM columns: dK, dV (D each); per chain x (64 queries of the tile) 128 columns: S^T_x (64 fp32) and dP^T_x
@@ -381,29 +382,42 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             ok = __all_sync(0xffffffffu, mbar_wait(acc_full, n & 1, abort_p));
             if (!ok) break;
             tc_fence_after();
-            const bool store = key < p.N;
+            // Each thread holds half a row (D/2 columns) of dK and of dV.  Written straight from the registers a warp's store
+            // would touch 32 different lines; the warp passes its 32 x D bytes through shared memory (16-byte pieces, piece
+            // index xor row so that neither side has bank conflicts beyond the minimum) and stores whole lines instead.
+            constexpr int kPieces = D / 16;                    // 16-byte pieces per half row
+            constexpr int kRowsPerStore = 32 / kPieces;
+            uint8_t* stage = smem + C::kOffStage + warp * (32 * D);
+            const int key_warp = t * kTileN + (warp & 3) * 32;     // key of lane 0
 #pragma unroll
             for (int which = 0; which < 2; ++which) {
                 const uint32_t tA = tmem_base + lane_addr + (which == 0 ? C::kColDK : C::kColDV) + wg * (D / 2);
                 const float f = which == 0 ? p.scale : 1.f;
-                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(which == 0 ? p.dk : p.dv) +
-                                     ((long long)bh * p.N + key) * D + wg * (D / 2);
 #pragma unroll
                 for (int c = 0; c < D / 64; ++c) {
                     uint32_t o[32];
                     tmem_ld32(tA + c * 32, o);
-                    if (store) {
 #pragma unroll
-                        for (int v4 = 0; v4 < 4; ++v4) {
-                            uint4 w;
-                            w.x = pack_bf16x2(__uint_as_float(o[v4 * 8 + 0]) * f, __uint_as_float(o[v4 * 8 + 1]) * f);
-                            w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * f, __uint_as_float(o[v4 * 8 + 3]) * f);
-                            w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * f, __uint_as_float(o[v4 * 8 + 5]) * f);
-                            w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * f, __uint_as_float(o[v4 * 8 + 7]) * f);
-                            *reinterpret_cast<uint4*>(dst + c * 32 + v4 * 8) = w;
-                        }
+                    for (int v4 = 0; v4 < 4; ++v4) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(o[v4 * 8 + 0]) * f, __uint_as_float(o[v4 * 8 + 1]) * f);
+                        w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * f, __uint_as_float(o[v4 * 8 + 3]) * f);
+                        w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * f, __uint_as_float(o[v4 * 8 + 5]) * f);
+                        w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * f, __uint_as_float(o[v4 * 8 + 7]) * f);
+                        const int piece = c * 4 + v4;
+                        *reinterpret_cast<uint4*>(stage + lane * D + ((piece ^ (lane & (kPieces - 1))) << 4)) = w;
                     }
                 }
+                __syncwarp();
+                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(which == 0 ? p.dk : p.dv) +
+                                     ((long long)bh * p.N + key_warp) * D + wg * (D / 2);
+#pragma unroll
+                for (int it = 0; it < 32 / kRowsPerStore; ++it) {
+                    const int rrow = it * kRowsPerStore + lane / kPieces, piece = lane % kPieces;
+                    const uint4 w = *reinterpret_cast<const uint4*>(stage + rrow * D + ((piece ^ (rrow & (kPieces - 1))) << 4));
+                    if (key_warp + rrow < p.N) *reinterpret_cast<uint4*>(dst + (long long)rrow * D + piece * 8) = w;
+                }
+                __syncwarp();
             }
             tc_fence_before();
             mbar_arrive(acc_empty);
