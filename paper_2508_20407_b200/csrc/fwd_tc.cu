@@ -67,10 +67,11 @@ template <int D>
 struct Cfg {
     static constexpr int kTileBytes = kQTile * D * 2;          // one 128-row tile of Q, K or V
     static constexpr int kBoxes = D / 64;                      // 64-element (128-byte) column blocks per tile
-    static constexpr int kSlots = D == 128 ? 5 : 8;            // K/V ring slots
+    static constexpr int kSlots = D == 128 ? 4 : 8;            // K/V ring slots
     static constexpr int kSmemTiles = (2 + kSlots) * kTileBytes;
+    static constexpr int kStageBytes = 8 * 32 * 128;           // per softmax warp 32 rows x 128 bytes: result rows on their way out
     static constexpr int kNumBars = 10 + 2 * kSlots;
-    static constexpr int kSmemBytes = kSmemTiles + kNumBars * 8 + 16 + 1024;   // + alignment slack
+    static constexpr int kSmemBytes = kSmemTiles + kStageBytes + kNumBars * 8 + 16 + 1024;   // + alignment slack
     // TMEM columns: S0, S1 (128 each), O0, O1 (D each)
     static constexpr uint32_t kColS = 0, kColO = 256;
 };
@@ -96,7 +97,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sQ = smem;                               // 2 tiles
     uint8_t* sRing = smem + 2 * C::kTileBytes;        // kSlots tiles
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kSmemTiles);
+    uint8_t* sStage = smem + C::kSmemTiles;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kSmemTiles + C::kStageBytes);
     uint64_t* q_full = bars + 0;
     uint64_t* q_empty = bars + 1;
     uint64_t* s_full = bars + 2;      // [2]
@@ -423,22 +425,27 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             const float inv_l = l > 0.f ? 1.f / l : 0.f;
             const float lse_val = l > 0.f ? (m_ref + log2f(l)) * kLn2 : -CUDART_INF_F;
             const bool store = row < p.W;
-            __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + ((long long)s.bh * p.W + row) * D;
             // partial result -> workspace slot (0: first segment of this CTA's range, 1: a later one)
             float* pbase = p.ws + ((long long)blockIdx.x * 2 + (s.bh == bh_first ? 0 : 1)) * (long long)kTileM * (D + 1);
-            float* prow = pbase + (long long)(i * kQTile + r) * D;
+            // A thread holds one row.  Stored straight from the registers a warp's store would touch 32 different lines, so
+            // the warp passes its rows through shared memory 128 bytes at a time (16-byte pieces, piece index xor row: no
+            // bank conflicts beyond the minimum on either side) and every store instruction writes four whole lines.
+            uint8_t* stage = sStage + warp * (32 * 128);
+            const int row_warp = row - lane;                   // row of lane 0
+            if (whole) {
+                __nv_bfloat16* owarp = reinterpret_cast<__nv_bfloat16*>(p.out) + ((long long)s.bh * p.W + row_warp) * D;
 #pragma unroll
-            for (int c = 0; c < D / 16; ++c) {
-                uint32_t o[16];
-                if (cnt_i > 0) {
-                    tmem_ld16_async(tO + c * 16, o);
-                    tmem_wait_ld16(o);
-                } else {
+                for (int h = 0; h < D / 64; ++h) {             // 64 bf16 columns per pass
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) o[e] = 0u;
-                }
-                if (whole) {
-                    if (store) {
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t o[16];
+                        if (cnt_i > 0) {
+                            tmem_ld16_async(tO + h * 64 + c * 16, o);
+                            tmem_wait_ld16(o);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) o[e] = 0u;
+                        }
 #pragma unroll
                         for (int v4 = 0; v4 < 2; ++v4) {
                             uint4 w;
@@ -446,19 +453,50 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                             w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * inv_l, __uint_as_float(o[v4 * 8 + 3]) * inv_l);
                             w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * inv_l, __uint_as_float(o[v4 * 8 + 5]) * inv_l);
                             w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * inv_l, __uint_as_float(o[v4 * 8 + 7]) * inv_l);
-                            *reinterpret_cast<uint4*>(orow + c * 16 + v4 * 8) = w;
+                            *reinterpret_cast<uint4*>(stage + lane * 128 + (((c * 2 + v4) ^ (lane & 7)) << 4)) = w;
                         }
                     }
-                } else {
+                    __syncwarp();
 #pragma unroll
-                    for (int v4 = 0; v4 < 4; ++v4) {
-                        float4 w;
-                        w.x = __uint_as_float(o[v4 * 4 + 0]) * inv_l;
-                        w.y = __uint_as_float(o[v4 * 4 + 1]) * inv_l;
-                        w.z = __uint_as_float(o[v4 * 4 + 2]) * inv_l;
-                        w.w = __uint_as_float(o[v4 * 4 + 3]) * inv_l;
-                        *reinterpret_cast<float4*>(prow + c * 16 + v4 * 4) = w;
+                    for (int it = 0; it < 8; ++it) {
+                        const int rrow = it * 4 + (lane >> 3), piece = lane & 7;
+                        const uint4 w = *reinterpret_cast<const uint4*>(stage + rrow * 128 + ((piece ^ (rrow & 7)) << 4));
+                        if (row_warp + rrow < p.W) *reinterpret_cast<uint4*>(owarp + (long long)rrow * D + h * 64 + piece * 8) = w;
                     }
+                    __syncwarp();
+                }
+            } else {
+                float* pwarp = pbase + (long long)(i * kQTile + (warp & 3) * 32) * D;
+#pragma unroll
+                for (int h = 0; h < D / 32; ++h) {             // 32 fp32 columns per pass
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t o[16];
+                        if (cnt_i > 0) {
+                            tmem_ld16_async(tO + h * 32 + c * 16, o);
+                            tmem_wait_ld16(o);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) o[e] = 0u;
+                        }
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            float4 w;
+                            w.x = __uint_as_float(o[v4 * 4 + 0]) * inv_l;
+                            w.y = __uint_as_float(o[v4 * 4 + 1]) * inv_l;
+                            w.z = __uint_as_float(o[v4 * 4 + 2]) * inv_l;
+                            w.w = __uint_as_float(o[v4 * 4 + 3]) * inv_l;
+                            *reinterpret_cast<float4*>(stage + lane * 128 + (((c * 4 + v4) ^ (lane & 7)) << 4)) = w;
+                        }
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
+                        const int rrow = it * 4 + (lane >> 3), piece = lane & 7;
+                        const float4 w = *reinterpret_cast<const float4*>(stage + rrow * 128 + ((piece ^ (rrow & 7)) << 4));
+                        *reinterpret_cast<float4*>(pwarp + (long long)rrow * D + h * 32 + piece * 4) = w;
+                    }
+                    __syncwarp();
                 }
             }
             if (whole) {
