@@ -188,7 +188,8 @@ L2_BYTES = 126e6
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from one-pass ncu captures of these
 # very workloads.  To be set to None whenever the kernel changes.
-FWD_TRAFFIC = {}
+FWD_TRAFFIC = {"cfg4_vlong": (2177.07e6 + 19.71e6, "ncu, full workload, fwd_tc_kernel<128>"),
+               "cfg3_long": (544.86e6 + 10.74e6, "ncu, full workload, fwd_tc_kernel<128>")}
 # decode: captured on a smaller cache (B8 H32, 4096 rows: 537.35 MB read + 3.9 MB written for 537.3 MB of cache) and
 # scaled by the cached rows of the timed steps; the kernel streams every cached byte once at any size
 DECODE_TRAFFIC_RATIO = (537.35 + 3.9) / 537.3
