@@ -38,6 +38,11 @@ def _load():
         lib.tlin_ref_attn_backward.argtypes = [vp, vp, vp, vp, i32, dp, dp, dp, i32, i32, i64, i64, i32, i32]
         lib.tlin_ref_decode_step.argtypes = [vp, vp, vp, vp, vp, i32, dp, dp, i32, i32, i64, i64, i32]
         lib.tlin_ref_merge_lse.argtypes = [dp, dp, dp, dp, dp, dp, i64, i32]
+        lib.tlin_ref_decode_step_fp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, dp, i32, i32, i64, i64, i32]
+        lib.tlin_ref_e4m3_decode.argtypes = [ctypes.c_uint8]
+        lib.tlin_ref_e4m3_decode.restype = ctypes.c_double
+        lib.tlin_ref_e4m3_encode.argtypes = [ctypes.c_float]
+        lib.tlin_ref_e4m3_encode.restype = ctypes.c_uint8
         lib.tlin_ref_allowed.argtypes = [i64, i64, i64, i64, i32]
         lib.tlin_ref_num_threads.argtypes = []
         _lib = lib
@@ -149,6 +154,49 @@ def decode_step(q_new, k_new, v_new, k_cache, v_cache, pos: int):
                                       _ptr(out), _ptr(lse), B, H, Ncap, int(pos), d)
     if rc != 0:
         raise ValueError(f"tlin_ref_decode_step rejected its arguments (rc={rc})")
+    return out, lse
+
+
+def e4m3_decode(code: int) -> float:
+    """Value of an E4M3 code (0..255); NaN for 0x7f and 0xff."""
+    return float(_load().tlin_ref_e4m3_decode(int(code) & 0xFF))
+
+
+def e4m3_encode(x: float) -> int:
+    """Nearest finite E4M3 code of an fp32 value (ties to even, saturating at +-448)."""
+    return int(_load().tlin_ref_e4m3_encode(float(np.float32(x))))
+
+
+def decode_step_fp8(q_new, k_new, v_new, k_cache, v_cache, k_scale, v_scale, pos: int):
+    """Cached decode step over an 8-bit (E4M3) cache; value = decode(code) * scale[b,h].
+
+    q_new,k_new,v_new: bf16 [B,H,1,d]; k_cache,v_cache: uint8 [B,H,Ncap,d], updated in place at row ``pos``;
+    k_scale,v_scale: float32 [B,H].  Returns (out f64 [B,H,1,d], lse f64 [B,H])."""
+    qa, tq = _as_elems(q_new)
+    kn, tk = _as_elems(k_new)
+    vn, tv = _as_elems(v_new)
+    if not (tq == tk == tv == BF16):
+        raise TypeError("q_new, k_new, v_new must be bf16")
+
+    def bytes_of(c):
+        if hasattr(c, "detach"):
+            if not c.is_contiguous():
+                raise ValueError("caches must be contiguous to be updated in place")
+            c = c.numpy()
+        if c.dtype != np.uint8 or not c.flags["C_CONTIGUOUS"]:
+            raise TypeError("caches are contiguous uint8 arrays")
+        return c
+
+    kc, vc = bytes_of(k_cache), bytes_of(v_cache)
+    ks = np.ascontiguousarray(k_scale.numpy() if hasattr(k_scale, "detach") else k_scale, dtype=np.float32)
+    vs = np.ascontiguousarray(v_scale.numpy() if hasattr(v_scale, "detach") else v_scale, dtype=np.float32)
+    B, H, Ncap, d = kc.shape
+    out = np.empty((B, H, 1, d), dtype=np.float64)
+    lse = np.empty((B, H), dtype=np.float64)
+    rc = _load().tlin_ref_decode_step_fp8(_ptr(qa), _ptr(kn), _ptr(vn), _ptr(kc), _ptr(vc), _ptr(ks), _ptr(vs),
+                                          _ptr(out), _ptr(lse), B, H, Ncap, int(pos), d)
+    if rc != 0:
+        raise ValueError(f"tlin_ref_decode_step_fp8 rejected its arguments (rc={rc})")
     return out, lse
 
 

@@ -42,7 +42,7 @@
 #include <omp.h>
 #endif
 
-enum { TLIN_REF_BF16 = 0, TLIN_REF_F32 = 1 };
+enum { TLIN_REF_BF16 = 0, TLIN_REF_F32 = 1, TLIN_REF_F64 = 2 /* internal: values already widened */ };
 
 static double widen(const void *base, int elem_type, int64_t idx)
 {
@@ -52,6 +52,7 @@ static double widen(const void *base, int elem_type, int64_t idx)
         memcpy(&f, &bits, sizeof f);
         return (double)f;
     }
+    if (elem_type == TLIN_REF_F64) return ((const double *)base)[idx];
     return (double)((const float *)base)[idx];
 }
 
@@ -174,6 +175,86 @@ int tlin_ref_decode_step(const void *q_new, const void *k_new, const void *v_new
             attend_row(q_new, kc, vc, elem_type, bh * d, 0, 0, L, 1, d, 0, scores, out + bh * d, lse + bh);
         }
         free(scores);
+    }
+    return failed ? -2 : 0;
+}
+
+/*
+ * 8-bit floating point, E4M3 (the "FN" variant of the OCP 8-bit floating point
+ * specification): 1 sign bit, 4 exponent bits with bias 7, 3 mantissa bits; no
+ * infinities; S.1111.111 is NaN; the largest finite value is S.1111.110 = 448;
+ * exponent field 0 holds the subnormals m * 2^-9.  Not in the paper: it is the
+ * storage format of the optional 8-bit key/value cache.
+ */
+double tlin_ref_e4m3_decode(uint8_t code)
+{
+    const int sign = code >> 7, e = (code >> 3) & 15, m = code & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m, -9);
+    else v = ldexp(1.0 + m / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
+/* Nearest finite code, ties to the code with an even mantissa, magnitudes beyond 448 saturate; NaN -> 0x7f. */
+uint8_t tlin_ref_e4m3_encode(float x)
+{
+    if (x != x) return 0x7f;
+    const uint8_t sign = signbit(x) ? 0x80 : 0x00;
+    const double a = fabs((double)x);
+    int best = 0;
+    double best_err = INFINITY;
+    for (int c = 0; c <= 0x7e; ++c) {          /* the 127 finite non-negative codes, in increasing order of value */
+        const double err = fabs(tlin_ref_e4m3_decode((uint8_t)c) - a);
+        if (err < best_err || (err == best_err && (c & 1) == 0)) { best_err = err; best = c; }
+    }
+    return (uint8_t)(sign | best);
+}
+
+/*
+ * The cached decode step over an 8-bit cache.  k_cache,v_cache:[B,H,Ncap,d] bytes (E4M3 codes); the value of
+ * an element is decode(code) * scale, with one fp32 scale per (b,h) for keys and one for values.  The new key
+ * and value rows (bf16) are stored as encode(x / scale), the division carried out in fp32 (the precision in
+ * which the kernel takes the same decision); the new query (bf16) then attends to the decoded rows [0, pos],
+ * its own included.  out:[B,H,1,d], lse:[B,H].
+ */
+int tlin_ref_decode_step_fp8(const uint16_t *q_new, const uint16_t *k_new, const uint16_t *v_new,
+                             uint8_t *k_cache, uint8_t *v_cache, const float *k_scale, const float *v_scale,
+                             double *out, double *lse, int B, int H, int64_t Ncap, int64_t pos, int d)
+{
+    if (!q_new || !k_new || !v_new || !k_cache || !v_cache || !k_scale || !v_scale || !out || !lse) return -1;
+    if (B <= 0 || H <= 0 || d <= 0 || Ncap <= 0 || pos < 0 || pos >= Ncap) return -1;
+    const int64_t L = pos + 1;
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *scores = (double *)malloc((size_t)L * sizeof(double));
+        double *kd = (double *)malloc((size_t)L * d * sizeof(double));
+        double *vd = (double *)malloc((size_t)L * d * sizeof(double));
+        double *qd = (double *)malloc((size_t)d * sizeof(double));
+        if (!scores || !kd || !vd || !qd) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t bh = 0; bh < (int64_t)B * H; ++bh) {
+            if (!scores || !kd || !vd || !qd) continue;
+            uint8_t *kc = k_cache + (size_t)(bh * Ncap) * d, *vc = v_cache + (size_t)(bh * Ncap) * d;
+            for (int c = 0; c < d; ++c) {
+                const float kx = (float)widen(k_new, TLIN_REF_BF16, bh * d + c) / k_scale[bh];
+                const float vx = (float)widen(v_new, TLIN_REF_BF16, bh * d + c) / v_scale[bh];
+                kc[(size_t)pos * d + c] = tlin_ref_e4m3_encode(kx);
+                vc[(size_t)pos * d + c] = tlin_ref_e4m3_encode(vx);
+                qd[c] = widen(q_new, TLIN_REF_BF16, bh * d + c);
+            }
+            for (int64_t j = 0; j < L; ++j)
+                for (int c = 0; c < d; ++c) {
+                    kd[j * d + c] = tlin_ref_e4m3_decode(kc[(size_t)j * d + c]) * (double)k_scale[bh];
+                    vd[j * d + c] = tlin_ref_e4m3_decode(vc[(size_t)j * d + c]) * (double)v_scale[bh];
+                }
+            attend_row(qd, kd, vd, TLIN_REF_F64, 0, 0, 0, L, 1, d, 0, scores, out + bh * d, lse + bh);
+        }
+        free(scores); free(kd); free(vd); free(qd);
     }
     return failed ? -2 : 0;
 }

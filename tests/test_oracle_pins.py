@@ -448,3 +448,57 @@ def test_backward_respects_the_causal_window():
     assert (dk[0, 0, N - W + 1:] == 0).all() and (dv[0, 0, N - W + 1:] == 0).all()
     assert (dq[0, 0, 1:] == 0).all() and np.abs(dq[0, 0, 0]).max() > 0
     assert np.abs(dv[0, 0, :N - W + 1]).min() > 0
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# 8-bit (E4M3) key/value cache: the codec against the published format and a library conversion, the decode step
+# against a probability matrix written out in numpy over values dequantised by the library conversion.
+def test_e4m3_decode_table_matches_the_format_and_the_library_view():
+    assert oracle.e4m3_decode(0x00) == 0.0 and oracle.e4m3_decode(0x38) == 1.0 and oracle.e4m3_decode(0x40) == 2.0
+    assert oracle.e4m3_decode(0x7E) == 448.0 and oracle.e4m3_decode(0x01) == 2.0 ** -9 and oracle.e4m3_decode(0x08) == 2.0 ** -6
+    assert oracle.e4m3_decode(0xC0) == -2.0 and np.isnan(oracle.e4m3_decode(0x7F)) and np.isnan(oracle.e4m3_decode(0xFF))
+    mine = np.array([oracle.e4m3_decode(c) for c in range(256)])
+    assert np.all(np.diff(mine[:0x7F]) > 0)                       # codes order the non-negative values
+    lib = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).float().numpy()
+    assert np.all((mine == lib) | (np.isnan(mine) & np.isnan(lib)))
+
+
+def test_e4m3_encode_rounds_to_nearest_even_and_saturates():
+    for c in list(range(0x7F)) + list(range(0x80, 0xFF)):
+        assert oracle.e4m3_encode(oracle.e4m3_decode(c)) == c      # every finite code is a fixed point (signed zero too)
+    assert oracle.e4m3_encode(1.0625) == 0x38 and oracle.e4m3_encode(1.1875) == 0x3A       # ties go to the even mantissa
+    assert oracle.e4m3_encode(2.0 ** -10) == 0x00 and oracle.e4m3_encode(3 * 2.0 ** -10) == 0x02   # ties among subnormals
+    assert oracle.e4m3_encode(449.0) == 0x7E and oracle.e4m3_encode(1e30) == 0x7E and oracle.e4m3_encode(-1e30) == 0xFE
+    assert oracle.e4m3_encode(float("nan")) == 0x7F
+    g = torch.Generator().manual_seed(0)
+    x = torch.cat([torch.randn(20000, generator=g) * s for s in (1e-3, 0.1, 3.0, 100.0)])
+    x = x[x.abs() <= 448.0]                                        # the library conversion does not saturate beyond
+    lib = x.to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    mine = np.array([oracle.e4m3_encode(float(v)) for v in x.numpy()], dtype=np.uint8)
+    assert np.array_equal(lib, mine)
+
+
+def test_fp8_decode_step_against_numpy_over_library_dequantised_values():
+    B, H, Ncap, d, pos = 2, 3, 20, 16, 11
+    g = torch.Generator().manual_seed(5)
+    k_scale = (torch.rand(B, H, generator=g) * 0.05 + 0.01).float()
+    v_scale = (torch.rand(B, H, generator=g) * 0.05 + 0.01).float()
+    kc = (torch.randn(B, H, Ncap, d, generator=g) / k_scale[:, :, None, None]).to(torch.float8_e4m3fn).view(torch.uint8).contiguous()
+    vc = (torch.randn(B, H, Ncap, d, generator=g) / v_scale[:, :, None, None]).to(torch.float8_e4m3fn).view(torch.uint8).contiguous()
+    q, kn, vn = (torch.randn(B, H, 1, d, generator=g).to(torch.bfloat16) for _ in range(3))
+    kc0, vc0 = kc.clone(), vc.clone()
+    out, lse = oracle.decode_step_fp8(q, kn, vn, kc, vc, k_scale, v_scale, pos)
+    # the appended row: fp32 division, then the library's conversion; nothing else changed
+    want_k = (kn.float() / k_scale[:, :, None, None]).to(torch.float8_e4m3fn).view(torch.uint8)[:, :, 0]
+    want_v = (vn.float() / v_scale[:, :, None, None]).to(torch.float8_e4m3fn).view(torch.uint8)[:, :, 0]
+    assert torch.equal(kc[:, :, pos], want_k) and torch.equal(vc[:, :, pos], want_v)
+    keep = [j for j in range(Ncap) if j != pos]
+    assert torch.equal(kc[:, :, keep], kc0[:, :, keep]) and torch.equal(vc[:, :, keep], vc0[:, :, keep])
+    # attention over the dequantised rows [0, pos], written out
+    kd = kc.view(torch.float8_e4m3fn).double().numpy() * k_scale.double().numpy()[:, :, None, None]
+    vd = vc.view(torch.float8_e4m3fn).double().numpy() * v_scale.double().numpy()[:, :, None, None]
+    s = np.einsum("bhqc,bhjc->bhqj", q.double().numpy(), kd[:, :, :pos + 1]) / np.sqrt(d)
+    p = np.exp(s - s.max(-1, keepdims=True))
+    want = np.einsum("bhqj,bhjc->bhqc", p / p.sum(-1, keepdims=True), vd[:, :, :pos + 1])
+    assert np.abs(out - want).max() < 1e-12
+    assert np.abs(lse - (np.log(p.sum(-1)) + s.max(-1))[:, :, 0]).max() < 1e-12
