@@ -113,6 +113,18 @@ int tlin_decode_step_ragged(const void* q_new, const void* k_new, const void* v_
                             void* k_cache, void* v_cache, void* out, float* lse,
                             int B, int H, int Ncap, const int32_t* pos, int max_pos, int d, tlin_stream_t stream);
 
+/* tlin_decode_step over an 8-bit cache (not in the paper; it halves the cache memory of Section 5.2 and the bytes a step
+ * streams).  k_cache, v_cache [B,H,Ncap,d] hold one byte per element: E4M3 codes of the 8-bit floating point format
+ * (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest finite value 448); the value of an element
+ * is decode(code) * scale, with k_scale, v_scale [B*H] fp32 in DEVICE memory (one scale per (b,h), chosen by the caller,
+ * positive and finite).  q_new, k_new, v_new, out are bf16 as in tlin_decode_step.  The new rows are stored at row `pos` as
+ * encode(x / scale): fp32 division, round to nearest with ties to the even code, magnitudes beyond 448 saturate.  The new
+ * query then attends to the decoded rows [0, pos], its own included.  d in {64,128}; workspace and errors as for
+ * tlin_decode_step. */
+int tlin_decode_step_fp8(const void* q_new, const void* k_new, const void* v_new,
+                         void* k_cache, void* v_cache, const float* k_scale, const float* v_scale,
+                         void* out, float* lse, int B, int H, int Ncap, int pos, int d, tlin_stream_t stream);
+
 /* tlin_decode_step with HOST q/k/v_new and out/lse (the caches stay on the device).  *_d are
  * DEVICE staging buffers ([B,H,1,d] each, lse_d [B,H]). */
 int tlin_decode_step_host(const void* q_new_h, const void* k_new_h, const void* v_new_h, void* out_h, float* lse_h,

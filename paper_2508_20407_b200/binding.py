@@ -51,6 +51,7 @@ SIGNATURES = {
     "tlin_decode_step_host": (_i, [_vp] * 12 + [_i] * 5 + [_vp]),
     "tlin_decode_step_static": (_i, [_vp] * 7 + [_i] * 5 + [_vp]),
     "tlin_decode_step_ragged": (_i, [_vp] * 7 + [_i] * 3 + [_vp, _i, _i, _vp]),
+    "tlin_decode_step_fp8": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
     "tlin_merge_lse": (_i, [_vp] * 6 + [_i64, _i, _vp]),
     "tlin_merge_lse_f32": (_i, [_vp] * 6 + [_i64, _i, _vp]),
     "tlin_workspace_bytes_forward": (_sz, [_i] * 6),
@@ -274,6 +275,27 @@ def tlin_decode_step(q_new, k_new, v_new, k_cache, v_cache, pos, out=None, lse=N
     ensure_workspace(workspace_bytes_decode(B, H, Ncap, d), q_new.device)
     _check(lib().tlin_decode_step(_ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache),
                                   _ptr(out), _ptr(lse), B, H, Ncap, int(pos), d, _stream(stream)), "tlin_decode_step")
+    return out, lse
+
+
+def tlin_decode_step_fp8(q_new, k_new, v_new, k_cache, v_cache, k_scale, v_scale, pos, out=None, lse=None, stream=None):
+    """Decode step over an 8-bit cache: k_cache, v_cache are uint8 [B,H,Ncap,d] (E4M3 codes), value = code * scale[b,h];
+    k_scale, v_scale fp32 device tensors [B,H]."""
+    B, H, Ncap, d = k_cache.shape
+    for t, n in ((q_new, "q_new"), (k_new, "k_new"), (v_new, "v_new")):
+        _dev(t, torch.bfloat16, (B, H, 1, d), n)
+    _dev(k_cache, torch.uint8, (B, H, Ncap, d), "k_cache")
+    _dev(v_cache, torch.uint8, (B, H, Ncap, d), "v_cache")
+    _dev(k_scale, torch.float32, (B, H), "k_scale")
+    _dev(v_scale, torch.float32, (B, H), "v_scale")
+    if out is None:
+        out = torch.empty_like(q_new)
+    if lse is None:
+        lse = torch.empty((B, H), dtype=torch.float32, device=q_new.device)
+    ensure_workspace(workspace_bytes_decode(B, H, Ncap, d), q_new.device)
+    _check(lib().tlin_decode_step_fp8(_ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(k_scale),
+                                      _ptr(v_scale), _ptr(out), _ptr(lse), B, H, Ncap, int(pos), d, _stream(stream)),
+           "tlin_decode_step_fp8")
     return out, lse
 
 

@@ -216,6 +216,29 @@ extern "C" int tlin_decode_step(const void* q_new, const void* k_new, const void
                          (float*)w.ptr, (cudaStream_t)stream);
 }
 
+extern "C" int tlin_decode_step_fp8(const void* q_new, const void* k_new, const void* v_new,
+                                    void* k_cache, void* v_cache, const float* k_scale, const float* v_scale,
+                                    void* out, float* lse, int B, int H, int Ncap, int pos, int d, tlin_stream_t stream) {
+    t_launches = 0;
+    if (!q_new || !k_new || !v_new || !k_cache || !v_cache || !k_scale || !v_scale || !out) return TLIN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || Ncap <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    if (pos < 0 || pos >= Ncap) return TLIN_ERR_INVALID_ARG;
+    if (!aligned16(q_new) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) ||
+        !aligned16(v_cache) || !aligned16(out) || (reinterpret_cast<uintptr_t>(k_scale) & 3u) ||
+        (reinterpret_cast<uintptr_t>(v_scale) & 3u)) return TLIN_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return TLIN_ERR_UNSUPPORTED;
+    int sms = 0;
+    int rc = device_info(&sms);
+    if (rc != TLIN_OK) return rc;
+    tlin_decode_plan plan;
+    rc = tlin_plan_decode(B, H, pos + 1, d, sms, &plan);
+    if (rc != TLIN_OK) return rc;
+    const Workspace w = workspace();
+    if (!w.ptr || w.bytes < (size_t)plan.workspace_bytes) return TLIN_ERR_WORKSPACE;
+    return launch_decode_fp8(q_new, k_new, v_new, k_cache, v_cache, k_scale, v_scale, out, lse, B, H, Ncap, pos, d, plan,
+                             (float*)w.ptr, (cudaStream_t)stream);
+}
+
 extern "C" int tlin_decode_step_ragged(const void* q_new, const void* k_new, const void* v_new,
                                        void* k_cache, void* v_cache, void* out, float* lse,
                                        int B, int H, int Ncap, const int32_t* pos, int max_pos, int d, tlin_stream_t stream) {

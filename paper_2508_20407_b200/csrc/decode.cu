@@ -9,6 +9,7 @@
 // they are combined at the end; the CTA writes one normalised partial (o, lse) to the workspace and
 // a second kernel merges the splits (log-sum-exp weights).
 #include "tlin_internal.h"
+#include <cuda_fp16.h>
 #include <math_constants.h>
 #include <mutex>
 
@@ -215,6 +216,178 @@ decode_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ 
     if (lse != nullptr && c == 0) lse[bh] = mm + logf(z);
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// The same step over an 8-bit cache (E4M3 codes, value = decode(code) * scale[b,h]; not in the paper: it halves the
+// bytes the step streams and the memory Section 5.2 accounts for).  A lane owns 16 columns of a row: one 16-byte load
+// each for K and V, codes widened in pairs by cvt.rn.f16x2.e4m3x2 (exact).  The key scale is folded into q, the value
+// scale into the final normalisation.  The new row is stored as encode(x / scale) (fp32 division, round to nearest
+// even, saturating) and every lane that meets it takes the same codes from k_new / v_new instead of the cache.
+__device__ __forceinline__ float2 e4m3x2_to_f32x2(uint32_t two_codes) {      // low byte -> x, next byte -> y
+    uint32_t h2;
+    asm("{\n\t.reg .b16 c;\n\tcvt.u16.u32 c, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, c;\n\t}" : "=r"(h2) : "r"(two_codes));
+    return __half22float2(*reinterpret_cast<const __half2*>(&h2));
+}
+__device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {     // lo -> low byte, hi -> next byte
+    uint32_t r;
+    asm("{\n\t.reg .b16 c;\n\tcvt.rn.satfinite.e4m3x2.f32 c, %1, %2;\n\tcvt.u32.u16 %0, c;\n\t}" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ void widen16(const uint4& c, float (&x)[16]) {
+    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 a = e4m3x2_to_f32x2(w[i] & 0xffffu), b = e4m3x2_to_f32x2(w[i] >> 16);
+        x[4 * i + 0] = a.x; x[4 * i + 1] = a.y; x[4 * i + 2] = b.x; x[4 * i + 3] = b.y;
+    }
+}
+// 16 bf16 values (two 16-byte words) divided by `scale` and encoded
+__device__ __forceinline__ uint4 quantise16(const uint4& lo8, const uint4& hi8, float scale) {
+    const uint32_t w[8] = {lo8.x, lo8.y, lo8.z, lo8.w, hi8.x, hi8.y, hi8.z, hi8.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t a = f32x2_to_e4m3x2(__fdiv_rn(bf_lo(w[2 * i]), scale), __fdiv_rn(bf_hi(w[2 * i]), scale));
+        const uint32_t b = f32x2_to_e4m3x2(__fdiv_rn(bf_lo(w[2 * i + 1]), scale), __fdiv_rn(bf_hi(w[2 * i + 1]), scale));
+        o[i] = a | (b << 16);
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kWarps * 32, kDecodeCtasPerSM)
+decode_fp8_splitk_kernel(const uint4* __restrict__ q_new, const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+                         uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
+                         const float* __restrict__ k_scale, const float* __restrict__ v_scale,
+                         float* __restrict__ part_o, float* __restrict__ part_lse,
+                         int Ncap, int pos, int splits, int kps, float scale_log2e) {
+    constexpr int LPR = D / 16;          // lanes (16-byte chunks of codes) per row
+    constexpr int RPW = 32 / LPR;        // rows per warp-load
+    constexpr int ROWS_PER_IT = kWarps * RPW * kUnroll;
+    const int bh = blockIdx.x / splits, sp = blockIdx.x - bh * splits;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane % LPR, rsel = lane / LPR;
+    const int L = pos + 1;
+    const int j0 = sp * kps, j1 = min(L, j0 + kps);
+    const float ks = k_scale[bh], vs = v_scale[bh];
+
+    const uint4* kc = k_cache + (int64_t)bh * Ncap * LPR;
+    const uint4* vc = v_cache + (int64_t)bh * Ncap * LPR;
+    // the new row's codes for this lane's 16 columns (bf16: two 16-byte words per lane)
+    const uint4 kn_codes = quantise16(k_new[(int64_t)bh * (D / 8) + 2 * sub], k_new[(int64_t)bh * (D / 8) + 2 * sub + 1], ks);
+    const uint4 vn_codes = quantise16(v_new[(int64_t)bh * (D / 8) + 2 * sub], v_new[(int64_t)bh * (D / 8) + 2 * sub + 1], vs);
+    // append by the CTA whose range holds row `pos`; nobody reads that row from the cache in this launch
+    if (pos >= j0 && pos < j1 && warp == 0 && lane < LPR) {
+        k_cache[((int64_t)bh * Ncap + pos) * LPR + lane] = kn_codes;
+        v_cache[((int64_t)bh * Ncap + pos) * LPR + lane] = vn_codes;
+    }
+
+    float qf[16];
+    {
+        const uint4 q0 = q_new[(int64_t)bh * (D / 8) + 2 * sub], q1 = q_new[(int64_t)bh * (D / 8) + 2 * sub + 1];
+        const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+        const float f = scale_log2e * ks;                 // the key scale rides on q
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            qf[2 * i] = bf_lo(w[i]) * f;
+            qf[2 * i + 1] = bf_hi(w[i]) * f;
+        }
+    }
+
+    float m = -CUDART_INF_F, l = 0.f;
+    float acc[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+
+    for (int base = j0; base < j1; base += ROWS_PER_IT) {
+        uint4 kv[kUnroll], vv[kUnroll];
+        bool ok[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int j = base + (u * kWarps + warp) * RPW + rsel;
+            ok[u] = j < j1;
+            kv[u] = make_uint4(0, 0, 0, 0);
+            vv[u] = make_uint4(0, 0, 0, 0);
+            if (ok[u]) {
+                if (j == pos) {
+                    kv[u] = kn_codes;
+                    vv[u] = vn_codes;
+                } else {
+                    kv[u] = ld_stream(kc + (int64_t)j * LPR + sub);
+                    vv[u] = ld_stream(vc + (int64_t)j * LPR + sub);
+                }
+            }
+        }
+        float s[kUnroll];
+        float mb = m;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            float kx[16];
+            widen16(kv[u], kx);
+            float x = 0.f;
+#pragma unroll
+            for (int e = 0; e < 16; ++e) x = fmaf(kx[e], qf[e], x);
+#pragma unroll
+            for (int o = LPR / 2; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+            s[u] = ok[u] ? x : -CUDART_INF_F;
+            mb = fmaxf(mb, s[u]);
+        }
+        const float ms = mb == -CUDART_INF_F ? 0.f : mb;
+        const float corr = exp2f(m - ms);
+        l *= corr;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) acc[e] *= corr;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const float pr = exp2f(s[u] - ms);
+            l += pr;
+            float vx[16];
+            widen16(vv[u], vx);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) acc[e] = fmaf(pr, vx[e], acc[e]);
+        }
+        m = mb;
+    }
+
+    // combine the row-groups of the warp
+#pragma unroll
+    for (int o = LPR; o < 32; o <<= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
+        const float l2 = __shfl_xor_sync(0xffffffffu, l, o);
+        const float mn = fmaxf(m, m2);
+        const float mz = mn == -CUDART_INF_F ? 0.f : mn;
+        const float c1 = exp2f(m - mz), c2 = exp2f(m2 - mz);
+        l = l * c1 + l2 * c2;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) acc[e] = acc[e] * c1 + __shfl_xor_sync(0xffffffffu, acc[e], o) * c2;
+        m = mn;
+    }
+    __shared__ float sm_m[kWarps], sm_l[kWarps];
+    __shared__ float sm_a[kWarps][D];
+    if (rsel == 0) {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) sm_a[warp][sub * 16 + e] = acc[e];
+        if (sub == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+    }
+    __syncthreads();
+    if (threadIdx.x < D) {
+        const int c = threadIdx.x;
+        float mm = -CUDART_INF_F;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) mm = fmaxf(mm, sm_m[w]);
+        const float ms = mm == -CUDART_INF_F ? 0.f : mm;
+        float ll = 0.f, a = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const float c1 = exp2f(sm_m[w] - ms);
+            ll += sm_l[w] * c1;
+            a += sm_a[w][c] * c1;
+        }
+        const int64_t slot = (int64_t)bh * splits + sp;
+        part_o[slot * D + c] = ll > 0.f ? a * vs / ll : 0.f;          // the value scale applied once per output element
+        if (c == 0) part_lse[slot] = ll > 0.f ? (mm + log2f(ll)) * kLn2 : -CUDART_INF_F;
+    }
+}
+
 template <int D>
 int launch_d(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
              void* out, float* lse, int B, int H, int Ncap, int pos, const int* pos_per_seq, const tlin_decode_plan& plan,
@@ -233,7 +406,33 @@ int launch_d(const void* q_new, const void* k_new, const void* v_new, void* k_ca
     return TLIN_OK;
 }
 
+template <int D>
+int launch_fp8_d(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                 const float* k_scale, const float* v_scale, void* out, float* lse, int B, int H, int Ncap, int pos,
+                 const tlin_decode_plan& plan, float* ws, cudaStream_t st) {
+    const int64_t bh = (int64_t)B * H;
+    float* part_o = ws;
+    float* part_lse = ws + bh * kDecodeMaxSplits * D;
+    const float scale_log2e = kLog2e / sqrtf((float)D);
+    decode_fp8_splitk_kernel<D><<<plan.n_ctas, kWarps * 32, 0, st>>>(
+        (const uint4*)q_new, (const uint4*)k_new, (const uint4*)v_new, (uint4*)k_cache, (uint4*)v_cache, k_scale, v_scale,
+        part_o, part_lse, Ncap, pos, plan.splits, plan.keys_per_split, scale_log2e);
+    TLIN_CUDA_CHECK(cudaGetLastError());
+    decode_merge_kernel<D><<<(unsigned)bh, D, 0, st>>>(part_o, part_lse, (__nv_bfloat16*)out, lse, plan.splits);
+    TLIN_CUDA_CHECK(cudaGetLastError());
+    count_launch(2);
+    return TLIN_OK;
+}
+
 }  // namespace
+
+int launch_decode_fp8(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                      const float* k_scale, const float* v_scale, void* out, float* lse, int B, int H, int Ncap, int pos,
+                      int d, const tlin_decode_plan& plan, float* ws, cudaStream_t st) {
+    if (d == 128) return launch_fp8_d<128>(q_new, k_new, v_new, k_cache, v_cache, k_scale, v_scale, out, lse, B, H, Ncap, pos, plan, ws, st);
+    if (d == 64) return launch_fp8_d<64>(q_new, k_new, v_new, k_cache, v_cache, k_scale, v_scale, out, lse, B, H, Ncap, pos, plan, ws, st);
+    return TLIN_ERR_UNSUPPORTED;
+}
 
 int launch_decode(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                   void* out, float* lse, int B, int H, int Ncap, int pos, const int* pos_per_seq, int d,

@@ -51,6 +51,9 @@ int launch_bwd_tc(const void* q, const void* k, const void* v, const void* out, 
                   void* dq, void* dk, void* dv, int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& plan,
                   float* ws, int num_sms, cudaStream_t st);
 size_t bwd_tc_workspace_bytes(long long B, long long H, long long W, int d, const tlin_fwd_plan& plan);
+int launch_decode_fp8(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                      const float* k_scale, const float* v_scale, void* out, float* lse, int B, int H, int Ncap, int pos,
+                      int d, const tlin_decode_plan& plan, float* ws, cudaStream_t st);
 int launch_merge_pair_bf16(const void* oa, const float* la, const void* ob, const float* lb,
                            void* out, float* lse, int64_t rows, int d, cudaStream_t st);
 int launch_merge_pair_f32(const float* oa, const float* la, const float* ob, const float* lb,

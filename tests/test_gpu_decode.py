@@ -192,3 +192,57 @@ def test_ragged_decode_loop_replays_from_a_cuda_graph():
     for t in range(total):
         assert torch.equal(got[t], ref_out[t]), f"step {t}"
     assert torch.equal(kc[:, :, :n0 + total], kc_ref[:, :, :n0 + total])
+
+
+def _fp8_cache(wl, pad):
+    """Quantises the seeded bf16 cache of `wl` to E4M3 codes on the host (library conversion, pinned against the oracle's
+    codec on the CPU side), one scale per (b,h) such that the largest magnitude maps to 224."""
+    (kc, vc), (qn, kn, vn) = synth.decode_inputs(wl, device="cpu")
+    B, H, d = wl.B, wl.H, wl.d
+    def scales(x):
+        amax = x.float().abs().amax(dim=(2, 3)) if x.shape[2] > 0 else torch.ones(B, H)
+        return (torch.clamp(amax, min=1e-3) / 224.0).float().contiguous()
+    ks, vs = scales(torch.cat([kc, kn.transpose(0, 2).reshape(B, H, -1, d)], 2)), scales(torch.cat([vc, vn.transpose(0, 2).reshape(B, H, -1, d)], 2))
+    def codes(x, s):
+        c = (x.float() / s[:, :, None, None]).to(torch.float8_e4m3fn).view(torch.uint8)
+        c = torch.cat([c, torch.zeros((B, H, pad, d), dtype=torch.uint8)], 2).contiguous()
+        c[:, :, wl.N:] = 0x55                # canary in every row that is not live yet
+        return c
+    return codes(kc, ks), codes(vc, vs), ks, vs, qn, kn, vn
+
+
+@pytest.mark.parametrize("B,H,d,N0,T", [(2, 3, 128, 1000, 5), (1, 2, 64, 5, 9), (1, 1, 128, 0, 4), (2, 2, 64, 4100, 3)])
+def test_fp8_decode_steps_elementwise_and_exact_codes(B, H, d, N0, T):
+    wl = synth.Workload("dec8", B, H, d, N0, T, seed=61 + N0, decode=True)
+    kc_h, vc_h, ks, vs, qn, kn, vn = _fp8_cache(wl, pad=2)
+    kc, vc = kc_h.to(DEV), vc_h.to(DEV)
+    ks_d, vs_d = ks.to(DEV), vs.to(DEV)
+    for t in range(T):
+        out, lse = tl.tlin_decode_step_fp8(qn[t].to(DEV), kn[t].to(DEV), vn[t].to(DEV), kc, vc, ks_d, vs_d, N0 + t)
+        torch.cuda.synchronize()
+        assert tl.tlin_get_status() == 0 and tl.tlin_last_launch_count() == 2
+        ref, ref_lse = oracle.decode_step_fp8(qn[t], kn[t], vn[t], kc_h, vc_h, ks, vs, N0 + t)
+        parity.check(out.float().cpu().numpy(), lse.cpu().numpy(), ref, ref_lse, "bf16", f"fp8 decode step {t}")
+        # byte-exact bookkeeping: the appended codes equal the oracle's (same fp32 division, same rounding), the canary
+        # rows above are untouched
+        assert torch.equal(kc.cpu(), kc_h) and torch.equal(vc.cpu(), vc_h)
+        assert (kc[:, :, N0 + t + 1:] == 0x55).all() and (vc[:, :, N0 + t + 1:] == 0x55).all()
+
+
+def test_fp8_decode_saturates_and_keeps_signed_zero_like_the_oracle():
+    B, H, d, Ncap = 1, 2, 64, 8
+    kc = torch.zeros(B, H, Ncap, d, dtype=torch.uint8, device=DEV)
+    vc = torch.zeros_like(kc)
+    ks = torch.full((B, H), 0.01, device=DEV)
+    vs = torch.full((B, H), 0.5, device=DEV)
+    kn = torch.linspace(-8.0, 8.0, d).repeat(B, H, 1, 1).to(torch.bfloat16)       # |x| / 0.01 goes far beyond 448
+    vn = torch.cat([torch.tensor([0.0, -0.0, 1e-4, -1e-4]), torch.linspace(-300, 300, d - 4)]).repeat(B, H, 1, 1).to(torch.bfloat16)
+    q = torch.ones(B, H, 1, d).to(torch.bfloat16)
+    kc_h, vc_h = kc.cpu(), vc.cpu()
+    out, lse = tl.tlin_decode_step_fp8(q.to(DEV), kn.to(DEV), vn.to(DEV), kc, vc, ks, vs, 0)
+    torch.cuda.synchronize()
+    ref, ref_lse = oracle.decode_step_fp8(q, kn, vn, kc_h, vc_h, ks.cpu(), vs.cpu(), 0)
+    assert torch.equal(kc.cpu(), kc_h) and torch.equal(vc.cpu(), vc_h)
+    assert int(kc_h[0, 0, 0].max()) <= 0xFE and 0x7E in kc_h[0, 0, 0].tolist() and 0xFE in kc_h[0, 0, 0].tolist()
+    got = out.float().cpu().numpy()
+    assert np.abs(got - ref).max() <= 2e-2 * max(1.0, float(np.abs(ref).max()))
