@@ -35,7 +35,7 @@ from paper_2508_20407_b200 import synth  # noqa: E402
 
 WORKLOADS = {"fwd128k": "cfg4_vlong", "fwd32k": "cfg3_long", "fwd8k": "cfg2_mid", "decode": "cfg5_decode",
              "restore": "restore_vlong", "inner_self": "inner_self", "inner_gen": "inner_gen",
-             "bwd_chunk": "train_chunk", "bwd32k": "cfg3_long"}
+             "bwd_chunk": "train_chunk", "bwd32k": "cfg3_long", "decode_fp8": "cfg5_decode"}
 BACKWARD = ("bwd_chunk", "bwd32k")      # legs that time tlin_attn_backward on the named shape
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -416,6 +416,46 @@ def run_decode(wl, args, rank, world, device, peaks, with_cpu):
     return res
 
 
+def run_decode_fp8(wl, args, rank, world, device, peaks):
+    """Decode over an 8-bit (E4M3) cache of the same shape: half the bytes per cached row.  The cache holds seeded random
+    codes (every finite code value, no NaN codes); scales 1/64 per (b,h)."""
+    from paper_2508_20407_b200 import binding as tl
+    ncap = wl.N + wl.W
+    g = torch.Generator(device=device).manual_seed(wl.seed + 8)
+    def codes():
+        c = torch.randint(0, 254, (wl.B, wl.H, ncap, wl.d), generator=g, device=device, dtype=torch.int16)
+        return (c + (c >= 127).to(torch.int16)).to(torch.uint8).contiguous()        # skips 0x7f; 0xff is never drawn
+    kc, vc = codes(), codes()
+    ks = torch.full((wl.B, wl.H), 1.0 / 64.0, device=device)
+    vs = torch.full((wl.B, wl.H), 1.0 / 64.0, device=device)
+    _, (qn, kn, vn) = synth.decode_inputs(synth.Workload("fp8_new", wl.B, wl.H, wl.d, 0, wl.W, seed=wl.seed, decode=True), device=device)
+    out = torch.empty((wl.B, wl.H, 1, wl.d), dtype=torch.bfloat16, device=device)
+    lse = torch.empty((wl.B, wl.H), dtype=torch.float32, device=device)
+    tl.ensure_workspace(tl.workspace_bytes_decode(wl.B, wl.H, ncap, wl.d), device)
+    launches = []
+    steps = args.decode_steps
+
+    def step(i):
+        t = i % wl.W
+        tl.tlin_decode_step_fp8(qn[t], kn[t], vn[t], kc, vc, ks, vs, wl.N + t, out, lse)
+        launches.append(tl.tlin_last_launch_count())
+
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    ms, clocks = time_steps(step, steps, args.warmup, world, device, sampler)
+    ms_step = ms / steps
+    tot = 0
+    for i in range(args.warmup, args.warmup + steps):
+        pos = wl.N + (i % wl.W)
+        tot += 2 * wl.B * wl.H * (pos + 1) * wl.d + 4 * wl.B * wl.H * wl.d * 2 + 4 * wl.B * wl.H
+    gbs = tot / (ms * 1e-3) / 1e9
+    roof = dict(bound="hbm", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s", frac=gbs / peaks["hbm_gbs"], traffic=None,
+                algorithmic_bytes=tot / steps, peak_source=peaks["source"], kernel="decode over an 8-bit cache (split-K kernel + merge)",
+                roofline_ms=tot / steps / (peaks["hbm_gbs"] * 1e9) * 1e3)
+    return dict(workload=wl.name + " 8-bit cache", ms_per_step=ms_step, gb_per_s=world * gbs, steps=steps,
+                decode_tokens_per_s=world * wl.B / (ms_step * 1e-3), roofline=roof, e2e=None, clocks=clocks,
+                gpu_launches=int(sum(launches[args.warmup:])), launches_per_step=launches[-1] if launches else 0)
+
+
 # ----------------------------------------------------------------------------- reference arm (the oracle)
 def run_reference(args, rank, world):
     if rank != 0:
@@ -501,12 +541,14 @@ def main():
     with_cpu = (not args.no_cpu) and world == 1
     if args.workload in BACKWARD:
         main_res = run_backward(wl, args, rank, world, device, peaks)
+    elif args.workload == "decode_fp8":
+        main_res = run_decode_fp8(wl, args, rank, world, device, peaks)
     else:
         runner = run_decode if wl.decode else run_forward
         main_res = runner(wl, args, rank, world, device, peaks, with_cpu)
     also = []
     if not args.only and world == 1:
-        for name in ("fwd32k", "decode", "restore", "inner_self", "inner_gen", "bwd_chunk", "bwd32k"):
+        for name in ("fwd32k", "decode", "restore", "inner_self", "inner_gen", "bwd_chunk", "bwd32k", "decode_fp8"):
             if name == args.workload:
                 continue
             torch.cuda.empty_cache()
@@ -516,6 +558,8 @@ def main():
             a2.no_e2e = args.no_e2e or name not in ("fwd32k", "decode")     # host-buffer legs only where they are cheap to set up
             if name in BACKWARD:
                 also.append(run_backward(w2, a2, rank, world, device, peaks))
+            elif name == "decode_fp8":
+                also.append(run_decode_fp8(w2, a2, rank, world, device, peaks))
             else:
                 also.append((run_decode if w2.decode else run_forward)(w2, a2, rank, world, device, peaks, False))
 
