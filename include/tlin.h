@@ -248,7 +248,8 @@ int tlin_get_status(tlin_stream_t stream);
 const char* tlin_status_string(int status);
 const char* tlin_version(void);
 /* Which kernel serves tlin_attn_forward: 0 = automatic, 1 = always the CUDA-core kernel,
- * 2 = tensor-core kernel (TLIN_ERR_UNSUPPORTED if the shape does not allow it).  Returns the old value. */
+ * 2 = tensor-core kernel (TLIN_ERR_UNSUPPORTED if the shape does not allow it).  tlin_attn_backward follows the same
+ * switch (1 = CUDA-core kernels for every head size).  Returns the old value. */
 int tlin_set_forward_impl(int impl);
 /* Number of kernels launched by the last tlin_* compute call on this thread. */
 int tlin_last_launch_count(void);
