@@ -52,6 +52,7 @@ struct BwdParams {
     int n_groups, q_tiles, key_tiles, schedule;   // dq kernel: the forward's plan fields
     int q_tiles128;           // ceil(W / 128)
     int N, W, Wpad, causal;
+    int wide_stores;          // dq and the workspace are 32-byte aligned: the dQ kernel may use 32-byte stores
     float scale_log2e, scale;
 };
 
@@ -768,18 +769,23 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
                     for (int e = 0; e < 16; ++e) o[e] = 0u;
                 }
+                // a thread holds one row: 32-byte stores halve the number of (scattered) store instructions
+                // (taken when dq and the workspace are 32-byte aligned; the interface only promises 16)
                 if (whole) {
                     if (row_ok) {
+                        uint32_t w[8];
 #pragma unroll
-                        for (int v4 = 0; v4 < 2; ++v4) {
-                            uint4 w;
-                            w.x = pack_bf16x2(__uint_as_float(o[v4 * 8 + 0]) * f, __uint_as_float(o[v4 * 8 + 1]) * f);
-                            w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * f, __uint_as_float(o[v4 * 8 + 3]) * f);
-                            w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * f, __uint_as_float(o[v4 * 8 + 5]) * f);
-                            w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * f, __uint_as_float(o[v4 * 8 + 7]) * f);
-                            *reinterpret_cast<uint4*>(drow + c * 16 + v4 * 8) = w;
+                        for (int e = 0; e < 8; ++e) w[e] = pack_bf16x2(__uint_as_float(o[2 * e]) * f, __uint_as_float(o[2 * e + 1]) * f);
+                        if (p.wide_stores) {
+                            st_global_v8(drow + c * 16, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+                        } else {
+                            *reinterpret_cast<uint4*>(drow + c * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+                            *reinterpret_cast<uint4*>(drow + c * 16 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
                         }
                     }
+                } else if (p.wide_stores) {
+                    st_global_v8(prow + c * 16, o[0], o[1], o[2], o[3], o[4], o[5], o[6], o[7]);
+                    st_global_v8(prow + c * 16 + 8, o[8], o[9], o[10], o[11], o[12], o[13], o[14], o[15]);
                 } else {
 #pragma unroll
                     for (int v4 = 0; v4 < 4; ++v4)
@@ -861,6 +867,7 @@ int launch_d(const void* q, const void* k, const void* v, const void* out, const
     p.N = N; p.W = W; p.Wpad = Wpad; p.causal = causal;
     p.scale = 1.f / sqrtf((float)D);
     p.scale_log2e = kLog2e * p.scale;
+    p.wide_stores = ((reinterpret_cast<uintptr_t>(dq) | reinterpret_cast<uintptr_t>(ws)) & 31u) == 0;
     static std::once_flag attr_once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(attr_once, [] {
