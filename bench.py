@@ -35,7 +35,8 @@ from paper_2508_20407_b200 import synth  # noqa: E402
 
 WORKLOADS = {"fwd128k": "cfg4_vlong", "fwd32k": "cfg3_long", "fwd8k": "cfg2_mid", "decode": "cfg5_decode",
              "restore": "restore_vlong", "inner_self": "inner_self", "inner_gen": "inner_gen",
-             "bwd_chunk": "train_chunk", "bwd32k": "cfg3_long", "decode_fp8": "cfg5_decode"}
+             "bwd_chunk": "train_chunk", "bwd32k": "cfg3_long", "decode_fp8": "cfg5_decode",
+             "nsweep": "cfg3_long"}
 BACKWARD = ("bwd_chunk", "bwd32k")      # legs that time tlin_attn_backward on the named shape
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -456,6 +457,48 @@ def run_decode_fp8(wl, args, rank, world, device, peaks):
                 gpu_launches=int(sum(launches[args.warmup:])), launches_per_step=launches[-1] if launches else 0)
 
 
+def run_n_sweep(args, rank, world, device, peaks):
+    """Forward time against context length at fixed B, H, W, d (the paper's claim is cost linear in N, Section 4 and
+    Appendix A): N = 8k ... 256k, least-squares line t = a + b*N and its largest relative residual; cfg3/cfg4 also with
+    causal_window = 0."""
+    from paper_2508_20407_b200 import binding as tl
+    pts = []
+    for n in (8192, 16384, 32768, 65536, 131072, 262144):
+        wl = synth.Workload(f"sweep_N{n}", 1, 32, 128, n, 512, seed=11, causal_window=1)
+        q, k, v = synth.forward_inputs(wl, device=device)
+        out = torch.empty_like(q)
+        lse = torch.empty((wl.B, wl.H, wl.W), dtype=torch.float32, device=device)
+        tl.ensure_workspace(tl.workspace_bytes_forward(wl.B, wl.H, wl.N, wl.W, wl.d, 1), device)
+        flush = torch.empty(int(2.5 * L2_BYTES), dtype=torch.uint8, device=device) if fwd_bytes(wl) < 2 * L2_BYTES else None
+        ms, _ = time_steps(lambda _: tl.tlin_attn_forward(q, k, v, out, lse, 1), args.steps, args.warmup, world, device, None, flush)
+        ms /= args.steps
+        pts.append(dict(N=n, ms=ms, tflops=4.0 * wl.B * wl.H * wl.W * n * wl.d / (ms * 1e-3) / 1e12))
+        del q, k, v, out, lse, flush
+        torch.cuda.empty_cache()
+    import numpy as np
+    x = np.array([p["N"] for p in pts], dtype=np.float64)
+    y = np.array([p["ms"] for p in pts], dtype=np.float64)
+    b, a = np.polyfit(x, y, 1)
+    resid = float(np.max(np.abs(a + b * x - y) / y))
+    unmasked = []
+    for name in ("cfg3_long", "cfg4_vlong"):
+        wl = synth.WORKLOADS[name]
+        q, k, v = synth.forward_inputs(wl, device=device)
+        out = torch.empty_like(q)
+        lse = torch.empty((wl.B, wl.H, wl.W), dtype=torch.float32, device=device)
+        row = dict(workload=name)
+        for causal in (1, 0):
+            tl.ensure_workspace(tl.workspace_bytes_forward(wl.B, wl.H, wl.N, wl.W, wl.d, causal), device)
+            ms, _ = time_steps(lambda _: tl.tlin_attn_forward(q, k, v, out, lse, causal), args.steps, args.warmup, world, device)
+            row[f"ms_causal_window_{causal}"] = ms / args.steps
+        unmasked.append(row)
+        del q, k, v, out, lse
+        torch.cuda.empty_cache()
+    return dict(points=pts, fit=dict(intercept_ms=float(a), ms_per_1k_keys=float(b * 1024), max_rel_residual=resid),
+                t_cfg4_over_t_cfg3=unmasked[1]["ms_causal_window_1"] / unmasked[0]["ms_causal_window_1"], flop_ratio=8.0,
+                causal_vs_unmasked=unmasked, shape="B1 H32 W512 d128, causal window")
+
+
 # ----------------------------------------------------------------------------- reference arm (the oracle)
 def run_reference(args, rank, world):
     if rank != 0:
@@ -533,6 +576,13 @@ def main():
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=device)
     peaks = load_peaks()
+    if args.workload == "nsweep":          # a measurement of its own (linearity in N), not a bench line
+        res = run_n_sweep(args, rank, world, device, peaks)
+        if rank == 0:
+            print(json.dumps({"metric": "forward_ms_vs_context_length", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, **res}), flush=True)
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return 0
     wl = synth.WORKLOADS[WORKLOADS[args.workload]]
     if args.shape:
         v = [int(x) for x in args.shape.split(",")]
