@@ -38,6 +38,7 @@ WORKLOADS = {"fwd128k": "cfg4_vlong", "fwd32k": "cfg3_long", "fwd8k": "cfg2_mid"
              "bwd_chunk": "train_chunk", "bwd32k": "cfg3_long", "decode_fp8": "cfg5_decode",
              "nsweep": "cfg3_long"}
 BACKWARD = ("bwd_chunk", "bwd32k")      # legs that time tlin_attn_backward on the named shape
+NOMINAL_BF16_TFLOPS, NOMINAL_HBM_GBS = 2250.0, 7700.0      # datasheet figures, reported beside the measured peaks
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -276,6 +277,7 @@ def run_forward(wl, args, rank, world, device, peaks, with_cpu):
                 roofline_ms=max(t_tensor, t_hbm) * 1e3)
     if bound == "tensor" and "bf16_tflops_sustained" in peaks:
         roof["frac_of_sustained_peak"] = tflops / peaks["bf16_tflops_sustained"]
+    roof["nominal"] = dict(peak=NOMINAL_BF16_TFLOPS, unit="TFLOP/s", frac=tflops / NOMINAL_BF16_TFLOPS, note="datasheet dense bf16, context only")
 
     # end to end: pinned host buffers through the host entry point
     e2e = None
@@ -345,6 +347,7 @@ def run_backward(wl, args, rank, world, device, peaks):
                 executed_over_counted_flops=1.4, roofline_ms=flop / (peaks["bf16_tflops"] * 1e12) * 1e3)
     if "bf16_tflops_sustained" in peaks:
         roof["frac_of_sustained_peak"] = tflops / peaks["bf16_tflops_sustained"]
+    roof["nominal"] = dict(peak=NOMINAL_BF16_TFLOPS, unit="TFLOP/s", frac=tflops / NOMINAL_BF16_TFLOPS, note="datasheet dense bf16, context only")
     l2_note = ("inputs+outputs %.0f MB > 2 x L2 (126 MB): back-to-back calls, no flush" % (nbytes / 1e6) if flush is None else
                "inputs+outputs %.0f MB: a %.0f MB buffer is overwritten before every timed call (L2 flush), calls timed one by one"
                % (nbytes / 1e6, flush.numel() / 1e6))
@@ -381,7 +384,8 @@ def run_decode(wl, args, rank, world, device, peaks, with_cpu):
                 traffic=tot / steps * DECODE_TRAFFIC_RATIO, algorithmic_bytes=tot / steps,
                 traffic_source="ncu on a 4096-row cache, scaled by the cached rows (traffic is proportional to them)",
                 peak_source=peaks["source"], kernel="decode (split-K kernel + merge)",
-                roofline_ms=tot / steps / (peaks["hbm_gbs"] * 1e9) * 1e3)
+                roofline_ms=tot / steps / (peaks["hbm_gbs"] * 1e9) * 1e3,
+                nominal=dict(peak=NOMINAL_HBM_GBS, unit="GB/s", frac=gbs / NOMINAL_HBM_GBS, note="datasheet HBM3e, context only"))
     e2e = None
     if not args.no_e2e:
         host = [t.cpu().pin_memory() for t in (qn, kn, vn)]
@@ -451,7 +455,8 @@ def run_decode_fp8(wl, args, rank, world, device, peaks):
     gbs = tot / (ms * 1e-3) / 1e9
     roof = dict(bound="hbm", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s", frac=gbs / peaks["hbm_gbs"], traffic=None,
                 algorithmic_bytes=tot / steps, peak_source=peaks["source"], kernel="decode over an 8-bit cache (split-K kernel + merge)",
-                roofline_ms=tot / steps / (peaks["hbm_gbs"] * 1e9) * 1e3)
+                roofline_ms=tot / steps / (peaks["hbm_gbs"] * 1e9) * 1e3,
+                nominal=dict(peak=NOMINAL_HBM_GBS, unit="GB/s", frac=gbs / NOMINAL_HBM_GBS, note="datasheet HBM3e, context only"))
     return dict(workload=wl.name + " 8-bit cache", ms_per_step=ms_step, gb_per_s=world * gbs, steps=steps,
                 decode_tokens_per_s=world * wl.B / (ms_step * 1e-3), roofline=roof, e2e=None, clocks=clocks,
                 gpu_launches=int(sum(launches[args.warmup:])), launches_per_step=launches[-1] if launches else 0)
