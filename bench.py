@@ -278,6 +278,11 @@ def run_forward(wl, args, rank, world, device, peaks, with_cpu):
     if bound == "tensor" and "bf16_tflops_sustained" in peaks:
         roof["frac_of_sustained_peak"] = tflops / peaks["bf16_tflops_sustained"]
     roof["nominal"] = dict(peak=NOMINAL_BF16_TFLOPS, unit="TFLOP/s", frac=tflops / NOMINAL_BF16_TFLOPS, note="datasheet dense bf16, context only")
+    # second ceiling: one exponential per (query, key) pair; the special-function units retire 16 per clock and SM
+    exps = float(wl.B) * wl.H * wl.W * wl.N
+    sfu_rate = 16.0 * 148 * 1.965e9
+    roof["secondary"] = dict(bound="special-function unit", exponentials=exps, roofline_ms=exps / sfu_rate * 1e3,
+                             note="16 ex2 per clock per SM x 148 SMs x 1965 MHz; the kernel evaluates 5/16 of them on the FMA pipe")
 
     # end to end: pinned host buffers through the host entry point
     e2e = None
