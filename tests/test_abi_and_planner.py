@@ -198,3 +198,14 @@ def test_backward_workspace_covers_row_statistics_and_partial_sums():
             need = max(need, tc)
         assert got == need, (B, H, N, W, d, got, need)
     assert tl.workspace_bytes_backward(0, 1, 1, 1, 64) == 0
+
+
+def test_prefix_workspace_is_the_largest_of_the_chunks():
+    import ctypes
+    B, H, W, d = 1, 8, 512, 128
+    n_keys = [512, 4096, 32768, 65536]
+    arr = (ctypes.c_int32 * len(n_keys))(*n_keys)
+    for causal in (0, 1):
+        got = int(tl.lib().tlin_workspace_bytes_forward_prefixes(B, H, W, d, len(n_keys), arr, causal))
+        assert got == max(tl.workspace_bytes_forward(B, H, n, W, d, causal) for n in n_keys)
+    assert int(tl.lib().tlin_workspace_bytes_forward_prefixes(B, H, W, d, 0, arr, 1)) == 0
