@@ -392,3 +392,33 @@ def tlin_set_forward_impl(impl: int) -> int:
 
 def tlin_last_launch_count() -> int:
     return int(lib().tlin_last_launch_count())
+
+
+# ------------------------------------------------------------------ autograd glue (marshalling only)
+class _AttentionFunction(torch.autograd.Function):
+    """Lets PyTorch's autograd call the library's forward and backward entry points; nothing is computed here."""
+
+    @staticmethod
+    def forward(ctx, q, k, v, causal_window):
+        f32 = q.dtype == torch.float32
+        q, k, v = q.contiguous(), k.contiguous(), v.contiguous()
+        out, lse = (tlin_attn_forward_f32 if f32 else tlin_attn_forward)(q, k, v, causal_window=causal_window)
+        ctx.save_for_backward(q, k, v, out, lse)
+        ctx.causal_window = int(causal_window)
+        ctx.f32 = f32
+        ctx.mark_non_differentiable(lse)
+        return out, lse
+
+    @staticmethod
+    def backward(ctx, dout, _dlse):
+        q, k, v, out, lse = ctx.saved_tensors
+        fn = tlin_attn_backward_f32 if ctx.f32 else tlin_attn_backward
+        dq, dk, dv = fn(q, k, v, out, lse, dout.contiguous(), causal_window=ctx.causal_window)
+        return dq, dk, dv, None
+
+
+def attention(q, k, v, causal_window=1):
+    """Differentiable attention for PyTorch training code: (out, lse) = tlin_attn_forward(q, k, v); gradients of `out`
+    with respect to q, k, v come from tlin_attn_backward (lse is returned for merging and is not differentiable).
+    bf16 or fp32 tensors, shapes as in tlin_attn_forward."""
+    return _AttentionFunction.apply(q, k, v, causal_window)

@@ -196,3 +196,27 @@ def test_backward_at_the_benchmarked_training_shape_on_two_heads():
         compare(dq[sl], rq, f"train_chunk b{b} h{h} dq")
         compare(dk[sl], rk, f"train_chunk b{b} h{h} dk")
         compare(dv[sl], rv, f"train_chunk b{b} h{h} dv")
+
+
+@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 128), (torch.float32, 36)])
+def test_autograd_glue_matches_pytorch_autograd_of_the_textbook_formula(dtype, d):
+    # tl.attention plugs the two entry points into torch.autograd; the reference differentiates the formula itself in fp64
+    B, H, N, W, causal = 2, 2, 300, 130, 1
+    g = torch.Generator(device="cpu").manual_seed(17)
+    mk = lambda *s: (torch.randn(*s, generator=g) / 3).to(dtype).to(DEV).requires_grad_(True)
+    q, k, v = mk(B, H, W, d), mk(B, H, N, d), mk(B, H, N, d)
+    w = torch.randn(B, H, W, d, generator=g).to(DEV)
+    out, lse = tl.attention(q, k, v, causal_window=causal)
+    (out.float() * w).sum().backward()
+    qd, kd, vd = (t.detach().double().cpu().requires_grad_(True) for t in (q, k, v))
+    s = qd @ kd.transpose(-1, -2) / d ** 0.5
+    i = torch.arange(W)[:, None]
+    j = torch.arange(N)[None, :]
+    s = s.masked_fill(j > (N - W) + i, float("-inf"))
+    ref = torch.softmax(s, -1) @ vd
+    (ref * w.double().cpu()).sum().backward()
+    tol = 2e-2 if dtype == torch.bfloat16 else 1e-4
+    for got, want, name in ((q.grad, qd.grad, "dq"), (k.grad, kd.grad, "dk"), (v.grad, vd.grad, "dv")):
+        err = float((got.double().cpu() - want).abs().max())
+        assert err <= tol * float(want.abs().max()) + 1e-6, f"{name}: {err:.3e}"
+    assert not lse.requires_grad
