@@ -232,6 +232,40 @@ __device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {     //
     asm("{\n\t.reg .b16 c;\n\tcvt.rn.satfinite.e4m3x2.f32 c, %1, %2;\n\tcvt.u32.u16 %0, c;\n\t}" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
+// sum += k . q for the 16 codes of `c` against 16 f16 values of q (8 packed words): codes widened to f16 pairs (exact),
+// products and sum in fp32 by the mixed-precision fma
+__device__ __forceinline__ float dot16_codes(const uint4& c, const uint32_t (&qh)[8]) {
+    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        asm("{\n\t.reg .b16 c0, c1, k0, k1, k2, k3, q0, q1, q2, q3;\n\t.reg .b32 h0, h1;\n\t"
+            "mov.b32 {c0, c1}, %1;\n\t"
+            "cvt.rn.f16x2.e4m3x2 h0, c0;\n\tcvt.rn.f16x2.e4m3x2 h1, c1;\n\t"
+            "mov.b32 {k0, k1}, h0;\n\tmov.b32 {k2, k3}, h1;\n\t"
+            "mov.b32 {q0, q1}, %2;\n\tmov.b32 {q2, q3}, %3;\n\t"
+            "fma.rn.f32.f16 %0, k0, q0, %0;\n\tfma.rn.f32.f16 %0, k1, q1, %0;\n\t"
+            "fma.rn.f32.f16 %0, k2, q2, %0;\n\tfma.rn.f32.f16 %0, k3, q3, %0;\n\t}"
+            : "+f"(s) : "r"(w[i]), "r"(qh[2 * i]), "r"(qh[2 * i + 1]));
+    }
+    return s;
+}
+// acc[e] += p * v_e for the 16 codes of `c`; p given twice in one word as f16 (weights lie in (0,1]: rounding them to
+// 11 mantissa bits is far below the bf16 rounding of the output), codes widened to f16 (exact), products and sums in fp32
+__device__ __forceinline__ void axpy16_codes(uint32_t p2, const uint4& c, float (&acc)[16]) {
+    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        asm("{\n\t.reg .b16 c0, c1, v0, v1, v2, v3, p0, p1;\n\t.reg .b32 h0, h1;\n\t"
+            "mov.b32 {c0, c1}, %4;\n\t"
+            "cvt.rn.f16x2.e4m3x2 h0, c0;\n\tcvt.rn.f16x2.e4m3x2 h1, c1;\n\t"
+            "mov.b32 {v0, v1}, h0;\n\tmov.b32 {v2, v3}, h1;\n\t"
+            "mov.b32 {p0, p1}, %5;\n\t"
+            "fma.rn.f32.f16 %0, v0, p0, %0;\n\tfma.rn.f32.f16 %1, v1, p0, %1;\n\t"
+            "fma.rn.f32.f16 %2, v2, p0, %2;\n\tfma.rn.f32.f16 %3, v3, p0, %3;\n\t}"
+            : "+f"(acc[4 * i]), "+f"(acc[4 * i + 1]), "+f"(acc[4 * i + 2]), "+f"(acc[4 * i + 3]) : "r"(w[i]), "r"(p2));
+    }
+}
 __device__ __forceinline__ void widen16(const uint4& c, float (&x)[16]) {
     const uint32_t w[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
@@ -281,15 +315,16 @@ decode_fp8_splitk_kernel(const uint4* __restrict__ q_new, const uint4* __restric
         v_cache[((int64_t)bh * Ncap + pos) * LPR + lane] = vn_codes;
     }
 
-    float qf[16];
+    // q * log2(e)/sqrt(d) as f16 pairs (|q| of a few units: no range issue; 11 mantissa bits against the 8 of the bf16
+    // input); the key scale multiplies the finished dot product
+    uint32_t qh[8];
     {
         const uint4 q0 = q_new[(int64_t)bh * (D / 8) + 2 * sub], q1 = q_new[(int64_t)bh * (D / 8) + 2 * sub + 1];
         const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
-        const float f = scale_log2e * ks;                 // the key scale rides on q
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            qf[2 * i] = bf_lo(w[i]) * f;
-            qf[2 * i + 1] = bf_hi(w[i]) * f;
+            const __half2 h = __floats2half2_rn(bf_lo(w[i]) * scale_log2e, bf_hi(w[i]) * scale_log2e);
+            qh[i] = *reinterpret_cast<const uint32_t*>(&h);
         }
     }
 
@@ -321,14 +356,10 @@ decode_fp8_splitk_kernel(const uint4* __restrict__ q_new, const uint4* __restric
         float mb = m;
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
-            float kx[16];
-            widen16(kv[u], kx);
-            float x = 0.f;
-#pragma unroll
-            for (int e = 0; e < 16; ++e) x = fmaf(kx[e], qf[e], x);
+            float x = dot16_codes(kv[u], qh);
 #pragma unroll
             for (int o = LPR / 2; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-            s[u] = ok[u] ? x : -CUDART_INF_F;
+            s[u] = ok[u] ? x * ks : -CUDART_INF_F;
             mb = fmaxf(mb, s[u]);
         }
         const float ms = mb == -CUDART_INF_F ? 0.f : mb;
@@ -339,11 +370,9 @@ decode_fp8_splitk_kernel(const uint4* __restrict__ q_new, const uint4* __restric
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
             const float pr = exp2f(s[u] - ms);
-            l += pr;
-            float vx[16];
-            widen16(vv[u], vx);
-#pragma unroll
-            for (int e = 0; e < 16; ++e) acc[e] = fmaf(pr, vx[e], acc[e]);
+            const __half2 ph = __float2half2_rn(pr);
+            l += __low2float(ph);                 // the same rounded weight in the numerator and the denominator
+            axpy16_codes(*reinterpret_cast<const uint32_t*>(&ph), vv[u], acc);
         }
         m = mb;
     }
