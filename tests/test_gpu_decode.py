@@ -246,3 +246,31 @@ def test_fp8_decode_saturates_and_keeps_signed_zero_like_the_oracle():
     assert int(kc_h[0, 0, 0].max()) <= 0xFE and 0x7E in kc_h[0, 0, 0].tolist() and 0xFE in kc_h[0, 0, 0].tolist()
     got = out.float().cpu().numpy()
     assert np.abs(got - ref).max() <= 2e-2 * max(1.0, float(np.abs(ref).max()))
+
+
+def test_fp8_decode_at_the_cfg5_size_on_sampled_heads():
+    # the benchmarked 8-bit configuration (B8 H32 d128, 65536 cached rows): three heads of three steps against the oracle,
+    # the appended codes of those heads byte for byte
+    wl = synth.WORKLOADS["cfg5_decode"]
+    B, H, d, N = wl.B, wl.H, wl.d, wl.N
+    g = torch.Generator(device=DEV).manual_seed(77)
+    def codes():
+        c = torch.randint(0, 254, (B, H, N + 8, d), generator=g, device=DEV, dtype=torch.int16)
+        return (c + (c >= 127).to(torch.int16)).to(torch.uint8).contiguous()       # every finite code, no NaN code
+    kc, vc = codes(), codes()
+    ks = (torch.rand(B, H, generator=g, device=DEV) * 0.01 + 0.002).float()
+    vs = (torch.rand(B, H, generator=g, device=DEV) * 0.01 + 0.002).float()
+    q, kn, vn = (torch.randn(3, B, H, 1, d, generator=g, device=DEV).to(torch.bfloat16) for _ in range(3))
+    heads = [(0, 0), (3, 17), (7, 31)]
+    host = {bh: (kc[bh[0], bh[1]].cpu().view(1, 1, -1, d).contiguous(), vc[bh[0], bh[1]].cpu().view(1, 1, -1, d).contiguous()) for bh in heads}
+    for t in range(3):
+        out, lse = tl.tlin_decode_step_fp8(q[t], kn[t], vn[t], kc, vc, ks, vs, N + t)
+        torch.cuda.synchronize()
+        assert tl.tlin_get_status() == 0
+        for (b, h) in heads:
+            sl = lambda x: x[b:b + 1, h:h + 1].cpu().contiguous()
+            kh, vh = host[(b, h)]
+            ref, ref_lse = oracle.decode_step_fp8(sl(q[t]), sl(kn[t]), sl(vn[t]), kh, vh, sl(ks), sl(vs), N + t)
+            parity.check(sl(out).float().numpy(), sl(lse).numpy(), ref, ref_lse, "bf16", f"8-bit cfg5 step {t} head {(b, h)}")
+    for (b, h) in heads:
+        assert torch.equal(kc[b, h].cpu(), host[(b, h)][0][0, 0]) and torch.equal(vc[b, h].cpu(), host[(b, h)][1][0, 0])
