@@ -597,7 +597,7 @@ def main():
     if args.shape:
         v = [int(x) for x in args.shape.split(",")]
         wl = synth.Workload("custom_" + args.shape.replace(",", "_"), v[0], v[1], v[4], v[2], v[3], seed=9,
-                            causal_window=v[5] if len(v) > 5 else 1, decode=args.workload == "decode")
+                            causal_window=v[5] if len(v) > 5 else 1, decode=args.workload in ("decode", "decode_fp8"))
     with_cpu = (not args.no_cpu) and world == 1
     if args.workload in BACKWARD:
         main_res = run_backward(wl, args, rank, world, device, peaks)
