@@ -195,6 +195,8 @@ FWD_TRAFFIC = {"cfg4_vlong": (2177.07e6 + 19.71e6, "ncu, full workload, fwd_tc_k
 # decode: captured on a smaller cache (B8 H32, 4096 rows: 537.35 MB read + 3.9 MB written for 537.3 MB of cache) and
 # scaled by the cached rows of the timed steps; the kernel streams every cached byte once at any size
 DECODE_TRAFFIC_RATIO = (537.35 + 3.9) / 537.3
+# 8-bit cache: 268.9 MB read + 4.0 MB written for 268.4 MB of codes (B8 H32, 4096 rows), scaled the same way
+DECODE_FP8_TRAFFIC_RATIO = (268.9 + 4.0) / 268.4
 
 
 # ----------------------------------------------------------------------------- the oracle as a timed baseline
@@ -458,7 +460,9 @@ def run_decode_fp8(wl, args, rank, world, device, peaks):
         pos = wl.N + (i % wl.W)
         tot += 2 * wl.B * wl.H * (pos + 1) * wl.d + 4 * wl.B * wl.H * wl.d * 2 + 4 * wl.B * wl.H
     gbs = tot / (ms * 1e-3) / 1e9
-    roof = dict(bound="hbm", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s", frac=gbs / peaks["hbm_gbs"], traffic=None,
+    roof = dict(bound="hbm", achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s", frac=gbs / peaks["hbm_gbs"],
+                traffic=tot / steps * DECODE_FP8_TRAFFIC_RATIO,
+                traffic_source="ncu on a 4096-row cache, scaled by the cached rows (traffic is proportional to them)",
                 algorithmic_bytes=tot / steps, peak_source=peaks["source"], kernel="decode over an 8-bit cache (split-K kernel + merge)",
                 roofline_ms=tot / steps / (peaks["hbm_gbs"] * 1e9) * 1e3,
                 nominal=dict(peak=NOMINAL_HBM_GBS, unit="GB/s", frac=gbs / NOMINAL_HBM_GBS, note="datasheet HBM3e, context only"))
