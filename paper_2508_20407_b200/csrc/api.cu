@@ -93,8 +93,9 @@ extern "C" int tlin_attn_forward_prefixes(const void* q, const void* k, const vo
                                           int B, int H, int L, int W, int d, int C, const int32_t* n_keys,
                                           int causal_window, tlin_stream_t stream) {
     if (!n_keys || C <= 0 || L <= 0 || B <= 0 || H <= 0 || W <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
-    for (int c = 0; c < C; ++c)
-        if (n_keys[c] <= 0 || n_keys[c] > L) return TLIN_ERR_INVALID_ARG;
+    if (causal_window != 0 && causal_window != 1) return TLIN_ERR_INVALID_ARG;
+    for (int c = 0; c < C; ++c)      // every chunk is checked before the first one is launched
+        if (n_keys[c] <= 0 || n_keys[c] > L || (causal_window && n_keys[c] < W)) return TLIN_ERR_INVALID_ARG;
     if (d != 64 && d != 128) return TLIN_ERR_UNSUPPORTED;
     const size_t q_chunk = (size_t)B * H * W * d * 2, lse_chunk = (size_t)B * H * W;
     int total = 0;                 // a chunked call counts the launches of all its chunks
