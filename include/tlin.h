@@ -231,6 +231,11 @@ typedef struct {
 /* num_sms <= 0 means "use the value of the B200 (148)". */
 int tlin_plan_forward(int B, int H, int N, int W, int d, int causal_window, int is_f32, int num_sms, tlin_fwd_plan* plan);
 int tlin_plan_decode(int B, int H, int L, int d, int num_sms, tlin_decode_plan* plan);
+/* Work sharing of the tensor-core dK/dV kernel of tlin_attn_backward: its units are (b,h,128-key tile) in that order and
+ * CTA `share` of `n_shares` starts at the unit returned here (share = n_shares gives the unit count B*H*ceil(N/128)).  The
+ * shares are balanced by the number of 128-row query tiles each key tile has to visit, which under the window rule falls
+ * towards the end of a (b,h).  -1 on bad arguments. */
+int64_t tlin_plan_backward_share_start(int B, int H, int N, int W, int causal_window, int share, int n_shares);
 /* First unit of group g: floor(g * total_units / n_groups). */
 int64_t tlin_plan_group_start(const tlin_fwd_plan* plan, int g);
 /* Mask predicate: may query i (0 <= i < W) use key j?  1 or 0. */

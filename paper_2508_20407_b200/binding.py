@@ -62,6 +62,7 @@ SIGNATURES = {
     "tlin_plan_forward": (_i, [_i] * 8 + [ctypes.POINTER(FwdPlan)]),
     "tlin_plan_decode": (_i, [_i] * 5 + [ctypes.POINTER(DecodePlan)]),
     "tlin_plan_group_start": (_i64, [ctypes.POINTER(FwdPlan), _i]),
+    "tlin_plan_backward_share_start": (_i64, [_i] * 7),
     "tlin_allowed": (_i, [_i64] * 4 + [_i]),
     "tlin_tile_class": (_i, [_i64, _i64, _i, _i, _i, _i, _i]),
     "tlin_get_status": (_i, [_vp]),

@@ -172,8 +172,10 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const uint32_t tmem_base = *tmem_slot;
     volatile int* abort_p = abort_flag;
 
-    const long long u_begin = (long long)(((unsigned long long)blockIdx.x * (unsigned long long)p.total_units) / gridDim.x);
-    const long long u_end = (long long)(((unsigned long long)(blockIdx.x + 1) * (unsigned long long)p.total_units) / gridDim.x);
+    // The CTAs share the (b,h,key tile) units by cost (query tiles a key tile has to visit), not by count: with the
+    // window rule the last key tiles of a (b,h) are cheaper, down to one step.
+    const long long u_begin = bwd_first_unit_of_share(p.N, p.W, p.causal, p.total_units, p.key_tiles, blockIdx.x, gridDim.x);
+    const long long u_end = bwd_first_unit_of_share(p.N, p.W, p.causal, p.total_units, p.key_tiles, blockIdx.x + 1, gridDim.x);
 
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ TMA producer: Q / dout / row statistics ring

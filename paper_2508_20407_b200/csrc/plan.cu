@@ -159,3 +159,10 @@ extern "C" size_t tlin_workspace_bytes_decode(int B, int H, int Ncap, int d) {
     if (tlin_plan_decode(B, H, Ncap > 0 ? Ncap : 1, d, 0, &p) != TLIN_OK) return 0;
     return (size_t)p.workspace_bytes;
 }
+
+extern "C" int64_t tlin_plan_backward_share_start(int B, int H, int N, int W, int causal_window, int share, int n_shares) {
+    if (B <= 0 || H <= 0 || N <= 0 || W <= 0 || n_shares <= 0 || share < 0) return -1;
+    if (causal_window && N < W) return -1;
+    const int key_tiles = (N + kTileN - 1) / kTileN;
+    return tlin::bwd_first_unit_of_share(N, W, causal_window, (long long)B * H * key_tiles, key_tiles, (unsigned)share, (unsigned)n_shares);
+}

@@ -22,6 +22,41 @@ int* status_word();                    // device address of the error word (boun
 void count_launch(int n = 1);
 int forward_impl();
 
+// Work sharing of the tensor-core dK/dV kernel (host and device use the same arithmetic).  Units are (b,h,key tile) in that
+// order, key tiles of 128 keys, query tiles of 128 rows; with the window rule key tile t is visited by the query tiles from
+// floor(max(0, 128 t - (N-W)) / 128) on, so the last key tiles of a (b,h) cost fewer steps, down to one.  Share c of G starts at
+// the smallest unit u such that the steps of the units before it reach c/G of all steps.
+__host__ __device__ inline long long bwd_first_unit_of_share(int N, int W, int causal, long long total_units, int key_tiles,
+                                                            unsigned c, unsigned G) {
+    const int T = key_tiles, Qt = (W + 127) / 128;
+    if (c >= G) return total_units;
+    if (!causal) return (long long)(((unsigned long long)c * (unsigned long long)total_units) / G);
+    auto steps_of = [&](long long t) {
+        const long long f = t * 128 - ((long long)N - W);
+        return (long long)Qt - (f <= 0 ? 0 : f / 128);
+    };
+    long long t_full = ((long long)N - W) / 128 + 1;                 // tiles [0, t_full) visit every query tile
+    if (t_full > T) t_full = T;
+    long long per_bh = t_full * Qt;
+    for (long long t = t_full; t < T; ++t) per_bh += steps_of(t);
+    const long long n_bh = total_units / T;
+    const unsigned long long target = ((unsigned long long)c * (unsigned long long)(per_bh * n_bh)) / G;
+    const long long bh = (long long)(target / (unsigned long long)per_bh);
+    const long long rem = (long long)(target - (unsigned long long)bh * (unsigned long long)per_bh);   // steps into this (b,h)
+    long long t;
+    if (rem <= t_full * Qt) {
+        t = (rem + Qt - 1) / Qt;                                      // smallest t with t * Qt >= rem
+    } else {
+        long long cum = t_full * Qt;
+        t = t_full;
+        while (t < T && cum < rem) {
+            cum += steps_of(t);
+            ++t;
+        }
+    }
+    return bh * T + t;
+}
+
 #define TLIN_CUDA_CHECK(expr)                                                              \
     do {                                                                                   \
         cudaError_t e__ = (expr);                                                          \

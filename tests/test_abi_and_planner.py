@@ -209,3 +209,29 @@ def test_prefix_workspace_is_the_largest_of_the_chunks():
         got = int(tl.lib().tlin_workspace_bytes_forward_prefixes(B, H, W, d, len(n_keys), arr, causal))
         assert got == max(tl.workspace_bytes_forward(B, H, n, W, d, causal) for n in n_keys)
     assert int(tl.lib().tlin_workspace_bytes_forward_prefixes(B, H, W, d, 0, arr, 1)) == 0
+
+
+def test_backward_key_tile_shares_cover_everything_and_balance_the_steps():
+    import random
+    L = tl.lib()
+    rnd = random.Random(3)
+    cases = [(1, 32, 32768, 512, 1), (4, 32, 8192, 1024, 1), (2, 3, 1024, 1024, 1), (1, 1, 1, 1, 1), (2, 5, 4000, 700, 0)]
+    cases += [(rnd.randint(1, 3), rnd.randint(1, 9), 0, rnd.randint(1, 1500), 1) for _ in range(40)]
+    for B, H, N, W, causal in cases:
+        if N == 0:
+            N = W + rnd.choice([0, 1, 127, 128, 129, rnd.randint(0, 5000)])
+        T, Qt = (N + 127) // 128, (W + 127) // 128
+        total = B * H * T
+        G = min(total, 148)
+        starts = [L.tlin_plan_backward_share_start(B, H, N, W, causal, c, G) for c in range(G + 1)]
+        assert starts[0] == 0 and starts[-1] == total
+        assert all(a <= b for a, b in zip(starts, starts[1:]))                 # contiguous, disjoint, complete
+
+        def steps(u):                                                          # query tiles key tile u % T has to visit
+            f = (u % T) * 128 - (N - W)
+            return Qt - (0 if (not causal or f <= 0) else f // 128)
+        loads = [sum(steps(u) for u in range(a, b)) for a, b in zip(starts, starts[1:])]
+        assert all(steps(u) >= 1 for u in range(min(total, 2 * T)))
+        mean = sum(loads) / G
+        assert max(loads) <= mean + Qt and min(loads) >= mean - Qt             # within one key tile's full cost of the mean
+    assert L.tlin_plan_backward_share_start(1, 1, 10, 20, 1, 0, 4) == -1       # N < W with the window rule
