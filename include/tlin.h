@@ -218,7 +218,9 @@ typedef struct {
                               focused attention and the generation window);
                               1: every CTA works through whole (b,h,query tile) problems, keys never split
                               (many query rows, short context: the restoring cross-attention of Section 3) */
-    int32_t reserved;
+    int32_t causal_window; /* the call's mask, N and W: the group boundaries of schedule 1 depend on them              */
+    int32_t n_keys;
+    int32_t n_queries;
 } tlin_fwd_plan;
 
 typedef struct {
@@ -236,7 +238,9 @@ int tlin_plan_decode(int B, int H, int L, int d, int num_sms, tlin_decode_plan* 
  * shares are balanced by the number of 128-row query tiles each key tile has to visit, which under the window rule falls
  * towards the end of a (b,h).  -1 on bad arguments. */
 int64_t tlin_plan_backward_share_start(int B, int H, int N, int W, int causal_window, int share, int n_shares);
-/* First unit of group g: floor(g * total_units / n_groups). */
+/* First unit of group g.  floor(g * total_units / n_groups), except under schedule 1 with the window rule: there a
+ * (b,h,query tile) problem costs the key tiles its rows may use (+2 for starting and finishing it), which grows with the
+ * query tile, and the groups share the problems by that cost when there are at least three problems per group. */
 int64_t tlin_plan_group_start(const tlin_fwd_plan* plan, int g);
 /* Mask predicate: may query i (0 <= i < W) use key j?  1 or 0. */
 int tlin_allowed(int64_t i, int64_t j, int64_t N, int64_t W, int causal_window);

@@ -29,7 +29,8 @@ class FwdPlan(ctypes.Structure):
                 ("key_tiles", ctypes.c_int32), ("n_groups", ctypes.c_int32), ("n_ctas", ctypes.c_int32),
                 ("total_units", ctypes.c_int64), ("uses_workspace", ctypes.c_int32),
                 ("tensor_path", ctypes.c_int32), ("workspace_bytes", ctypes.c_int64),
-                ("schedule", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("schedule", ctypes.c_int32), ("causal_window", ctypes.c_int32),
+                ("n_keys", ctypes.c_int32), ("n_queries", ctypes.c_int32)]
 
 
 class DecodePlan(ctypes.Structure):

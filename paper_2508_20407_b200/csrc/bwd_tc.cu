@@ -449,7 +449,7 @@ struct BCfg {
     static constexpr int kOffV = (4 + kKSlots) * kTileBytes;
     static constexpr int kOffBars = (4 + kKSlots + kVSlots) * kTileBytes;
     static constexpr int kNumBars = 11 + 2 * kKSlots + 2 * kVSlots;
-    static constexpr int kSmemBytes = kOffBars + kNumBars * 8 + 16;
+    static constexpr int kSmemBytes = kOffBars + kNumBars * 8 + 32;   // + TMEM slot, abort flag, unit range
     // TMEM columns: R0, R1 (S, then dP, then dS as bf16; 128 each), dQ0, dQ1 (D each)
     static constexpr uint32_t kColR = 0, kColDQ = 256;
     static constexpr int kThreads = 32 * 12;                   // warps 10 and 11 only lend their registers
@@ -462,7 +462,8 @@ struct BCfg {
 template <int D>
 __global__ void __launch_bounds__(BCfg<D>::kThreads, 1)
 bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do, const BwdParams p) {
+                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do, const BwdParams p,
+                 const __grid_constant__ GroupStarts starts) {
     using C = BCfg<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* sQ = smem + C::kOffQ;
@@ -531,7 +532,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (lane == 0) {
             uint32_t kit = 0, vit = 0, seg_idx = 0;
             bool ok = base_ok;
-            SegmentWalker walk(p);
+            SegmentWalker walk(p, starts);
             Segment s;
             while (ok && walk.next(s)) {
                 const int row0 = s.qt * kTileM;
@@ -610,7 +611,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         uint32_t kit = 0, vit = 0, seg_idx = 0;
         uint32_t n_step[2] = {0, 0};
         bool ok = base_ok;
-        SegmentWalker walk(p);
+        SegmentWalker walk(p, starts);
         Segment s;
         while (ok && walk.next(s)) {
             const int row0 = s.qt * kTileM;
@@ -687,7 +688,7 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint32_t tDQ = tmem_base + lane_addr + C::kColDQ + i * D;
         uint32_t n = 0, seg_idx = 0;
         bool ok = base_ok;
-        SegmentWalker walk(p);
+        SegmentWalker walk(p, starts);
         const int bh_first = (int)(walk.u / p.key_tiles);     // (b,h) of this CTA's first unit (used under schedule 0 only)
         Segment s;
         while (ok && walk.next(s)) {
@@ -892,7 +893,10 @@ int launch_d(const void* q, const void* k, const void* v, const void* out, const
     // dQ: the forward's plan
     BwdParams pb = p;
     pb.total_units = plan.total_units; pb.n_groups = plan.n_groups; pb.q_tiles = plan.q_tiles; pb.schedule = plan.schedule;
-    bwd_dq_tc_kernel<D><<<plan.n_ctas, BCfg<D>::kThreads, BCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mdo, pb);
+    if (plan.n_groups > kMaxGroups) return TLIN_ERR_UNSUPPORTED;
+    GroupStarts starts;
+    fwd_group_starts(plan, &starts);
+    bwd_dq_tc_kernel<D><<<plan.n_ctas, BCfg<D>::kThreads, BCfg<D>::kSmemBytes, st>>>(mq, mk, mv, mdo, pb, starts);
     TLIN_CUDA_CHECK(cudaGetLastError());
     count_launch(3);
     if (plan.uses_workspace) {

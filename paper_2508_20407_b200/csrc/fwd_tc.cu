@@ -91,7 +91,7 @@ struct Params {
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-              const __grid_constant__ CUtensorMap map_v, const Params p) {
+              const __grid_constant__ CUtensorMap map_v, const Params p, const __grid_constant__ GroupStarts starts) {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -152,7 +152,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             uint32_t it = 0;           // ring counter
             uint32_t seg_idx = 0;
             bool ok = true;
-            SegmentWalker walk(p);
+            SegmentWalker walk(p, starts);
             Segment s;
             while (ok && walk.next(s)) {
                 const int row0 = s.qt * kTileM;
@@ -228,7 +228,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 }
                 if (half == 1) commit_elected(&pv_done[i]);
             };
-            SegmentWalker walk(p);
+            SegmentWalker walk(p, starts);
             Segment s;
             while (ok && walk.next(s)) {
                 const int row0 = s.qt * kTileM;
@@ -299,7 +299,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         const uint32_t tO = tmem_base + lane_addr + C::kColO + i * D;
         uint32_t n = 0;     // tiles processed by this warpgroup (phase counter of s_full/p_full/pv_done)
         bool ok = true;
-        SegmentWalker walk(p);
+        SegmentWalker walk(p, starts);
         const int bh_first = (int)(walk.u / p.key_tiles);  // (b,h) of this CTA's first unit (used under schedule 0 only)
         Segment s;
         while (ok && walk.next(s)) {
@@ -631,7 +631,10 @@ int launch_d(const void* q, const void* k, const void* v, void* out, float* lse,
         attr_err = cudaFuncSetAttribute(fwd_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
     });
     TLIN_CUDA_CHECK(attr_err);
-    fwd_tc_kernel<D><<<plan.n_ctas, kThreads, C::kSmemBytes, st>>>(mq, mk, mv, p);
+    if (plan.n_groups > kMaxGroups) return TLIN_ERR_UNSUPPORTED;
+    GroupStarts starts;
+    fwd_group_starts(plan, &starts);
+    fwd_tc_kernel<D><<<plan.n_ctas, kThreads, C::kSmemBytes, st>>>(mq, mk, mv, p, starts);
     TLIN_CUDA_CHECK(cudaGetLastError());
     count_launch();
     if (plan.uses_workspace) {

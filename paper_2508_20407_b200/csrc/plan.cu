@@ -2,6 +2,8 @@
 // anything; what it fixes is the set of (query,key) pairs a call evaluates (Section 3, causal
 // rule; Appendix A, cost terms), and every function here is tested against that count.
 #include "tlin_internal.h"
+#include <algorithm>
+#include <vector>
 
 using namespace tlin;
 
@@ -25,12 +27,41 @@ extern "C" int tlin_tile_class(int64_t N, int64_t W, int causal_window, int tile
     return j1 < N ? 1 : 2;
 }
 
+void tlin::fwd_group_starts(const tlin_fwd_plan& plan, GroupStarts* starts) {
+    const int G = plan.n_groups;
+    const long long U = plan.total_units;
+    const bool by_cost = plan.schedule != 0 && plan.causal_window && plan.q_tiles > 1 && U >= 3LL * G;
+    if (!by_cost) {
+        for (int g = 0; g <= G; ++g) starts->u[g] = (long long)(((unsigned long long)g * (unsigned long long)U) / (unsigned)G);
+        return;
+    }
+    // prefix[n] = cost of the first n problems of a (b,h)
+    thread_local std::vector<long long> prefix;
+    prefix.assign((size_t)plan.q_tiles + 1, 0);
+    for (int qt = 0; qt < plan.q_tiles; ++qt)
+        prefix[qt + 1] = prefix[qt] + fwd_problem_cost(plan.n_keys, plan.n_queries, plan.key_tiles, qt);
+    const unsigned long long per_bh = (unsigned long long)prefix[plan.q_tiles];
+    const unsigned long long total = per_bh * (unsigned long long)(U / plan.q_tiles);
+    for (int g = 0; g < G; ++g) {
+        const unsigned long long target = ((unsigned long long)g * total) / (unsigned)G;
+        const unsigned long long bh = target / per_bh;
+        const long long rem = (long long)(target - bh * per_bh);
+        // smallest n with prefix[n] >= rem
+        const long long n = std::lower_bound(prefix.begin(), prefix.end(), rem) - prefix.begin();
+        starts->u[g] = (long long)bh * plan.q_tiles + n;
+    }
+    starts->u[G] = U;
+}
+
 extern "C" int64_t tlin_plan_group_start(const tlin_fwd_plan* plan, int g) {
     if (!plan || plan->n_groups <= 0) return 0;
     if (g <= 0) return 0;
     if (g >= plan->n_groups) return plan->total_units;
-    // total_units < 2^31 * 2^24 / n_groups bound: B*H*key_tiles fits comfortably in 63 bits after *g
-    return (int64_t)(((__int128)g * plan->total_units) / plan->n_groups);
+    if (!plan->tensor_path || plan->n_groups > kMaxGroups)      // CUDA-core path: one group per (b,h), equal counts
+        return (int64_t)(((unsigned long long)g * (unsigned long long)plan->total_units) / (unsigned)plan->n_groups);
+    GroupStarts starts;
+    fwd_group_starts(*plan, &starts);
+    return starts.u[g];
 }
 
 extern "C" int tlin_plan_forward(int B, int H, int N, int W, int d, int causal_window, int is_f32,
@@ -47,6 +78,9 @@ extern "C" int tlin_plan_forward(int B, int H, int N, int W, int d, int causal_w
     tlin_fwd_plan p = {};
     const int64_t bh = (int64_t)B * H;
     p.tensor_path = tc ? 1 : 0;
+    p.causal_window = causal_window;
+    p.n_keys = N;
+    p.n_queries = W;
     if (!tc) {
         p.tile_m = kSimtRows;
         p.tile_n = kSimtKeys;
@@ -61,6 +95,7 @@ extern "C" int tlin_plan_forward(int B, int H, int N, int W, int d, int causal_w
         *plan = p;
         return TLIN_OK;
     }
+    if (num_sms > kMaxGroups) num_sms = kMaxGroups;   // size of the table of group starts handed to the kernels
     p.tile_m = 256;            // two 128-row Q tiles per CTA
     p.tile_n = kTileN;
     p.q_tiles = (W + p.tile_m - 1) / p.tile_m;
@@ -85,10 +120,27 @@ extern "C" int tlin_plan_forward(int B, int H, int N, int W, int d, int causal_w
         const int64_t cost0 = waves0 * (per_group + 2 * segments0) + (splits0 ? 6 : 0);
         const int64_t problems = bh * p.q_tiles;
         const int64_t ctas1 = num_sms < problems ? num_sms : problems;
-        const int64_t cost1 = ((problems + ctas1 - 1) / ctas1) * ((int64_t)p.key_tiles + 2);
         const int64_t kv_bytes = 2 * bh * (int64_t)N * d * 2;
         const bool kv_in_l2 = p.q_tiles == 1 || kv_bytes <= (int64_t)64 << 20;
-        wide = kv_in_l2 && cost1 < cost0;
+        int64_t cost1 = ((problems + ctas1 - 1) / ctas1) * ((int64_t)p.key_tiles + 2);
+        bool allow1 = kv_in_l2;
+        if (causal_window && p.q_tiles > 1) {
+            // With the window rule a problem only needs the key tiles its rows may use, and under schedule 0 the CTAs of
+            // the early query tiles would idle while the last one finishes.  Problems are shared by cost (the same
+            // arithmetic as the kernel's); an indivisible problem can leave a CTA half its cost above the mean.  When K and
+            // V exceed L2 the tiles come from HBM at unrelated times: measured about 15 % slower per tile.
+            int64_t per_bh = 0, biggest = 0;
+            for (int qt = 0; qt < p.q_tiles; ++qt) {
+                const int64_t c = fwd_problem_cost(N, W, p.key_tiles, qt);
+                per_bh += c;
+                if (c > biggest) biggest = c;
+            }
+            cost1 = (per_bh * bh + ctas1 - 1) / ctas1 + (problems > ctas1 ? biggest / 2 : 0);
+            if (cost1 < biggest) cost1 = biggest;
+            if (!kv_in_l2) cost1 += cost1 * 15 / 100;
+            allow1 = true;
+        }
+        wide = allow1 && cost1 < cost0;
     }
     if (wide) {
         p.schedule = 1;
@@ -109,8 +161,10 @@ extern "C" int tlin_plan_forward(int B, int H, int N, int W, int d, int causal_w
     p.n_groups = (int32_t)groups;
     p.n_ctas = p.n_groups * p.q_tiles;
     p.uses_workspace = 0;
+    GroupStarts starts;
+    fwd_group_starts(p, &starts);
     for (int g = 1; g < p.n_groups; ++g)
-        if (tlin_plan_group_start(&p, g) % p.key_tiles != 0) { p.uses_workspace = 1; break; }
+        if (starts.u[g] % p.key_tiles != 0) { p.uses_workspace = 1; break; }
     // two partial slots per CTA (first and last segment of its unit range), each tile_m x (d + 1) floats
     p.workspace_bytes = p.uses_workspace ? (int64_t)p.n_ctas * 2 * p.tile_m * (d + 1) * (int64_t)sizeof(float) : 0;
     *plan = p;

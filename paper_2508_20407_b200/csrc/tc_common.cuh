@@ -19,15 +19,16 @@ constexpr int kTileM = 2 * kQTile;          // query rows per CTA
 // borders.  Schedule 1: the units are whole (b,h,q-tile pair) problems and a CTA takes a contiguous run of them.
 struct Segment { int bh, qt, t_begin, t_end; };
 
+// The first unit of every group comes from the host as a launch parameter (GroupStarts, in the constant bank).
 struct SegmentWalker {
     long long u, u1;
     int T, q_tiles, qt_fixed, schedule;
     template <class P>
-    __device__ SegmentWalker(const P& p) : T(p.key_tiles), q_tiles(p.q_tiles), schedule(p.schedule) {
+    __device__ SegmentWalker(const P& p, const GroupStarts& starts) : T(p.key_tiles), q_tiles(p.q_tiles), schedule(p.schedule) {
         const int g = schedule == 0 ? (int)(blockIdx.x / p.q_tiles) : (int)blockIdx.x;
         qt_fixed = schedule == 0 ? (int)(blockIdx.x - g * p.q_tiles) : 0;
-        u = (long long)(((unsigned long long)g * (unsigned long long)p.total_units) / (unsigned)p.n_groups);
-        u1 = (long long)(((unsigned long long)(g + 1) * (unsigned long long)p.total_units) / (unsigned)p.n_groups);
+        u = starts.u[g];
+        u1 = starts.u[g + 1];
     }
     __device__ bool next(Segment& s) {
         if (u >= u1) return false;

@@ -22,6 +22,25 @@ int* status_word();                    // device address of the error word (boun
 void count_launch(int n = 1);
 int forward_impl();
 
+// Work sharing of the tensor-core forward and dQ kernels.  The host works out the first unit of every group and passes the
+// table to the kernel as a launch parameter (the CTAs only index it).
+// Schedule 0 (units = (b,h,key tile)) and unmasked schedule 1 (units = (b,h,256-row query tile pair) problems, all of one
+// cost): equal counts, group g starts at floor(g * units / groups).  Schedule 1 with the window rule: problem qt may use
+// ceil((N-W+min(W,256(qt+1)))/128) key tiles; its cost is that number plus 2 (starting and finishing a problem), and, when there
+// are at least three problems per group, group g starts at the first problem at which the cost of the problems before it reaches
+// g/groups of the total (with fewer, the indivisible problems dominate and equal counts do as well).
+constexpr int kMaxGroups = 192;        // groups never exceed the SM count (148 on B200); the planner clamps to this
+struct GroupStarts { long long u[kMaxGroups + 1]; };   // u[g] = first unit of group g, u[n_groups] = total_units
+inline long long fwd_problem_cost(int N, int W, int key_tiles, int qt) {
+    long long rows_end = (long long)(qt + 1) * 256;
+    if (rows_end > W) rows_end = W;
+    long long tiles = ((long long)N - W + rows_end + 127) / 128;
+    if (tiles > key_tiles) tiles = key_tiles;
+    return tiles + 2;
+}
+// fills starts->u[0 .. plan.n_groups]; plan.n_groups <= kMaxGroups
+void fwd_group_starts(const tlin_fwd_plan& plan, GroupStarts* starts);
+
 // Work sharing of the tensor-core dK/dV kernel (host and device use the same arithmetic).  Units are (b,h,key tile) in that
 // order, key tiles of 128 keys, query tiles of 128 rows; with the window rule key tile t is visited by the query tiles from
 // floor(max(0, 128 t - (N-W)) / 128) on, so the last key tiles of a (b,h) cost fewer steps, down to one.  Share c of G starts at

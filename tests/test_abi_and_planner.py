@@ -102,7 +102,16 @@ def _check_plan(p, B, H, N, W, d, causal):
     starts = [tl.tlin_plan_group_start(p, g) for g in range(p.n_groups + 1)]
     assert starts[0] == 0 and starts[-1] == p.total_units
     sizes = np.diff(starts)
-    assert (sizes >= 1).all() and sizes.max() - sizes.min() <= 1
+    by_cost = p.schedule == 1 and causal and p.q_tiles > 1 and p.total_units >= 3 * p.n_groups
+    if by_cost:
+        # window rule, whole problems per CTA: problem qt may use ceil((N-W+min(W,256(qt+1)))/128) key tiles; the groups share
+        # the problems by that cost (+2 per problem), each within one problem of the mean
+        cost = [min(p.key_tiles, -(-(N - W + min(W, 256 * (qt + 1))) // 128)) + 2 for qt in range(p.q_tiles)]
+        loads = [sum(cost[u % p.q_tiles] for u in range(a, b)) for a, b in zip(starts, starts[1:])]
+        mean = sum(loads) / len(loads)
+        assert (sizes >= 0).all() and max(loads) <= mean + max(cost) and min(loads) >= mean - max(cost)
+    else:
+        assert (sizes >= 1).all() and sizes.max() - sizes.min() <= 1
     if p.schedule == 0:
         # unit = (b,h,key tile); a group is q_tiles CTAs (one per pair of query tiles) walking the same units
         assert p.total_units == B * H * p.key_tiles
