@@ -36,8 +36,8 @@ from paper_2508_20407_b200 import synth  # noqa: E402
 WORKLOADS = {"fwd128k": "cfg4_vlong", "fwd32k": "cfg3_long", "fwd8k": "cfg2_mid", "decode": "cfg5_decode",
              "restore": "restore_vlong", "inner_self": "inner_self", "inner_gen": "inner_gen",
              "bwd_chunk": "train_chunk", "bwd32k": "cfg3_long", "decode_fp8": "cfg5_decode",
-             "nsweep": "cfg3_long"}
-BACKWARD = ("bwd_chunk", "bwd32k")      # legs that time tlin_attn_backward on the named shape
+             "nsweep": "cfg3_long", "fwd_seq": "train_seq", "bwd_seq": "train_seq"}
+BACKWARD = ("bwd_chunk", "bwd32k", "bwd_seq")      # legs that time tlin_attn_backward on the named shape
 NOMINAL_BF16_TFLOPS, NOMINAL_HBM_GBS = 2250.0, 7700.0      # datasheet figures, reported beside the measured peaks
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -190,8 +190,8 @@ L2_BYTES = 126e6
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from one-pass ncu captures of these
 # very workloads.  To be set to None whenever the kernel changes.
-FWD_TRAFFIC = {"cfg4_vlong": (2177.07e6 + 19.71e6, "ncu, full workload, fwd_tc_kernel<128>"),
-               "cfg3_long": (544.86e6 + 10.74e6, "ncu, full workload, fwd_tc_kernel<128>")}
+FWD_TRAFFIC = {"cfg4_vlong": (2168.65e6 + 20.05e6, "ncu, full workload, fwd_tc_kernel<128>"),
+               "cfg3_long": (544.75e6 + 10.74e6, "ncu, full workload, fwd_tc_kernel<128>")}
 # decode: captured on a smaller cache (B8 H32, 4096 rows: 537.35 MB read + 3.9 MB written for 537.3 MB of cache) and
 # scaled by the cached rows of the timed steps; the kernel streams every cached byte once at any size
 DECODE_TRAFFIC_RATIO = (537.35 + 3.9) / 537.3
@@ -241,6 +241,13 @@ def cpu_baseline_decode(wl, kc_heads, vc_heads, q_new, k_new, v_new, pos, n_head
 
 
 # ----------------------------------------------------------------------------- GPU legs
+def allowed_pairs(wl):
+    """(query, key) pairs the attention rule lets through, per (b,h): the scores that enter the softmax."""
+    if wl.causal_window:
+        return wl.W * (wl.N - wl.W) + wl.W * (wl.W + 1) // 2
+    return wl.W * wl.N
+
+
 def fwd_bytes(wl):
     return 2 * (2 * wl.B * wl.H * wl.N * wl.d + 2 * wl.B * wl.H * wl.W * wl.d) + 4 * wl.B * wl.H * wl.W
 
@@ -262,7 +269,7 @@ def run_forward(wl, args, rank, world, device, peaks, with_cpu):
     flush = torch.empty(int(2.5 * L2_BYTES), dtype=torch.uint8, device=device) if fwd_bytes(wl) < 2 * L2_BYTES else None
     ms, clocks = time_steps(step, args.steps, args.warmup, world, device, sampler, flush)
     ms_step = ms / args.steps
-    flop = 4.0 * wl.B * wl.H * wl.W * wl.N * wl.d
+    flop = 4.0 * wl.B * wl.H * allowed_pairs(wl) * wl.d
     tflops = flop / (ms_step * 1e-3) / 1e12
     t_tensor = flop / (peaks["bf16_tflops"] * 1e12)
     t_hbm = fwd_bytes(wl) / (peaks["hbm_gbs"] * 1e9)
@@ -281,7 +288,7 @@ def run_forward(wl, args, rank, world, device, peaks, with_cpu):
         roof["frac_of_sustained_peak"] = tflops / peaks["bf16_tflops_sustained"]
     roof["nominal"] = dict(peak=NOMINAL_BF16_TFLOPS, unit="TFLOP/s", frac=tflops / NOMINAL_BF16_TFLOPS, note="datasheet dense bf16, context only")
     # second ceiling: one exponential per (query, key) pair; the special-function units retire 16 per clock and SM
-    exps = float(wl.B) * wl.H * wl.W * wl.N
+    exps = float(wl.B) * wl.H * allowed_pairs(wl)
     sfu_rate = 16.0 * 148 * 1.965e9
     roof["secondary"] = dict(bound="special-function unit", exponentials=exps, roofline_ms=exps / sfu_rate * 1e3,
                              note="16 ex2 per clock per SM x 148 SMs x 1965 MHz; the kernel evaluates 5/16 of them on the FMA pipe")
@@ -346,7 +353,7 @@ def run_backward(wl, args, rank, world, device, peaks):
     flush = torch.empty(int(2.5 * L2_BYTES), dtype=torch.uint8, device=device) if nbytes < 2 * L2_BYTES else None
     ms, clocks = time_steps(step, args.steps, args.warmup, world, device, sampler, flush)
     ms_step = ms / args.steps
-    flop = 10.0 * wl.B * wl.H * wl.W * wl.N * wl.d
+    flop = 10.0 * wl.B * wl.H * allowed_pairs(wl) * wl.d
     tflops = flop / (ms_step * 1e-3) / 1e12
     roof = dict(bound="tensor", achieved=tflops, peak=peaks["bf16_tflops"], unit="TFLOP/s", frac=tflops / peaks["bf16_tflops"],
                 traffic=None, algorithmic_bytes=nbytes, peak_source=peaks["source"] + " (burst)",
@@ -612,7 +619,7 @@ def main():
         main_res = runner(wl, args, rank, world, device, peaks, with_cpu)
     also = []
     if not args.only and world == 1:
-        for name in ("fwd32k", "decode", "restore", "inner_self", "inner_gen", "bwd_chunk", "bwd32k", "decode_fp8"):
+        for name in ("fwd32k", "decode", "restore", "inner_self", "inner_gen", "fwd_seq", "bwd_chunk", "bwd32k", "bwd_seq", "decode_fp8"):
             if name == args.workload:
                 continue
             torch.cuda.empty_cache()

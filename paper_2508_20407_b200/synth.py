@@ -158,6 +158,9 @@ WORKLOADS = {
     # --- training (forward + backward): the last of the 8 windows of a sliding-window pass (stride W_og = 1024) over
     # sequences of 8192 tokens: W_og window queries over the whole sequence so far, causal inside the window
     "train_chunk": _w("train_chunk", 4, 32, 128, 8192, 1024, 8, causal_window=1),
+    # plain causal attention of a whole 4096-token sequence over itself (N = W): the layer of the standard architecture
+    # the paper compares with, and the window rule at its widest (half of the rectangle is masked)
+    "train_seq": _w("train_seq", 4, 32, 128, 4096, 4096, 10, causal_window=1),
 }
 
 Q_ID, K_ID, V_ID, QNEW_ID, KNEW_ID, VNEW_ID = 0, 1, 2, 3, 4, 5

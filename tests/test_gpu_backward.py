@@ -182,20 +182,22 @@ def test_backward_f32(B, H, N, W, d, causal):
             assert e["rel_l2"] <= 1e-4, f"{name}: rel L2 {e['rel_l2']:.3e}"
 
 
-def test_backward_at_the_benchmarked_training_shape_on_two_heads():
-    # the full train_chunk workload (B4 H32 N8192 W1024 d128, the launch configuration bench.py times); the oracle
-    # recomputes two (b,h) pairs of it, which are independent problems
-    wl = synth.WORKLOADS["train_chunk"]
+@pytest.mark.parametrize("name,heads", [("train_chunk", ((0, 0), (3, 17))), ("train_seq", ((2, 9),))])
+def test_backward_at_the_benchmarked_training_shapes_on_sampled_heads(name, heads):
+    # the full workloads bench.py times (train_chunk: B4 H32 N8192 W1024, the last window of a sliding-window pass;
+    # train_seq: B4 H32 N=W=4096, a whole sequence over itself, where the CTAs share whole problems by cost); the
+    # oracle recomputes sampled (b,h) pairs, which are independent problems
+    wl = synth.WORKLOADS[name]
     q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
     g = torch.Generator(device="cpu").manual_seed(wl.seed + 99)
     dout = torch.randn(q.shape, generator=g, dtype=torch.float32).to(torch.bfloat16).to(DEV)
     dq, dk, dv = grads(q, k, v, dout, wl.causal_window, 0)
-    for b, h in ((0, 0), (3, 17)):
+    for b, h in heads:
         sl = (slice(b, b + 1), slice(h, h + 1))
         rq, rk, rv = oracle.attn_backward(q[sl].cpu(), k[sl].cpu(), v[sl].cpu(), dout[sl].cpu(), wl.causal_window)
-        compare(dq[sl], rq, f"train_chunk b{b} h{h} dq")
-        compare(dk[sl], rk, f"train_chunk b{b} h{h} dk")
-        compare(dv[sl], rv, f"train_chunk b{b} h{h} dv")
+        compare(dq[sl], rq, f"{name} b{b} h{h} dq")
+        compare(dk[sl], rk, f"{name} b{b} h{h} dk")
+        compare(dv[sl], rv, f"{name} b{b} h{h} dv")
 
 
 @pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 128), (torch.float32, 36)])

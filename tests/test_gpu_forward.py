@@ -217,6 +217,17 @@ def test_full_size_sampled_rows(name, causal):
     sampled_rows_compare(wl, impl, 6, [(0, 0), (0, wl.H // 2), (0, wl.H - 1)], causal)
 
 
+def test_whole_sequence_causal_attention_sampled_rows():
+    # N = W = 4096 over B4 H32: whole (b,h,query tile) problems per CTA, shared between the CTAs by cost, so a CTA's
+    # run of problems crosses (b,h) borders; rows sampled in the first, a middle and the last (b,h)
+    wl = synth.WORKLOADS["train_seq"]
+    impl = 2 if TC_AVAILABLE else 1
+    plan = tl.tlin_plan_forward(wl.B, wl.H, wl.N, wl.W, wl.d, 1)
+    if impl == 2:
+        assert plan.schedule == 1 and plan.uses_workspace == 0
+    sampled_rows_compare(wl, impl, 14, [(0, 0), (1, 17), (wl.B - 1, wl.H - 1)], 1)
+
+
 def test_chunk_scheduled_forward_equals_per_chunk_calls_and_full_causal_attention():
     # Sliding-window training (Section 5.1): C windows of W tokens, window c attends to everything up to its own end.
     # One call over shared k, v; each chunk must equal the oracle on the key prefix, and the chunks laid end to end are
