@@ -57,34 +57,53 @@ struct BwdParams {
 };
 
 // ------------------------------------------------------------------------------------------ preparation
+// Row statistics of the backward pass: lse2 = lse * log2(e) and delta = sum_c out*dout, on rows padded to 128 per (b,h)
+// (padding rows: +inf and 0).  D/8 lanes share a row with one 16-byte load per tensor each; a warp keeps kPrepPasses
+// groups of rows in flight, so that enough bytes are outstanding to stream at HBM speed.
+constexpr int kPrepPasses = 4;
+template <int D>
+__host__ __device__ constexpr int prep_rows_per_block() { return 8 * (32 / (D / 8)) * kPrepPasses; }
+
 template <int D>
 __global__ void __launch_bounds__(256)
 bwd_prep_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout, const float* __restrict__ lse,
                 float* __restrict__ lse2, float* __restrict__ delta, int W, int Wpad, long long rows_padded) {
-    const long long prow = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (prow >= rows_padded) return;
-    const int lane = threadIdx.x & 31;
-    const long long bh = prow / Wpad;
-    const int i = (int)(prow - bh * Wpad);
-    if (i >= W) {
-        if (lane == 0) {
-            lse2[prow] = CUDART_INF_F;
-            delta[prow] = 0.f;
+    constexpr int LPR = D / 8;              // lanes per row
+    constexpr int RPP = 32 / LPR;           // rows per pass of a warp
+    const int lane = threadIdx.x & 31, sub = lane / LPR, l = lane % LPR;
+    const long long first = ((long long)blockIdx.x * 8 + (threadIdx.x >> 5)) * (RPP * kPrepPasses) + sub;
+    uint4 a[kPrepPasses], b[kPrepPasses];
+    long long row[kPrepPasses];
+#pragma unroll
+    for (int ps = 0; ps < kPrepPasses; ++ps) {
+        const long long prow = first + ps * RPP;
+        const long long bh = prow / Wpad;
+        const int i = (int)(prow - bh * Wpad);
+        row[ps] = (prow < rows_padded && i < W) ? bh * W + i : -1;
+        a[ps] = b[ps] = make_uint4(0u, 0u, 0u, 0u);
+        if (row[ps] >= 0) {
+            a[ps] = *reinterpret_cast<const uint4*>(out + row[ps] * D + l * 8);
+            b[ps] = *reinterpret_cast<const uint4*>(dout + row[ps] * D + l * 8);
         }
-        return;
-    }
-    const long long row = bh * W + i;
-    float acc = 0.f;
-    for (int c = lane * 2; c < D; c += 64) {
-        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(out + row * D + c));
-        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(dout + row * D + c));
-        acc = fmaf(a.x, b.x, fmaf(a.y, b.y, acc));
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) {
-        lse2[prow] = lse[row] * kLog2e;
-        delta[prow] = acc;
+    for (int ps = 0; ps < kPrepPasses; ++ps) {
+        const uint32_t* aw = reinterpret_cast<const uint32_t*>(&a[ps]);
+        const uint32_t* bw = reinterpret_cast<const uint32_t*>(&b[ps]);
+        float acc = 0.f;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw[e]));
+            const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw[e]));
+            acc = fmaf(x.x, y.x, fmaf(x.y, y.y, acc));
+        }
+#pragma unroll
+        for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        const long long prow = first + ps * RPP;
+        if (l == 0 && prow < rows_padded) {
+            lse2[prow] = row[ps] >= 0 ? lse[row[ps]] * kLog2e : CUDART_INF_F;
+            delta[prow] = row[ps] >= 0 ? acc : 0.f;
+        }
     }
 }
 
@@ -880,7 +899,7 @@ int launch_d(const void* q, const void* k, const void* v, const void* out, const
     });
     TLIN_CUDA_CHECK(attr_err);
     const long long rows_padded = bh * Wpad;
-    bwd_prep_kernel<D><<<(unsigned)((rows_padded + 7) / 8), 256, 0, st>>>(
+    bwd_prep_kernel<D><<<(unsigned)((rows_padded + prep_rows_per_block<D>() - 1) / prep_rows_per_block<D>()), 256, 0, st>>>(
         (const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse, lse2, delta, W, Wpad, rows_padded);
     TLIN_CUDA_CHECK(cudaGetLastError());
     // dK, dV: the units are (b,h,key tile); a CTA takes a contiguous run of them
