@@ -92,7 +92,9 @@ def test_backward_peaked_softmax(impl):
 # many CTAs per (b,h) on the dQ side (key range split between groups, partial sums added by the reduce kernel), several
 # key tiles per CTA on the dK/dV side, both schedules of the plan
 BIG = [(1, 2, 40000, 300, 128, 1), (2, 3, 20000, 520, 64, 1), (1, 160, 384, 512, 64, 0), (6, 16, 1024, 1000, 64, 1),
-       (1, 1, 30000, 1024, 128, 0)]
+       (1, 1, 30000, 1024, 128, 0),
+       # the dQ kernel on a plan whose CTAs share whole problems by cost (window rule, >= three problems per CTA)
+       (2, 40, 1600, 1500, 128, 1), (3, 50, 900, 900, 64, 1)]
 
 
 @pytest.mark.parametrize("B,H,N,W,d,causal", BIG)
