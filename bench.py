@@ -39,6 +39,7 @@ WORKLOADS = {"fwd128k": "cfg4_vlong", "fwd32k": "cfg3_long", "fwd8k": "cfg2_mid"
              "nsweep": "cfg3_long", "fwd_seq": "train_seq", "bwd_seq": "train_seq"}
 BACKWARD = ("bwd_chunk", "bwd32k", "bwd_seq")      # legs that time tlin_attn_backward on the named shape
 NOMINAL_BF16_TFLOPS, NOMINAL_HBM_GBS = 2250.0, 7700.0      # datasheet figures, reported beside the measured peaks
+REFERENCE_BUDGET_S = 100.0     # --impl reference: target duration of all its steps together
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -542,9 +543,28 @@ def run_reference(args, rank, world):
         value, unit, metric = gb / t_full, "GB/s", "decode_kv_GB_per_s"
         sample = f"one decode step at pos={wl.N} for {n_heads} of {wl.B * wl.H} (b,h) pairs per step, scaled"
     else:
-        rows = max(cores, 8)
-        q, k, v = synth.forward_inputs_head(wl, 0, 0, q_rows=slice(wl.W - rows, wl.W))
-        q, k, v = q.view(1, 1, rows, wl.d), k.view(1, 1, wl.N, wl.d), v.view(1, 1, wl.N, wl.d)
+        # Rows per step: as many of the head's last query rows as keep the whole run near REFERENCE_BUDGET_S.  Two untimed
+        # probes (16 and 128 rows) give the oracle's fixed cost per call (the fp64 copies of K and V) and its cost per row;
+        # few rows per call would charge the fixed cost to every row and understate the oracle.
+        def head_rows(rows):
+            q, k, v = synth.forward_inputs_head(wl, 0, 0, q_rows=slice(wl.W - rows, wl.W))
+            return q.view(1, 1, rows, wl.d), k.view(1, 1, wl.N, wl.d), v.view(1, 1, wl.N, wl.d)
+
+        def probe(rows):
+            q, k, v = head_rows(rows)
+            t0 = time.perf_counter()
+            oracle.attn_forward(q, k, v, wl.causal_window)
+            return time.perf_counter() - t0
+
+        r_lo, r_hi = min(16, wl.W), min(128, wl.W)
+        probe(r_lo)                                         # first touch of the library and the thread pool
+        t_lo, t_hi = probe(r_lo), probe(r_hi)
+        per_row = max((t_hi - t_lo) / max(r_hi - r_lo, 1), 1e-6)
+        fixed = max(t_lo - per_row * r_lo, 0.0)
+        per_step = REFERENCE_BUDGET_S / max(args.warmup + args.steps, 1)
+        rows = int(min(wl.W, max(8, (per_step - fixed) / per_row)))
+        rows = max(8, rows // 8 * 8) if rows < wl.W else wl.W
+        q, k, v = head_rows(rows)
         times = []
         for i in range(args.warmup + args.steps):
             t0 = time.perf_counter()
