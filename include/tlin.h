@@ -240,7 +240,8 @@ int tlin_plan_decode(int B, int H, int L, int d, int num_sms, tlin_decode_plan* 
 int64_t tlin_plan_backward_share_start(int B, int H, int N, int W, int causal_window, int share, int n_shares);
 /* First unit of group g.  floor(g * total_units / n_groups), except under schedule 1 with the window rule: there a
  * (b,h,query tile) problem costs the key tiles its rows may use (+2 for starting and finishing it), which grows with the
- * query tile, and the groups share the problems by that cost when there are at least three problems per group. */
+ * query tile, and when there are at least three problems per group the groups take contiguous runs of problems whose
+ * costliest run is as cheap as contiguous runs allow (long problems) and which stay close to equal shares of the cost. */
 int64_t tlin_plan_group_start(const tlin_fwd_plan* plan, int g);
 /* Mask predicate: may query i (0 <= i < W) use key j?  1 or 0. */
 int tlin_allowed(int64_t i, int64_t j, int64_t N, int64_t W, int causal_window);

@@ -40,15 +40,54 @@ void tlin::fwd_group_starts(const tlin_fwd_plan& plan, GroupStarts* starts) {
     prefix.assign((size_t)plan.q_tiles + 1, 0);
     for (int qt = 0; qt < plan.q_tiles; ++qt)
         prefix[qt + 1] = prefix[qt] + fwd_problem_cost(plan.n_keys, plan.n_queries, plan.key_tiles, qt);
-    const unsigned long long per_bh = (unsigned long long)prefix[plan.q_tiles];
-    const unsigned long long total = per_bh * (unsigned long long)(U / plan.q_tiles);
-    for (int g = 0; g < G; ++g) {
-        const unsigned long long target = ((unsigned long long)g * total) / (unsigned)G;
-        const unsigned long long bh = target / per_bh;
-        const long long rem = (long long)(target - bh * per_bh);
-        // smallest n with prefix[n] >= rem
-        const long long n = std::lower_bound(prefix.begin(), prefix.end(), rem) - prefix.begin();
-        starts->u[g] = (long long)bh * plan.q_tiles + n;
+    const long long q = plan.q_tiles, n_bh = U / q, per_bh = prefix[q], total = per_bh * n_bh;
+    long long biggest = 0;
+    for (int qt = 0; qt < q; ++qt) biggest = std::max(biggest, prefix[qt + 1] - prefix[qt]);
+    // The costs repeat with every (b,h): P(x) = cost of the first x problems, and its two inverses
+    auto P = [&](long long x) { return (x / q) * per_bh + prefix[x % q]; };
+    auto last_le = [&](long long v) {        // largest x <= U with P(x) <= v   (v >= 0)
+        const long long bh = v / per_bh;
+        if (bh >= n_bh) return U;
+        return bh * q + ((std::upper_bound(prefix.begin(), prefix.end(), v - bh * per_bh) - prefix.begin()) - 1);
+    };
+    auto first_ge = [&](long long v) {       // smallest x >= 0 with P(x) >= v   (v <= total)
+        if (v <= 0) return 0LL;
+        const long long bh = v / per_bh;
+        return bh * q + (long long)(std::lower_bound(prefix.begin(), prefix.end(), v - bh * per_bh) - prefix.begin());
+    };
+    auto proportional = [&](int g) {         // group g starts where the cost before it reaches g/G of the total
+        return first_ge((long long)(((unsigned long long)g * (unsigned long long)total) / (unsigned)G));
+    };
+    starts->u[G] = U;
+    if (per_bh < 10 * q) {
+        // short problems (10 key-tile times on average, overheads included): the cost model is too coarse for more than
+        // the proportional split (measured: the exact optimum below is 5-10 % slower at N = W = 1024, 3-8 % faster from 2048 on)
+        for (int g = 0; g < G; ++g) starts->u[g] = proportional(g);
+        return;
+    }
+    // G contiguous runs, none costlier than cap: possible iff filling every run to the brim reaches the end
+    auto feasible = [&](long long cap) {
+        long long pos = 0;
+        for (int g = 0; g < G && pos < U; ++g) pos = last_le(P(pos) + cap);
+        return pos >= U;
+    };
+    // the slowest CTA decides the kernel's time: smallest cap that works (between the mean and one problem above it)
+    long long cap = std::max(biggest, (total + G - 1) / G), hi = (total + G - 1) / G + biggest;
+    while (cap < hi) {
+        const long long mid = (cap + hi) / 2;
+        if (feasible(mid)) hi = mid; else cap = mid + 1;
+    }
+    // Among the splits that respect cap, stay as close as possible to the proportional one (group g starting where the cost
+    // before it reaches g/G of the total), so that no CTA is left without work when it can be helped.  earliest[g]: first
+    // problem group g may start at such that the groups from g on can still take the rest.
+    long long earliest[kMaxGroups + 1];
+    earliest[G] = U;
+    for (int g = G - 1; g >= 0; --g) earliest[g] = first_ge(P(earliest[g + 1]) - cap);
+    starts->u[0] = 0;
+    for (int g = 0; g + 1 < G; ++g) {
+        const long long from = starts->u[g];
+        const long long lo = std::max(earliest[g + 1], from), up = last_le(P(from) + cap);
+        starts->u[g + 1] = std::min(std::max(proportional(g + 1), lo), up);
     }
     starts->u[G] = U;
 }

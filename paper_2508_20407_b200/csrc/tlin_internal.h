@@ -27,8 +27,10 @@ int forward_impl();
 // Schedule 0 (units = (b,h,key tile)) and unmasked schedule 1 (units = (b,h,256-row query tile pair) problems, all of one
 // cost): equal counts, group g starts at floor(g * units / groups).  Schedule 1 with the window rule: problem qt may use
 // ceil((N-W+min(W,256(qt+1)))/128) key tiles; its cost is that number plus 2 (starting and finishing a problem), and, when there
-// are at least three problems per group, group g starts at the first problem at which the cost of the problems before it reaches
-// g/groups of the total (with fewer, the indivisible problems dominate and equal counts do as well).
+// are at least three problems per group, the groups take contiguous runs of problems by cost: every group starting where the
+// cost before it reaches its share of the total, and, for problems of 10 key-tile times or more on average, moved as little
+// as needed to make the costliest run as cheap as contiguous runs allow (with fewer than three problems per group the
+// indivisible problems dominate and equal counts do as well).
 constexpr int kMaxGroups = 192;        // groups never exceed the SM count (148 on B200); the planner clamps to this
 struct GroupStarts { long long u[kMaxGroups + 1]; };   // u[g] = first unit of group g, u[n_groups] = total_units
 inline long long fwd_problem_cost(int N, int W, int key_tiles, int qt) {

@@ -104,12 +104,32 @@ def _check_plan(p, B, H, N, W, d, causal):
     sizes = np.diff(starts)
     by_cost = p.schedule == 1 and causal and p.q_tiles > 1 and p.total_units >= 3 * p.n_groups
     if by_cost:
-        # window rule, whole problems per CTA: problem qt may use ceil((N-W+min(W,256(qt+1)))/128) key tiles; the groups share
-        # the problems by that cost (+2 per problem), each within one problem of the mean
+        # window rule, whole problems per CTA: problem qt may use ceil((N-W+min(W,256(qt+1)))/128) key tiles; the groups take
+        # contiguous runs of problems, and the costliest run (cost = tiles + 2 per problem) must be the optimum over all ways
+        # of cutting the list into n_groups runs, found here by bisection over a plain greedy pass
         cost = [min(p.key_tiles, -(-(N - W + min(W, 256 * (qt + 1))) // 128)) + 2 for qt in range(p.q_tiles)]
-        loads = [sum(cost[u % p.q_tiles] for u in range(a, b)) for a, b in zip(starts, starts[1:])]
-        mean = sum(loads) / len(loads)
-        assert (sizes >= 0).all() and max(loads) <= mean + max(cost) and min(loads) >= mean - max(cost)
+        all_costs = cost * (p.total_units // p.q_tiles)
+        loads = [sum(all_costs[a:b]) for a, b in zip(starts, starts[1:])]
+
+        def runs_needed(cap):
+            n, cur = 1, 0
+            for c in all_costs:
+                if cur + c > cap:
+                    n, cur = n + 1, c
+                else:
+                    cur += c
+            return n
+
+        lo, hi = max(cost), sum(all_costs)
+        while lo < hi:
+            mid = (lo + hi) // 2
+            lo, hi = (lo, mid) if runs_needed(mid) <= p.n_groups else (mid + 1, hi)
+        mean = sum(all_costs) / p.n_groups
+        assert (sizes >= 0).all() and lo <= mean + max(cost)
+        if sum(cost) >= 10 * p.q_tiles:
+            assert max(loads) == lo and min(loads) > 0
+        else:       # short problems: every group starts where the cost before it reaches its share of the total
+            assert max(loads) <= mean + max(cost) and min(loads) >= mean - max(cost)
     else:
         assert (sizes >= 1).all() and sizes.max() - sizes.min() <= 1
     if p.schedule == 0:
@@ -141,7 +161,10 @@ def test_forward_plan_partitions_the_units(B, H, N, W, d, causal):
 
 
 WIDE = [(1, 32, 1024, 130048, 128, 0), (1, 32, 512, 32256, 128, 0), (2, 3, 300, 40000, 64, 0), (8, 16, 1024, 1024, 64, 1),
-        (1, 32, 1024, 1024, 128, 0), (1, 32, 2048, 1024, 128, 1)]
+        (1, 32, 1024, 1024, 128, 0), (1, 32, 2048, 1024, 128, 1),
+        # plain causal attention over whole sequences: problems of very different cost, shared between the CTAs by cost
+        (4, 32, 4096, 4096, 128, 1), (1, 32, 8192, 8192, 128, 1), (1, 8, 16384, 16384, 128, 1), (2, 40, 1600, 1500, 128, 1),
+        (3, 50, 900, 900, 64, 1), (4, 32, 4096, 2048, 128, 1)]
 
 
 @pytest.mark.parametrize("B,H,N,W,d,causal", WIDE)
