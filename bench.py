@@ -187,6 +187,15 @@ def time_steps(step_fn, steps, warmup, world, device, sampler=None, flush_buf=No
     return max_over_ranks(ms, world, device), clocks
 
 
+def sustained_leg(step_fn, ms_step, world, device, rank, seconds=1.2):
+    """The same call repeated back to back for about `seconds` inside one pair of events (its own loop, beside the
+    timed steps), with the SM clock sampled meanwhile: the figure a long-running job sees once the power cap acts."""
+    n = max(3, int(seconds * 1e3 / max(ms_step, 1e-3)) + 1)
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    ms, clocks = time_steps(step_fn, n, 3, world, device, sampler)
+    return ms / n, n, clocks
+
+
 L2_BYTES = 126e6
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from one-pass ncu captures of these
@@ -270,6 +279,7 @@ def run_forward(wl, args, rank, world, device, peaks, with_cpu):
     flush = torch.empty(int(2.5 * L2_BYTES), dtype=torch.uint8, device=device) if fwd_bytes(wl) < 2 * L2_BYTES else None
     ms, clocks = time_steps(step, args.steps, args.warmup, world, device, sampler, flush)
     ms_step = ms / args.steps
+    timed_launches = int(sum(launches[args.warmup:args.warmup + args.steps]))
     flop = 4.0 * wl.B * wl.H * allowed_pairs(wl) * wl.d
     tflops = flop / (ms_step * 1e-3) / 1e12
     t_tensor = flop / (peaks["bf16_tflops"] * 1e12)
@@ -293,6 +303,17 @@ def run_forward(wl, args, rank, world, device, peaks, with_cpu):
     sfu_rate = 16.0 * 148 * 1.965e9
     roof["secondary"] = dict(bound="special-function unit", exponentials=exps, roofline_ms=exps / sfu_rate * 1e3,
                              note="16 ex2 per clock per SM x 148 SMs x 1965 MHz; the kernel evaluates 5/16 of them on the FMA pipe")
+
+    if getattr(args, "sustained", False) and flush is None:
+        ms_s, n_s, clk_s = sustained_leg(step, ms_step, world, device, rank)
+        tf_s = flop / (ms_s * 1e-3) / 1e12
+        mhz = clk_s["sm_mhz"] if clk_s else None
+        roof["sustained"] = dict(calls=n_s, seconds=ms_s * n_s * 1e-3, ms_per_step=ms_s, achieved=tf_s, unit="TFLOP/s",
+                                 frac_of_burst_peak=tf_s / peaks["bf16_tflops"],
+                                 frac_of_sustained_peak=tf_s / peaks["bf16_tflops_sustained"] if "bf16_tflops_sustained" in peaks else None,
+                                 sm_mhz=mhz, reasons=clk_s["reasons"] if clk_s else [],
+                                 ms_times_mhz=ms_s * mhz if mhz else None,
+                                 ms_times_mhz_of_timed_steps=ms_step * clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None)
 
     # end to end: pinned host buffers through the host entry point
     e2e = None
@@ -319,7 +340,7 @@ def run_forward(wl, args, rank, world, device, peaks, with_cpu):
     res = dict(workload=wl.name, shape=dict(B=wl.B, H=wl.H, N=wl.N, W=wl.W, d=wl.d, causal_window=wl.causal_window), l2=l2_note,
                ms_per_step=ms_step, tokens_per_s=world * wl.B * wl.N / (ms_step * 1e-3),
                tflops=tflops, roofline=roof, e2e=e2e, clocks=clocks,
-               gpu_launches=int(sum(launches[args.warmup:])), launches_per_step=launches[-1] if launches else 0)
+               gpu_launches=timed_launches, launches_per_step=launches[-1] if launches else 0)
 
     if with_cpu and rank == 0:
         tl.tlin_attn_forward(q, k, v, out, lse, wl.causal_window)
@@ -401,6 +422,16 @@ def run_decode(wl, args, rank, world, device, peaks, with_cpu):
                 peak_source=peaks["source"], kernel="decode (split-K kernel + merge)",
                 roofline_ms=tot / steps / (peaks["hbm_gbs"] * 1e9) * 1e3,
                 nominal=dict(peak=NOMINAL_HBM_GBS, unit="GB/s", frac=gbs / NOMINAL_HBM_GBS, note="datasheet HBM3e, context only"))
+    timed_launches = int(sum(launches[args.warmup:args.warmup + steps]))
+    if getattr(args, "sustained", False):
+        # steady state at the last position of the window, back to back for about a second
+        fixed = lambda _i: tl.tlin_decode_step(qn[wl.W - 1], kn[wl.W - 1], vn[wl.W - 1], kc, vc, wl.N + wl.W - 1, out, lse)
+        ms_s, n_s, clk_s = sustained_leg(fixed, ms_step, world, device, rank)
+        b_s = 2 * wl.B * wl.H * (wl.N + wl.W) * wl.d * 2 + 4 * wl.B * wl.H * wl.d * 2 + 4 * wl.B * wl.H
+        gb_s = b_s / (ms_s * 1e-3) / 1e9
+        roof["sustained"] = dict(calls=n_s, seconds=ms_s * n_s * 1e-3, ms_per_step=ms_s, achieved=gb_s, unit="GB/s",
+                                 frac=gb_s / peaks["hbm_gbs"], sm_mhz=clk_s["sm_mhz"] if clk_s else None,
+                                 reasons=clk_s["reasons"] if clk_s else [])
     e2e = None
     if not args.no_e2e:
         host = [t.cpu().pin_memory() for t in (qn, kn, vn)]
@@ -420,7 +451,7 @@ def run_decode(wl, args, rank, world, device, peaks, with_cpu):
                    d2h_bytes_per_step=nb + wl.B * wl.H * 4, ms_per_step=ms_e / n_e2e, steps=n_e2e)
     res = dict(workload=wl.name, ms_per_step=ms_step, gb_per_s=world * gbs, steps=steps,
                decode_tokens_per_s=world * wl.B / (ms_step * 1e-3), roofline=roof, e2e=e2e, clocks=clocks,
-               gpu_launches=int(sum(launches[args.warmup:])), launches_per_step=launches[-1] if launches else 0)
+               gpu_launches=timed_launches, launches_per_step=launches[-1] if launches else 0)
     if with_cpu and rank == 0:
         n_heads = 8
         t = 0
@@ -577,11 +608,41 @@ def run_reference(args, rank, world):
     return {"impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_full * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "W": wl.W, "d": wl.d,
-                       "causal_window": wl.causal_window},
+            "config": config_of(wl, max(world, 1)),
             "cpu_baseline": {"value": value, "unit": unit, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
+
+
+def config_of(wl, world):
+    """The `config` object of the JSON line; both arms (this library and the oracle) print the same one."""
+    if wl.decode:
+        kv = 4e-6 * wl.B * wl.H * wl.N * wl.d
+        l2 = "cached K+V %.0f MB > L2 (126 MB): steps back to back, no flush" % kv
+    elif fwd_bytes(wl) < 2 * L2_BYTES:
+        l2 = ("inputs+outputs %.0f MB: a %.0f MB buffer is overwritten before every timed call (L2 flush), calls timed one by one"
+              % (fwd_bytes(wl) / 1e6, int(2.5 * L2_BYTES) / 1e6))
+    else:
+        l2 = "inputs+outputs %.0f MB > 2 x L2 (126 MB): back-to-back calls, no flush" % (fwd_bytes(wl) / 1e6)
+    return {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "W": wl.W, "d": wl.d, "causal_window": wl.causal_window,
+            "parallelism": f"replicas x{world}", "l2": l2}
+
+
+def compact_leg(leg):
+    """An 'also' leg without the long descriptive fields (the headline keeps them): what was run, its time, the
+    roofline figures and the clocks."""
+    r = leg["roofline"]
+    roof = {k: r[k] for k in ("bound", "achieved", "peak", "unit", "frac", "frac_of_sustained_peak", "traffic", "algorithmic_bytes",
+                              "executed_over_counted_flops", "sustained") if k in r}
+    c = leg.get("clocks") or {}
+    out = {k: leg[k] for k in ("workload", "shape", "ms_per_step", "tflops", "gb_per_s", "tokens_per_s", "decode_tokens_per_s", "steps",
+                               "gpu_launches", "launches_per_step") if k in leg}
+    out["roofline"] = roof
+    out["clocks"] = {"sm_mhz": c.get("sm_mhz"), "sm_max_mhz": c.get("sm_max_mhz"), "reasons": c.get("reasons", [])}
+    if leg.get("e2e"):
+        out["e2e"] = leg["e2e"]
+    out["l2_flush"] = "between calls" if "flush" in leg.get("l2", "") and "no flush" not in leg.get("l2", "") else "inputs larger than L2"
+    return out
 
 
 # ----------------------------------------------------------------------------- main
@@ -595,6 +656,8 @@ def main():
     ap.add_argument("--only", action="store_true", help="time only --workload (no 'also' legs)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-sustained", dest="sustained", action="store_false",
+                    help="skip the back-to-back loops of about a second on the workloads with a target")
     ap.add_argument("--decode-steps", type=int, default=0, help="timed decode steps (default: max(steps, 64))")
     ap.add_argument("--shape", default="", help="custom shape B,H,N,W,d[,causal] instead of the named workload (profiling); with --workload decode, N is the "
                          "number of cached rows and W the number of decode steps available")
@@ -638,6 +701,7 @@ def main():
         runner = run_decode if wl.decode else run_forward
         main_res = runner(wl, args, rank, world, device, peaks, with_cpu)
     also = []
+    full_legs = {args.workload: main_res}
     if not args.only and world == 1:
         for name in ("fwd32k", "decode", "restore", "inner_self", "inner_gen", "fwd_seq", "bwd_chunk", "bwd32k", "bwd_seq", "decode_fp8"):
             if name == args.workload:
@@ -647,12 +711,15 @@ def main():
             w2 = synth.WORKLOADS[WORKLOADS[name]]
             a2 = argparse.Namespace(**vars(args))
             a2.no_e2e = args.no_e2e or name not in ("fwd32k", "decode")     # host-buffer legs only where they are cheap to set up
+            a2.sustained = args.sustained and name in ("fwd32k", "decode")  # the legs with a stated target
             if name in BACKWARD:
-                also.append(run_backward(w2, a2, rank, world, device, peaks))
+                leg = run_backward(w2, a2, rank, world, device, peaks)
             elif name == "decode_fp8":
-                also.append(run_decode_fp8(w2, a2, rank, world, device, peaks))
+                leg = run_decode_fp8(w2, a2, rank, world, device, peaks)
             else:
-                also.append((run_decode if w2.decode else run_forward)(w2, a2, rank, world, device, peaks, False))
+                leg = (run_decode if w2.decode else run_forward)(w2, a2, rank, world, device, peaks, False)
+            full_legs[name] = leg
+            also.append(compact_leg(leg))
 
     if rank == 0:
         if args.workload in BACKWARD:
@@ -661,19 +728,34 @@ def main():
             metric, unit, value = "decode_kv_GB_per_s", "GB/s", main_res["gb_per_s"]
         else:
             metric, unit, value = "context_tokens_per_s", "context tokens/s", main_res["tokens_per_s"]
+        # the three workloads with a stated target (>= 0.60 of the tensor roofline forward, >= 0.70 of the HBM roofline
+        # decode), in one compact object at the very end of the line
+        targets = {}
+        for key, leg_name, bar in (("cfg3", "fwd32k", 0.60), ("cfg4", "fwd128k", 0.60), ("cfg5", "decode", 0.70)):
+            leg = full_legs.get(leg_name)
+            if leg is None:
+                continue
+            r, c = leg["roofline"], leg.get("clocks") or {}
+            t = dict(ms_per_step=round(leg["ms_per_step"], 5), achieved=round(r["achieved"], 1), unit=r["unit"], peak=r["peak"],
+                     frac=round(r["frac"], 4), bar=bar, met=bool(r["frac"] >= bar), sm_mhz=c.get("sm_mhz"), reasons=c.get("reasons", []))
+            if "sustained" in r:
+                sr = r["sustained"]
+                t["sustained"] = dict(seconds=round(sr["seconds"], 2), achieved=round(sr["achieved"], 1), sm_mhz=sr["sm_mhz"], reasons=sr["reasons"],
+                                      frac_of_burst_peak=round(sr.get("frac_of_burst_peak", sr.get("frac", 0.0)), 4))
+                if sr.get("frac_of_sustained_peak") is not None:
+                    t["sustained"]["frac_of_sustained_peak"] = round(sr["frac_of_sustained_peak"], 4)
+            targets[key] = t
         line = {
             "metric": metric, "value": value, "unit": unit, "n_gpus": world,
             "steps": main_res.get("steps", args.steps), "warmup": args.warmup, "ms_per_step": main_res["ms_per_step"],
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "W": wl.W, "d": wl.d,
-                       "causal_window": wl.causal_window, "parallelism": f"replicas x{world}",
-                       "l2": main_res.get("l2", ("inputs larger than L2 (K+V %.0f MB vs 126 MB), no flush" if 4 * wl.B * wl.H * wl.N * wl.d > L2_BYTES
-                                                  else "K+V %.0f MB fit the 126 MB L2: steps after the first are served from it") % (4e-6 * wl.B * wl.H * wl.N * wl.d))},
+            "config": config_of(wl, world),
+            "also": also,
             "tflops": main_res.get("tflops"),
-            "roofline": main_res["roofline"], "e2e": main_res["e2e"], "clocks": main_res["clocks"],
             "gpu_launches": main_res["gpu_launches"], "launches_per_step": main_res["launches_per_step"],
-            "cpu_baseline": main_res.get("cpu_baseline"), "also": also,
+            "cpu_baseline": main_res.get("cpu_baseline"), "e2e": main_res["e2e"], "clocks": main_res["clocks"],
+            "roofline": main_res["roofline"], "targets": targets,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -70,12 +70,28 @@ int tlin_attn_forward_f32(const float* q, const float* k, const float* v, float*
  *   out [C,B,H,W,d]   lse [C,B,H,W] (may be NULL)
  * causal_window as in tlin_attn_forward, applied per chunk with N = n_keys[c] (with n_keys[c] = (c+1)*W and
  * causal_window = 1 chunk c is the c-th window of the training pass).  The chunks are issued as C launches of the forward
- * kernel on `stream`, each with its own plan, reading k and v in place through a strided tensor map; nothing is copied.
- * bf16, d in {64,128} (tensor-core path) only; other shapes return TLIN_ERR_UNSUPPORTED.  Workspace:
- * tlin_workspace_bytes_forward_prefixes (the largest of the chunks' needs). */
+ * kernel on `stream`, each with its own plan, reading k and v in place (row stride L); nothing is copied.
+ * bf16, head sizes as for tlin_attn_forward.  Workspace: tlin_workspace_bytes_forward_prefixes (the largest of the
+ * chunks' needs).  tlin_attn_forward_batched runs such a list, and any other, as one launch. */
 int tlin_attn_forward_prefixes(const void* q, const void* k, const void* v, void* out, float* lse,
                                int B, int H, int L, int W, int d, int C, const int32_t* n_keys,
                                int causal_window, tlin_stream_t stream);
+
+/* Cache-miss forward over a decode cache, in place.  Section 4.1 ("Cache Miss") names two inference cases that
+ * recompute from scratch: the first token, and "the first new token immediately after the historical context window
+ * has been updated (i.e., slided)"; Section 5.2: the history cache stays static only while the window does not slide.
+ * After W_og cached steps (tlin_decode_step) the window is full, its rows become history, and the layers that look at
+ * the history run again over what the cache now holds:
+ *   k_cache, v_cache [B,H,Ncap,d] bf16 as in tlin_decode_step; the call uses rows [0, n_keys) of every (b,h)
+ *   (0 < n_keys <= Ncap) through the cache's own row stride.  Nothing is copied, rows >= n_keys are not read, the
+ *   caches are not written.
+ *   q [B,H,W,d], out, lse, causal_window, head sizes, workspace and errors: as tlin_attn_forward with N = n_keys
+ *   (causal_window = 0: summary queries over the new history, Section 3 "Focused Attention"; causal_window = 1: the
+ *   last W cached positions as a window, which reproduces what the W decode steps returned).
+ * The caller keeps the position count and decides when a window is full; tlin_decode_step continues on the same
+ * buffers afterwards. */
+int tlin_attn_forward_cache(const void* q, const void* k_cache, const void* v_cache, void* out, float* lse,
+                            int B, int H, int Ncap, int n_keys, int W, int d, int causal_window, tlin_stream_t stream);
 
 /* Same as tlin_attn_forward with HOST input/output buffers (ideally pinned).  *_h are HOST
  * pointers; *_d are DEVICE staging buffers of the same shapes, supplied by the caller.  Copies
@@ -186,9 +202,11 @@ int tlin_merge_lse_f32(const float* out_a, const float* lse_a, const float* out_
                        float* out, float* lse, int64_t rows, int d, tlin_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------
- * Workspace.  Split-K partial results live in one caller-owned device buffer, registered once per
- * process (per device) and borrowed until replaced.  Calls on different streams that both need the
- * workspace must not overlap.  The *_bytes functions are pure host arithmetic.
+ * Workspace.  Split-K partial results live in one caller-owned device buffer per device:
+ * tlin_set_workspace registers it for the device that is current at the call (one buffer per device and
+ * process), borrowed until replaced; compute calls use the buffer of their current device.  Calls on
+ * different streams that both need the workspace must not overlap.  The *_bytes functions are pure host
+ * arithmetic.  With TLIN_LOG=1 in the environment every compute call prints the plan it chose to stderr.
  */
 size_t tlin_workspace_bytes_forward(int B, int H, int N, int W, int d, int causal_window);
 size_t tlin_workspace_bytes_decode(int B, int H, int Ncap, int d);
@@ -252,9 +270,20 @@ int tlin_tile_class(int64_t N, int64_t W, int causal_window, int tile_m, int til
 /* ------------------------------------------------------------------------------------------
  * Status and options.
  */
-/* Synchronises `stream`, then returns and clears the device-side error word (TLIN_OK or
- * TLIN_ERR_TIMEOUT), or TLIN_ERR_CUDA if the stream reports an error. */
+/* Synchronises `stream`, then returns and clears the device-side error word of the current device:
+ *   TLIN_OK               nothing was reported since the last call;
+ *   TLIN_ERR_TIMEOUT      a bounded device-side wait of a tensor-core kernel ran out (the CTA drained and left);
+ *   TLIN_ERR_INVALID_ARG  tlin_decode_step_ragged met a pos[b] outside its bounds (only the kernel can see it);
+ *   TLIN_ERR_CUDA         a backward tensor-core kernel found its shared-memory layout unusable and did no work,
+ *                         or the stream / a copy reported an error.
+ * When several kernels reported, the last writer's code is returned. */
 int tlin_get_status(tlin_stream_t stream);
+/* Diagnostic (not in the paper): launches one tiny kernel that waits, with the bounded wait of the tensor-core
+ * kernels, on a barrier nothing ever signals.  The wait gives up after `limit_cycles` SM clocks (1 .. 2e9) and the
+ * kernel reports TLIN_ERR_TIMEOUT through tlin_get_status, which is how a stalled attention kernel would end.
+ * waited_cycles: DEVICE pointer to one int64 receiving the clocks the kernel spent waiting, or NULL.
+ * Nothing faults or hangs; the library stays usable. */
+int tlin_debug_wait_expires(long long limit_cycles, long long* waited_cycles, tlin_stream_t stream);
 const char* tlin_status_string(int status);
 const char* tlin_version(void);
 /* Which kernel serves tlin_attn_forward: 0 = automatic, 1 = always the CUDA-core kernel,

@@ -46,6 +46,7 @@ SIGNATURES = {
     "tlin_attn_forward_f32": (_i, [_vp] * 5 + [_i] * 6 + [_vp]),
     "tlin_attn_forward_prefixes": (_i, [_vp] * 5 + [_i] * 6 + [_vp, _i, _vp]),
     "tlin_attn_forward_host": (_i, [_vp] * 10 + [_i] * 6 + [_vp]),
+    "tlin_attn_forward_cache": (_i, [_vp] * 5 + [_i] * 7 + [_vp]),
     "tlin_attn_backward": (_i, [_vp] * 9 + [_i] * 6 + [_vp]),
     "tlin_attn_backward_f32": (_i, [_vp] * 9 + [_i] * 6 + [_vp]),
     "tlin_decode_step": (_i, [_vp] * 7 + [_i] * 5 + [_vp]),
@@ -67,6 +68,7 @@ SIGNATURES = {
     "tlin_allowed": (_i, [_i64] * 4 + [_i]),
     "tlin_tile_class": (_i, [_i64, _i64, _i, _i, _i, _i, _i]),
     "tlin_get_status": (_i, [_vp]),
+    "tlin_debug_wait_expires": (_i, [ctypes.c_longlong, _vp, _vp]),
     "tlin_status_string": (ctypes.c_char_p, [_i]),
     "tlin_version": (ctypes.c_char_p, []),
     "tlin_set_forward_impl": (_i, [_i]),
@@ -197,6 +199,25 @@ def tlin_attn_forward_prefixes(q, k, v, n_keys, out=None, lse=None, causal_windo
     ensure_workspace(int(lib().tlin_workspace_bytes_forward_prefixes(B, H, W, d, C, arr, int(causal_window))), q.device)
     _check(lib().tlin_attn_forward_prefixes(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), B, H, L, W, d, C, arr,
                                             int(causal_window), _stream(stream)), "tlin_attn_forward_prefixes")
+    return out, lse
+
+
+def tlin_attn_forward_cache(q, k_cache, v_cache, n_keys, out=None, lse=None, causal_window=1, stream=None):
+    """Cache-miss forward over the first ``n_keys`` rows of decode caches [B,H,Ncap,d], in place."""
+    B, H, W, d = q.shape
+    Ncap = k_cache.shape[2]
+    _dev(q, torch.bfloat16, (B, H, W, d), "q")
+    _dev(k_cache, torch.bfloat16, (B, H, Ncap, d), "k_cache")
+    _dev(v_cache, torch.bfloat16, (B, H, Ncap, d), "v_cache")
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((B, H, W), dtype=torch.float32, device=q.device)
+    _dev(out, torch.bfloat16, (B, H, W, d), "out")
+    _dev(lse, torch.float32, (B, H, W), "lse")
+    ensure_workspace(workspace_bytes_forward(B, H, int(n_keys), W, d, causal_window), q.device)
+    _check(lib().tlin_attn_forward_cache(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(out), _ptr(lse), B, H, Ncap, int(n_keys),
+                                         W, d, int(causal_window), _stream(stream)), "tlin_attn_forward_cache")
     return out, lse
 
 
@@ -386,6 +407,11 @@ def tlin_tile_class(N, W, causal_window, tile_m, tile_n, qt, kt) -> int:
 
 def tlin_get_status(stream=None) -> int:
     return int(lib().tlin_get_status(_stream(stream)))
+
+
+def tlin_debug_wait_expires(limit_cycles: int, waited=None, stream=None) -> None:
+    """Launches the diagnostic kernel whose bounded wait runs out; ``waited`` is an optional int64 device tensor."""
+    _check(lib().tlin_debug_wait_expires(int(limit_cycles), _ptr(waited), _stream(stream)), "tlin_debug_wait_expires")
 
 
 def tlin_set_forward_impl(impl: int) -> int:

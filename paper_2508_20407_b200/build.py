@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(CSRC, "_build")
 LIB = os.path.join(HERE, "libtlin.so")
-SOURCES = ["api.cu", "plan.cu", "fwd_simt.cu", "fwd_tc.cu", "decode.cu", "merge.cu", "bwd_simt.cu", "bwd_tc.cu"]
+SOURCES = ["api.cu", "plan.cu", "fwd_simt.cu", "fwd_tc.cu", "decode.cu", "merge.cu", "bwd_simt.cu", "bwd_tc.cu", "debug.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -3,26 +3,28 @@
 #include "tlin_internal.h"
 #include <atomic>
 #include <mutex>
+#include <stdlib.h>
 
 namespace tlin {
 
 namespace {
+constexpr int kMaxDevices = 64;
 std::mutex g_mu;
-Workspace g_ws = {nullptr, 0};
+Workspace g_ws[kMaxDevices] = {};          // one registered workspace per device (indexed by the current device)
 std::atomic<int> g_impl{0};
 thread_local int t_launches = 0;
 __device__ int g_status_word = 0;
 
 struct DevInfo { int checked; int major; int sms; };
-DevInfo g_dev[64] = {};
+DevInfo g_dev[kMaxDevices] = {};
 
 int device_info(int* sms) {
     int dev = 0;
     TLIN_CUDA_CHECK(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64) return TLIN_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return TLIN_ERR_CUDA;
+    std::lock_guard<std::mutex> lk(g_mu);
     DevInfo& di = g_dev[dev];
     if (!di.checked) {
-        std::lock_guard<std::mutex> lk(g_mu);
         TLIN_CUDA_CHECK(cudaDeviceGetAttribute(&di.major, cudaDevAttrComputeCapabilityMajor, dev));
         TLIN_CUDA_CHECK(cudaDeviceGetAttribute(&di.sms, cudaDevAttrMultiProcessorCount, dev));
         di.checked = 1;
@@ -33,12 +35,45 @@ int device_info(int* sms) {
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// TLIN_LOG=1 in the environment: every compute call prints the plan it chose to stderr.
+bool log_plans() {
+    static const bool on = [] {
+        const char* e = getenv("TLIN_LOG");
+        return e != nullptr && e[0] != '\0' && e[0] != '0';
+    }();
+    return on;
+}
+void log_fwd_plan(const char* what, int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& p) {
+    fprintf(stderr, "libtlin: %s B=%d H=%d N=%d W=%d d=%d causal_window=%d -> %s, schedule %d, tile %dx%d, q_tiles %d, key_tiles %d, "
+                    "groups %d, ctas %d, units %lld, workspace %lld bytes%s\n",
+            what, B, H, N, W, d, causal, p.tensor_path ? "tensor cores" : "CUDA cores", p.schedule, p.tile_m, p.tile_n, p.q_tiles,
+            p.key_tiles, p.n_groups, p.n_ctas, (long long)p.total_units, (long long)p.workspace_bytes,
+            p.uses_workspace ? " (split, merged by a second kernel)" : "");
+}
+void log_decode_plan(const char* what, int B, int H, int Ncap, int pos, int d, const tlin_decode_plan& p) {
+    fprintf(stderr, "libtlin: %s B=%d H=%d Ncap=%d pos=%d d=%d -> %d splits of %d keys, %d ctas, workspace %lld bytes\n",
+            what, B, H, Ncap, pos, d, p.splits, p.keys_per_split, p.n_ctas, (long long)p.workspace_bytes);
+}
 }  // namespace
 
-Workspace workspace() {
-    std::lock_guard<std::mutex> lk(g_mu);
-    return g_ws;
+// Index of the current device in the per-device tables; 0 where no device can be asked (registering a workspace is
+// host bookkeeping and works without one); -1 beyond the tables.
+int current_device_slot() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
+    return dev >= 0 && dev < 64 ? dev : -1;
 }
+Workspace workspace() {
+    const int dev = current_device_slot();
+    if (dev < 0) return Workspace{nullptr, 0};
+    std::lock_guard<std::mutex> lk(g_mu);
+    return g_ws[dev];
+}
+void reset_launches() { t_launches = 0; }
 int* status_word() {
     int* p = nullptr;
     if (cudaGetSymbolAddress((void**)&p, g_status_word) != cudaSuccess) return nullptr;
@@ -70,11 +105,12 @@ static int forward_common(const void* q, const void* k, const void* v, void* out
     if (rc != TLIN_OK) return rc;
     rc = tlin_plan_forward(B, H, N, W, d, causal_window, is_f32, sms, &plan);
     if (rc != TLIN_OK) return rc;
-    if (kv_rows_alloc > 0 && (is_f32 || !plan.tensor_path)) return TLIN_ERR_UNSUPPORTED;   // strided k, v: tensor path only
+    if (log_plans()) log_fwd_plan(is_f32 ? "forward (fp32)" : "forward", B, H, N, W, d, causal_window, plan);
     if (is_f32)
-        return launch_fwd_simt_f32((const float*)q, (const float*)k, (const float*)v, (float*)out, lse, B, H, N, W, d, causal_window, st);
+        return launch_fwd_simt_f32((const float*)q, (const float*)k, (const float*)v, (float*)out, lse, B, H, N, W, d, causal_window,
+                                   kv_rows_alloc, st);
     if (!plan.tensor_path)
-        return launch_fwd_simt_bf16(q, k, v, out, lse, B, H, N, W, d, causal_window, st);
+        return launch_fwd_simt_bf16(q, k, v, out, lse, B, H, N, W, d, causal_window, kv_rows_alloc, st);
     float* ws = nullptr;
     if (plan.uses_workspace) {
         const Workspace w = workspace();
@@ -96,7 +132,6 @@ extern "C" int tlin_attn_forward_prefixes(const void* q, const void* k, const vo
     if (causal_window != 0 && causal_window != 1) return TLIN_ERR_INVALID_ARG;
     for (int c = 0; c < C; ++c)      // every chunk is checked before the first one is launched
         if (n_keys[c] <= 0 || n_keys[c] > L || (causal_window && n_keys[c] < W)) return TLIN_ERR_INVALID_ARG;
-    if (d != 64 && d != 128) return TLIN_ERR_UNSUPPORTED;
     const size_t q_chunk = (size_t)B * H * W * d * 2, lse_chunk = (size_t)B * H * W;
     int total = 0;                 // a chunked call counts the launches of all its chunks
     for (int c = 0; c < C; ++c) {
@@ -107,6 +142,13 @@ extern "C" int tlin_attn_forward_prefixes(const void* q, const void* k, const vo
     }
     t_launches = total;
     return TLIN_OK;
+}
+
+extern "C" int tlin_attn_forward_cache(const void* q, const void* k_cache, const void* v_cache, void* out, float* lse,
+                                       int B, int H, int Ncap, int n_keys, int W, int d, int causal_window, tlin_stream_t stream) {
+    if (Ncap <= 0 || n_keys <= 0 || n_keys > Ncap) return TLIN_ERR_INVALID_ARG;
+    // the first n_keys rows of every (b,h) block of Ncap rows, read in place (row stride of the cache, nothing copied)
+    return forward_common(q, k_cache, v_cache, out, lse, B, H, n_keys, W, d, causal_window, 0, (cudaStream_t)stream, Ncap);
 }
 
 extern "C" size_t tlin_workspace_bytes_forward_prefixes(int B, int H, int W, int d, int C, const int32_t* n_keys, int causal_window) {
@@ -166,6 +208,7 @@ static int backward_common(const void* q, const void* k, const void* v, const vo
     tlin_fwd_plan plan;
     rc = tlin_plan_forward(B, H, N, W, d, causal_window, 0, sms, &plan);   // the dQ kernel follows the forward's plan
     if (rc != TLIN_OK) return rc;
+    if (log_plans()) log_fwd_plan("backward (dQ kernel follows this plan)", B, H, N, W, d, causal_window, plan);
     if (!w.ptr || w.bytes < bwd_tc_workspace_bytes(B, H, W, d, plan)) return TLIN_ERR_WORKSPACE;
     return launch_bwd_tc(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, d, causal_window, plan, (float*)w.ptr, sms, st);
 }
@@ -211,6 +254,7 @@ extern "C" int tlin_decode_step(const void* q_new, const void* k_new, const void
     tlin_decode_plan plan;
     rc = tlin_plan_decode(B, H, pos + 1, d, sms, &plan);
     if (rc != TLIN_OK) return rc;
+    if (log_plans()) log_decode_plan("decode", B, H, Ncap, pos, d, plan);
     const Workspace w = workspace();
     if (!w.ptr || w.bytes < (size_t)plan.workspace_bytes) return TLIN_ERR_WORKSPACE;
     return launch_decode(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, nullptr, d, plan,
@@ -306,9 +350,11 @@ extern "C" int tlin_merge_lse_f32(const float* out_a, const float* lse_a, const 
 extern "C" int tlin_set_workspace(void* dev_ptr, size_t bytes) {
     if ((dev_ptr == nullptr) != (bytes == 0)) return TLIN_ERR_INVALID_ARG;
     if (!aligned16(dev_ptr)) return TLIN_ERR_INVALID_ARG;
+    const int dev = current_device_slot();
+    if (dev < 0) return TLIN_ERR_CUDA;
     std::lock_guard<std::mutex> lk(g_mu);
-    g_ws.ptr = dev_ptr;
-    g_ws.bytes = bytes;
+    g_ws[dev].ptr = dev_ptr;
+    g_ws[dev].bytes = bytes;
     return TLIN_OK;
 }
 

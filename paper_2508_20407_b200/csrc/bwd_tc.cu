@@ -890,14 +890,9 @@ int launch_d(const void* q, const void* k, const void* v, const void* out, const
     p.scale = 1.f / sqrtf((float)D);
     p.scale_log2e = kLog2e * p.scale;
     p.wide_stores = ((reinterpret_cast<uintptr_t>(dq) | reinterpret_cast<uintptr_t>(ws)) & 31u) == 0;
-    static std::once_flag attr_once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(attr_once, [] {
-        attr_err = cudaFuncSetAttribute(bwd_dkdv_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, ACfg<D>::kSmemBytes);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(bwd_dq_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, BCfg<D>::kSmemBytes);
-    });
-    TLIN_CUDA_CHECK(attr_err);
+    static bool smem_allowed_a[64] = {}, smem_allowed_b[64] = {};
+    TLIN_CUDA_CHECK(allow_dynamic_smem(bwd_dkdv_tc_kernel<D>, ACfg<D>::kSmemBytes, smem_allowed_a));
+    TLIN_CUDA_CHECK(allow_dynamic_smem(bwd_dq_tc_kernel<D>, BCfg<D>::kSmemBytes, smem_allowed_b));
     const long long rows_padded = bh * Wpad;
     bwd_prep_kernel<D><<<(unsigned)((rows_padded + prep_rows_per_block<D>() - 1) / prep_rows_per_block<D>()), 256, 0, st>>>(
         (const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse, lse2, delta, W, Wpad, rows_padded);

@@ -206,6 +206,11 @@ decode_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ 
     const float* pl = part_lse + (int64_t)bh * splits;
     float mm = -CUDART_INF_F;
     for (int s = 0; s < splits; ++s) mm = fmaxf(mm, pl[s]);
+    if (mm == -CUDART_INF_F) {          // every split empty (a ragged sequence whose position was rejected): zeros, not NaN
+        out[(int64_t)bh * D + c] = __float2bfloat16_rn(0.f);
+        if (lse != nullptr && c == 0) lse[bh] = -CUDART_INF_F;
+        return;
+    }
     float z = 0.f, a = 0.f;
     for (int s = 0; s < splits; ++s) {
         const float w = expf(pl[s] - mm);
@@ -516,6 +521,7 @@ extern "C" int tlin_decode_step_static(const void* q_new, const void* k_new, con
                                        void* k_cache, void* v_cache, void* out, float* lse,
                                        int B, int H, int Ncap, int pos, int d, tlin_stream_t stream) {
     using namespace tlin;
+    reset_launches();
     if (!q_new || !k_new || !v_new || !k_cache || !v_cache || !out) return TLIN_ERR_INVALID_ARG;
     if (B <= 0 || H <= 0 || Ncap <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
     if (pos < 0 || pos >= Ncap) return TLIN_ERR_INVALID_ARG;

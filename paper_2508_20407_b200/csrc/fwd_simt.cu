@@ -35,7 +35,7 @@ template <typename T>
 __global__ void __launch_bounds__(ROWS * 32)
 fwd_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                 T* __restrict__ out, float* __restrict__ lse,
-                int N, int W, int d, int causal, int q_tiles, float scale) {
+                int N, int W, int d, int causal, int q_tiles, float scale, int64_t kv_rows) {
     extern __shared__ float smem[];
     const int kstride = d + 4;                 // padded: lanes reading different rows hit different banks
     float* Qs = smem;                          // [ROWS][d]
@@ -48,8 +48,8 @@ fwd_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
     const int i = row0 + warp;
     const bool row_ok = i < W;
     const T* qb = q + (bh * W + row0) * (int64_t)d;
-    const T* kb = k + bh * (int64_t)N * d;
-    const T* vb = v + bh * (int64_t)N * d;
+    const T* kb = k + bh * kv_rows * d;        // kv_rows >= N: rows per (b,h) of the key/value allocation
+    const T* vb = v + bh * kv_rows * d;
 
     const int rows_here = min(ROWS, W - row0);
     for (int idx = threadIdx.x; idx < rows_here * d; idx += blockDim.x) Qs[idx] = to_f32(qb[idx]);
@@ -119,13 +119,14 @@ fwd_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __res
 
 template <typename T>
 int launch(const T* q, const T* k, const T* v, T* out, float* lse, int B, int H, int N, int W, int d,
-           int causal, cudaStream_t st) {
+           int causal, long long kv_rows_alloc, cudaStream_t st) {
     const int q_tiles = (W + ROWS - 1) / ROWS;
     const int64_t blocks = (int64_t)B * H * q_tiles;
     const size_t smem = sizeof(float) * ((size_t)ROWS * d + (size_t)KT * (d + 4) + (size_t)KT * d);
     TLIN_CUDA_CHECK(cudaFuncSetAttribute(fwd_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     fwd_simt_kernel<T><<<(unsigned)blocks, ROWS * 32, smem, st>>>(q, k, v, out, lse, N, W, d, causal, q_tiles,
-                                                                   1.0f / sqrtf((float)d));
+                                                                   1.0f / sqrtf((float)d),
+                                                                   kv_rows_alloc > 0 ? (int64_t)kv_rows_alloc : (int64_t)N);
     TLIN_CUDA_CHECK(cudaGetLastError());
     count_launch();
     return TLIN_OK;
@@ -134,13 +135,13 @@ int launch(const T* q, const T* k, const T* v, T* out, float* lse, int B, int H,
 }  // namespace
 
 int launch_fwd_simt_bf16(const void* q, const void* k, const void* v, void* out, float* lse,
-                         int B, int H, int N, int W, int d, int causal, cudaStream_t st) {
+                         int B, int H, int N, int W, int d, int causal, long long kv_rows_alloc, cudaStream_t st) {
     return launch<__nv_bfloat16>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
-                                 (__nv_bfloat16*)out, lse, B, H, N, W, d, causal, st);
+                                 (__nv_bfloat16*)out, lse, B, H, N, W, d, causal, kv_rows_alloc, st);
 }
 int launch_fwd_simt_f32(const float* q, const float* k, const float* v, float* out, float* lse,
-                        int B, int H, int N, int W, int d, int causal, cudaStream_t st) {
-    return launch<float>(q, k, v, out, lse, B, H, N, W, d, causal, st);
+                        int B, int H, int N, int W, int d, int causal, long long kv_rows_alloc, cudaStream_t st) {
+    return launch<float>(q, k, v, out, lse, B, H, N, W, d, causal, kv_rows_alloc, st);
 }
 
 }  // namespace tlin

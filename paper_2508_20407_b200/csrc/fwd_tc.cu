@@ -187,6 +187,11 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     int dummy = 0;
                     mbar_wait(&kv_full[slot], round & 1, &dummy, 200000000LL);
                 }
+                // seg_idx counts the Q loads armed so far; the last one may still be on its way
+                if (seg_idx > 0) {
+                    int dummy = 0;
+                    mbar_wait(q_full, (seg_idx - 1) & 1, &dummy, 200000000LL);
+                }
             }
         }
     } else if (warp == kMmaWarp) {
@@ -625,12 +630,8 @@ int launch_d(const void* q, const void* k, const void* v, void* out, float* lse,
     p.total_units = plan.total_units; p.n_groups = plan.n_groups; p.q_tiles = plan.q_tiles; p.key_tiles = plan.key_tiles;
     p.N = N; p.W = W; p.causal = causal; p.schedule = plan.schedule;
     p.scale_log2e = kLog2e / sqrtf((float)D);
-    static std::once_flag attr_once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(attr_once, [] {
-        attr_err = cudaFuncSetAttribute(fwd_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-    });
-    TLIN_CUDA_CHECK(attr_err);
+    static bool smem_allowed[64] = {};
+    TLIN_CUDA_CHECK(allow_dynamic_smem(fwd_tc_kernel<D>, C::kSmemBytes, smem_allowed));
     if (plan.n_groups > kMaxGroups) return TLIN_ERR_UNSUPPORTED;
     GroupStarts starts;
     fwd_group_starts(plan, &starts);

@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <stdio.h>
+#include <mutex>
 #include "../../include/tlin.h"
 
 namespace tlin {
@@ -20,7 +21,23 @@ struct Workspace { void* ptr; size_t bytes; };
 Workspace workspace();
 int* status_word();                    // device address of the error word (bounded waits report here)
 void count_launch(int n = 1);
+void reset_launches();                 // every compute entry point starts its count at zero
+int current_device_slot();             // index of the current device in per-device tables (-1: beyond them)
 int forward_impl();
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) holds for the device that is current when it is called, so a kernel
+// that needs more than 48 KB asks once per device.  `done` is a table of 64 flags owned by the caller (one per kernel).
+template <class Kernel>
+inline cudaError_t allow_dynamic_smem(Kernel kernel, int bytes, bool (&done)[64]) {
+    static std::mutex mu;
+    const int dev = current_device_slot();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lk(mu);
+    if (done[dev]) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) done[dev] = true;
+    return e;
+}
 
 // Work sharing of the tensor-core forward and dQ kernels.  The host works out the first unit of every group and passes the
 // table to the kernel as a launch parameter (the CTAs only index it).
@@ -90,9 +107,9 @@ __host__ __device__ inline long long bwd_first_unit_of_share(int N, int W, int c
 
 // ---- launchers (one per kernel family); all validate nothing: api.cu has done it ----------
 int launch_fwd_simt_bf16(const void* q, const void* k, const void* v, void* out, float* lse,
-                         int B, int H, int N, int W, int d, int causal, cudaStream_t st);
+                         int B, int H, int N, int W, int d, int causal, long long kv_rows_alloc, cudaStream_t st);
 int launch_fwd_simt_f32(const float* q, const float* k, const float* v, float* out, float* lse,
-                        int B, int H, int N, int W, int d, int causal, cudaStream_t st);
+                        int B, int H, int N, int W, int d, int causal, long long kv_rows_alloc, cudaStream_t st);
 int launch_fwd_tc(const void* q, const void* k, const void* v, void* out, float* lse,
                   int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& plan,
                   float* ws, long long kv_rows_alloc, cudaStream_t st);   // kv_rows_alloc: rows per (b,h) of k, v (0 = N)

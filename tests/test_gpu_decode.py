@@ -131,12 +131,17 @@ def test_ragged_decode_reports_a_position_beyond_the_bound():
     kc_before = kc.clone()
     x = torch.ones((B, H, 1, d), dtype=torch.bfloat16, device=DEV)
     pos = torch.tensor([5, 40], dtype=torch.int32, device=DEV)      # 40 exceeds the bound given below
+    kc_h, vc_h = kc.cpu(), vc.cpu()
     out, lse = tl.tlin_decode_step_ragged(x, x, x, kc, vc, pos, 10)
     torch.cuda.synchronize()
     assert tl.tlin_get_status() == tl.ERR_INVALID_ARG
     assert tl.tlin_get_status() == 0                                  # reading clears it
     assert torch.equal(kc[1], kc_before[1])                           # the offending sequence's cache is untouched
     assert (kc[0, :, 5] == 1).all()                                   # the valid one was appended
+    # the rejected sequence gets zeros and an empty log-sum-exp, not NaN; the valid one its ordinary result
+    assert float(out[1].float().abs().max()) == 0.0 and bool((lse[1] == float("-inf")).all())
+    ref, ref_lse = oracle.decode_step(x[:1].cpu(), x[:1].cpu(), x[:1].cpu(), kc_h[:1], vc_h[:1], 5)
+    parity.check(out[:1].float().cpu().numpy(), lse[:1].cpu().numpy(), ref, ref_lse, "bf16", "valid sequence beside a rejected one")
     with pytest.raises(tl.TlinError):
         tl.tlin_decode_step_ragged(x, x, x, kc, vc, pos, 64)          # bound outside the cache: rejected on the host
 
@@ -274,3 +279,70 @@ def test_fp8_decode_at_the_cfg5_size_on_sampled_heads():
             parity.check(sl(out).float().numpy(), sl(lse).numpy(), ref, ref_lse, "bf16", f"8-bit cfg5 step {t} head {(b, h)}")
     for (b, h) in heads:
         assert torch.equal(kc[b, h].cpu(), host[(b, h)][0][0, 0]) and torch.equal(vc[b, h].cpu(), host[(b, h)][1][0, 0])
+
+
+@pytest.mark.parametrize("B,H,d,hist,W_og,W_oh,extra", [(2, 3, 128, 300, 64, 48, 5), (1, 2, 64, 1000, 130, 40, 3), (1, 2, 72, 90, 20, 8, 2)])
+def test_window_slide_cycle_on_the_cache_in_place(B, H, d, hist, W_og, W_oh, extra):
+    """Section 4.1 / 5.2: decode W_og cached steps, then the window slides and the layers that look at the history run
+    again from scratch -- here directly on the cache buffer (first n rows of a larger allocation, nothing copied) --
+    and decoding continues on the same buffers.  Every output against the oracle; the caches bit-equal throughout."""
+    if d not in (64, 128):
+        steps_ok = False        # the decode kernel serves d in {64,128}; other head sizes exercise the forward over the cache only
+    else:
+        steps_ok = True
+    total = W_og + extra
+    wl = synth.Workload("slide", B, H, d, hist, total, seed=500 + hist, decode=True)
+    (kc, vc), (qn, kn, vn) = synth.decode_inputs(wl, device=DEV)
+    pad = 3                                                    # canary rows above everything that is ever written
+    kc = torch.cat([kc, torch.full((B, H, pad, d), -7.0, dtype=kc.dtype, device=DEV)], dim=2).contiguous()
+    vc = torch.cat([vc, torch.full((B, H, pad, d), -7.0, dtype=vc.dtype, device=DEV)], dim=2).contiguous()
+    kc[:, :, hist:] = -7.0
+    vc[:, :, hist:] = -7.0
+    kc_h, vc_h = kc.cpu(), vc.cpu()
+    dec_out, dec_lse = [], []
+
+    def decode(t):
+        if steps_ok:
+            o, l = tl.tlin_decode_step(qn[t], kn[t], vn[t], kc, vc, hist + t)
+            torch.cuda.synchronize()
+            assert tl.tlin_get_status() == 0
+        ref, ref_lse = oracle.decode_step(qn[t].cpu(), kn[t].cpu(), vn[t].cpu(), kc_h, vc_h, hist + t)
+        if steps_ok:
+            parity.check(o.float().cpu().numpy(), l.cpu().numpy(), ref, ref_lse, "bf16", f"decode step {t}")
+            assert torch.equal(kc.cpu(), kc_h) and torch.equal(vc.cpu(), vc_h)
+            dec_out.append(o.clone())
+            dec_lse.append(l.clone())
+        else:                                                   # no decode kernel for this head size: place the rows by copy
+            kc[:, :, hist + t] = kn[t][:, :, 0]
+            vc[:, :, hist + t] = vn[t][:, :, 0]
+
+    for t in range(W_og):                                       # the window fills up
+        decode(t)
+    pos = hist + W_og                                           # the window slides: all `pos` cached rows are history now
+    # (a) summary queries over the new history (focused attention), on the cache in place
+    g = torch.Generator(device="cpu").manual_seed(hist)
+    q_sum = torch.randn((B, H, W_oh, d), generator=g).to(torch.bfloat16).to(DEV)
+    out, lse = tl.tlin_attn_forward_cache(q_sum, kc, vc, pos, causal_window=0)
+    torch.cuda.synchronize()
+    assert tl.tlin_get_status() == 0
+    ref, ref_lse = oracle.attn_forward(q_sum.cpu(), kc_h[:, :, :pos].contiguous(), vc_h[:, :, :pos].contiguous(), 0)
+    parity.check(out.float().cpu().numpy(), lse.cpu().numpy(), ref, ref_lse, "bf16", "summary queries over the slid history")
+    # (b) the window just completed, recomputed as a cache-miss forward: its rows are what the decode steps returned
+    q_win = torch.cat([qn[t] for t in range(W_og)], dim=2).contiguous()
+    out, lse = tl.tlin_attn_forward_cache(q_win, kc, vc, pos, causal_window=1)
+    torch.cuda.synchronize()
+    assert tl.tlin_get_status() == 0
+    ref, ref_lse = oracle.attn_forward(q_win.cpu(), kc_h[:, :, :pos].contiguous(), vc_h[:, :, :pos].contiguous(), 1)
+    parity.check(out.float().cpu().numpy(), lse.cpu().numpy(), ref, ref_lse, "bf16", "window recomputed over the cache")
+    if steps_ok:
+        steps = torch.cat(dec_out, dim=2).float()
+        assert float((steps - out.float()).abs().max()) <= 2e-2
+        assert float((torch.stack(dec_lse, dim=2) - lse).abs().max()) <= 1e-3
+    # the forward calls wrote nothing into the caches, and the rows above `pos` still hold the canary
+    assert torch.equal(kc.cpu(), kc_h) and torch.equal(vc.cpu(), vc_h)
+    assert (kc[:, :, pos:] == -7.0).all() and (vc[:, :, pos:] == -7.0).all()
+    for t in range(W_og, total):                                # decoding continues in the next window
+        decode(t)
+    assert (kc[:, :, hist + total:] == -7.0).all() and (vc[:, :, hist + total:] == -7.0).all()
+    with pytest.raises(tl.TlinError):
+        tl.tlin_attn_forward_cache(q_sum, kc, vc, kc.shape[2] + 1, causal_window=0)      # more rows than the cache has

@@ -8,6 +8,7 @@ import torch
 
 import oracle
 import parity
+from guards import Guarded
 from paper_2508_20407_b200 import binding as tl
 from paper_2508_20407_b200 import synth
 
@@ -75,11 +76,68 @@ SHAPES = [  # B, H, N, W, d, causal
 ]
 
 
+def guarded_compare(wl, impl):
+    """full_compare with out, lse and the split workspace inside guarded buffers of exactly the documented sizes."""
+    causal = wl.causal_window
+    q, k, v = synth.forward_inputs(wl, device=DEV)
+    out_g = Guarded(q.shape, torch.bfloat16, DEV)
+    lse_g = Guarded((wl.B, wl.H, wl.W), torch.float32, DEV)
+    saved = tl._workspace_tensor
+    prev = tl.tlin_set_forward_impl(impl)
+    try:
+        need = tl.workspace_bytes_forward(wl.B, wl.H, wl.N, wl.W, wl.d, causal)
+        ws_g = Guarded((max(need, 16),), torch.uint8, DEV)
+        tl.set_workspace(ws_g.t)
+        out, lse = tl.tlin_attn_forward(q, k, v, out_g.t, lse_g.t, causal_window=causal)
+        torch.cuda.synchronize()
+        assert tl.tlin_get_status() == 0 and tl.tlin_last_launch_count() >= 1
+        assert tl._workspace_tensor is ws_g.t          # the call used the guarded workspace, nothing larger
+    finally:
+        tl.tlin_set_forward_impl(prev)
+        tl.set_workspace(saved)
+    for g, name in ((out_g, "out"), (lse_g, "lse"), (ws_g, "workspace")):
+        g.check(f"{wl.name} impl={impl} {name}")
+    ref, ref_lse = oracle.attn_forward(q.cpu(), k.cpu(), v.cpu(), causal)
+    return parity.check(out.float().cpu().numpy(), lse.cpu().numpy(), ref, ref_lse, "bf16", f"{wl.name} impl={impl}")
+
+
 @pytest.mark.parametrize("B,H,N,W,d,causal", SHAPES)
 def test_awkward_shapes_bf16(B, H, N, W, d, causal):
     wl = synth.Workload("shape", B, H, d, N, W, seed=100 + N + W, causal_window=causal)
     for impl in impls_for(d):
-        full_compare(wl, impl)
+        guarded_compare(wl, impl)
+
+
+def partials_per_head(plan):
+    """For a schedule-0 plan: how many groups (= partial results per query row) each (b,h) is spread over."""
+    starts = [tl.tlin_plan_group_start(plan, g) for g in range(plan.n_groups + 1)]
+    T = plan.key_tiles
+    counts = []
+    for bh in range(plan.total_units // T):
+        lo, hi = bh * T, (bh + 1) * T
+        counts.append(sum(1 for g in range(plan.n_groups) if starts[g] < hi and starts[g + 1] > lo))
+    return counts
+
+
+def test_awkward_shapes_reach_both_branches_of_the_split_merge():
+    # the merge kernel combines up to 8 partial results per row from registers and more than 8 in a loop: the shapes
+    # above must keep exercising both, whatever the planner turns into
+    if not TC_AVAILABLE:
+        pytest.skip("tensor path not built")
+    few = many = False
+    prev = tl.tlin_set_forward_impl(2)
+    try:
+        for (B, H, N, W, d, causal) in SHAPES:
+            plan = tl.tlin_plan_forward(B, H, N, W, d, causal)
+            if not (plan.tensor_path and plan.schedule == 0 and plan.uses_workspace):
+                continue
+            c = partials_per_head(plan)
+            few = few or any(2 <= x <= 8 for x in c)
+            many = many or any(x > 8 for x in c)
+    finally:
+        tl.tlin_set_forward_impl(prev)
+    assert few, "no awkward shape is split into 2..8 partial results per row"
+    assert many, "no awkward shape is split into more than 8 partial results per row"
 
 
 @pytest.mark.parametrize("B,H,N,W,d,causal", [(1, 2, 333, 40, 36, 1), (1, 1, 1024, 128, 64, 1), (2, 2, 200, 200, 128, 1),
@@ -214,11 +272,84 @@ def test_cfg2_mid_sampled_heads_full_rows():
             parity.check(sl(out).float().numpy(), sl(lse).numpy(), ref, ref_lse, "bf16", f"cfg2 head {(b, h)} impl={impl}")
 
 
-@pytest.mark.parametrize("name,causal", [("cfg3_long", 1), ("cfg3_long", 0), ("cfg4_vlong", 1)])
+def stratified_rows(wl, b, h, per_tile):
+    """`per_tile` hashed rows in every 128-row query tile of head (b,h): each CTA of any plan (256 query rows of one or
+    several heads) then has sampled rows in both of its query tiles, in its first and in its last head."""
+    rng = np.random.default_rng(wl.seed * 1000003 + b * 131 + h)
+    rows = []
+    for r0 in range(0, wl.W, 128):
+        r1 = min(r0 + 128, wl.W)
+        rows.extend(int(x) for x in rng.choice(np.arange(r0, r1), size=min(per_tile, r1 - r0), replace=False))
+    return sorted(rows)
+
+
+@pytest.mark.parametrize("name,causal", [("cfg3_long", 1), ("cfg3_long", 0), ("cfg4_vlong", 1), ("cfg4_vlong", 0)])
 def test_full_size_sampled_rows(name, causal):
+    """The benchmarked launch at full size: every row of heads {0, H/2, H-1} and 16 hashed rows of every other head
+    against the oracle.  The rows are spread over all 128-row query tiles, so every CTA of the plan, whose key range
+    may start or end inside a head (partial results, merged by the second kernel), has checked rows in the first and
+    in the last head it works on."""
     wl = synth.WORKLOADS[name]
     impl = 2 if TC_AVAILABLE else 1
-    sampled_rows_compare(wl, impl, 6, [(0, 0), (0, wl.H // 2), (0, wl.H - 1)], causal)
+    q, k, v = synth.forward_inputs(wl, device=DEV)
+    out, lse = run_impl(impl, tl.tlin_attn_forward, q, k, v, causal_window=causal)
+    assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
+    full_heads = [(0, 0), (0, wl.H // 2), (0, wl.H - 1)]
+    per_tile = max(1, 16 // ((wl.W + 127) // 128))
+    sampled = {(b, h): stratified_rows(wl, b, h, per_tile) for b in range(wl.B) for h in range(wl.H) if (b, h) not in full_heads}
+    # every CTA = (group, 256-row query tile pair) has checked rows in the first and the last head of its unit range
+    plan = tl.tlin_plan_forward(wl.B, wl.H, wl.N, wl.W, wl.d, causal)
+    if plan.tensor_path and plan.schedule == 0:
+        starts = [tl.tlin_plan_group_start(plan, g) for g in range(plan.n_groups + 1)]
+        for g in range(plan.n_groups):
+            for bh in {starts[g] // plan.key_tiles, (starts[g + 1] - 1) // plan.key_tiles}:
+                head = (bh // wl.H, bh % wl.H)
+                rows = range(wl.W) if head in full_heads else sampled[head]
+                for qt in range(plan.q_tiles):
+                    for half in range(2):
+                        lo = qt * 256 + half * 128
+                        if lo < wl.W:
+                            assert any(lo <= r < lo + 128 for r in rows), (g, head, qt, half)
+    for (b, h) in full_heads:
+        sl = lambda t: t[b:b + 1, h:h + 1].contiguous().cpu()
+        ref, ref_lse = oracle.attn_forward(sl(q), sl(k), sl(v), causal)
+        parity.check(sl(out).float().numpy(), sl(lse).numpy(), ref, ref_lse, "bf16", f"{name} causal={causal} head {(b, h)}, all rows")
+    got, got_lse, ref, ref_lse = [], [], [], []
+    for (b, h), rows in sampled.items():
+        kh, vh = k[b, h].cpu(), v[b, h].cpu()
+        qh = q[b, h].cpu()
+        if causal:      # row i alone over the keys it may use, through the unmasked oracle call
+            jobs = []
+            for i in rows:
+                limit = wl.N - wl.W + i + 1
+                jobs.append((qh[i].view(1, 1, 1, wl.d), kh[:limit].view(1, 1, limit, wl.d), vh[:limit].view(1, 1, limit, wl.d)))
+            with ThreadPoolExecutor(max_workers=8) as ex:
+                res = list(ex.map(lambda j: oracle.attn_forward(j[0], j[1], j[2], 0), jobs))
+            ref.extend(r[0].reshape(-1) for r in res)
+            ref_lse.extend(float(r[1].reshape(-1)[0]) for r in res)
+        else:
+            r, rl = oracle.attn_forward(qh[rows].view(1, 1, len(rows), wl.d), kh.view(1, 1, wl.N, wl.d), vh.view(1, 1, wl.N, wl.d), 0)
+            ref.extend(r[0, 0])
+            ref_lse.extend(rl[0, 0])
+        got.extend(out[b, h, rows].float().cpu().numpy())
+        got_lse.extend(lse[b, h, rows].cpu().numpy())
+    parity.check(np.stack(got), np.array(got_lse), np.stack(ref), np.array(ref_lse), "bf16", f"{name} causal={causal}, hashed rows of the other heads")
+
+
+@pytest.mark.parametrize("name", ["cfg3_long", "cfg4_vlong"])
+def test_full_size_tensor_core_path_agrees_with_the_cuda_core_path_everywhere(name):
+    # CUDA against CUDA, a supplement to the oracle checks above (it proves nothing by itself): the two kernels share no
+    # tiling, schedule or split, and the CUDA-core one is the path verified element by element on the small shapes
+    if not TC_AVAILABLE:
+        pytest.skip("tensor path not built")
+    wl = synth.WORKLOADS[name]
+    q, k, v = synth.forward_inputs(wl, device=DEV)
+    a, la = run_impl(2, tl.tlin_attn_forward, q, k, v, causal_window=1)
+    b, lb = run_impl(1, tl.tlin_attn_forward, q, k, v, causal_window=1)
+    # both results are rounded to bf16 (8 significant bits): two last places of the larger value, plus a floor
+    excess = (a.float() - b.float()).abs() - (2.0 ** -6) * torch.maximum(a.float().abs(), b.float().abs())
+    assert float(excess.max()) <= 2e-3
+    assert float((la - lb).abs().max()) <= 1e-3
 
 
 def test_whole_sequence_causal_attention_sampled_rows():
