@@ -36,7 +36,7 @@ from paper_2508_20407_b200 import synth  # noqa: E402
 WORKLOADS = {"fwd128k": "cfg4_vlong", "fwd32k": "cfg3_long", "fwd8k": "cfg2_mid", "decode": "cfg5_decode",
              "restore": "restore_vlong", "inner_self": "inner_self", "inner_gen": "inner_gen",
              "bwd_chunk": "train_chunk", "bwd32k": "cfg3_long", "decode_fp8": "cfg5_decode",
-             "nsweep": "cfg3_long", "fwd_seq": "train_seq", "bwd_seq": "train_seq"}
+             "nsweep": "cfg3_long", "fwd_seq": "train_seq", "bwd_seq": "train_seq", "inner_batched": "inner_self"}
 BACKWARD = ("bwd_chunk", "bwd32k", "bwd_seq")      # legs that time tlin_attn_backward on the named shape
 NOMINAL_BF16_TFLOPS, NOMINAL_HBM_GBS = 2250.0, 7700.0      # datasheet figures, reported beside the measured peaks
 REFERENCE_BUDGET_S = 100.0     # --impl reference: target duration of all its steps together
@@ -510,6 +510,49 @@ def run_decode_fp8(wl, args, rank, world, device, peaks):
                 gpu_launches=int(sum(launches[args.warmup:])), launches_per_step=launches[-1] if launches else 0)
 
 
+def run_batched(args, rank, world, device, peaks):
+    """The inner layers of one depth step of a block (Appendix A: self-attention over the W_oh summary tokens; a generation
+    layer over [summary tokens; window]) as a table in ONE launch, beside the same two problems as two calls.  Both read
+    the same inputs; a buffer larger than L2 is overwritten before every timed step."""
+    from paper_2508_20407_b200 import binding as tl
+    wls = [synth.WORKLOADS["inner_self"], synth.WORKLOADS["inner_gen"]]
+    tensors = []
+    for wl in wls:
+        q, k, v = synth.forward_inputs(wl, device=device)
+        tensors.append((wl, q, k, v, torch.empty_like(q), torch.empty((wl.B, wl.H, wl.W), dtype=torch.float32, device=device)))
+        tl.ensure_workspace(tl.workspace_bytes_forward(wl.B, wl.H, wl.N, wl.W, wl.d, wl.causal_window), device)
+    table = [(q, k, v, out, lse, None, wl.causal_window) for (wl, q, k, v, out, lse) in tensors]
+    launches = {"batched": [], "separate": []}
+
+    def step_batched(_):
+        tl.tlin_attn_forward_batched(table)
+        launches["batched"].append(tl.tlin_last_launch_count())
+
+    def step_separate(_):
+        n = 0
+        for (wl, q, k, v, out, lse) in tensors:
+            tl.tlin_attn_forward(q, k, v, out, lse, wl.causal_window)
+            n += tl.tlin_last_launch_count()
+        launches["separate"].append(n)
+
+    flush = torch.empty(int(2.5 * L2_BYTES), dtype=torch.uint8, device=device)
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    ms_b, clocks = time_steps(step_batched, args.steps, args.warmup, world, device, sampler, flush)
+    ms_s, _ = time_steps(step_separate, args.steps, args.warmup, world, device, None, flush)
+    ms_b /= args.steps
+    ms_s /= args.steps
+    flop = sum(4.0 * wl.B * wl.H * allowed_pairs(wl) * wl.d for wl in wls)
+    tflops = flop / (ms_b * 1e-3) / 1e12
+    roof = dict(bound="tensor", achieved=tflops, peak=peaks["bf16_tflops"], unit="TFLOP/s", frac=tflops / peaks["bf16_tflops"],
+                traffic=None, algorithmic_bytes=sum(fwd_bytes(wl) for wl in wls), peak_source=peaks["source"] + " (burst)",
+                kernel="forward, two problems in one launch", roofline_ms=flop / (peaks["bf16_tflops"] * 1e12) * 1e3)
+    return dict(workload="inner_self + inner_gen as one table", ms_per_step=ms_b, tflops=tflops, roofline=roof, e2e=None, clocks=clocks,
+                separate_calls_ms_per_step=ms_s, batched_over_separate=ms_b / ms_s,
+                l2="a %.0f MB buffer is overwritten before every timed step (L2 flush), steps timed one by one" % (flush.numel() / 1e6),
+                gpu_launches=int(sum(launches["batched"][args.warmup:args.warmup + args.steps])),
+                launches_per_step=launches["batched"][-1], separate_launches_per_step=launches["separate"][-1])
+
+
 def run_n_sweep(args, rank, world, device, peaks):
     """Forward time against context length at fixed B, H, W, d (the paper's claim is cost linear in N, Section 4 and
     Appendix A): N = 8k ... 256k, least-squares line t = a + b*N and its largest relative residual; cfg3/cfg4 also with
@@ -636,7 +679,8 @@ def compact_leg(leg):
                               "executed_over_counted_flops", "sustained") if k in r}
     c = leg.get("clocks") or {}
     out = {k: leg[k] for k in ("workload", "shape", "ms_per_step", "tflops", "gb_per_s", "tokens_per_s", "decode_tokens_per_s", "steps",
-                               "gpu_launches", "launches_per_step") if k in leg}
+                               "gpu_launches", "launches_per_step", "separate_calls_ms_per_step", "batched_over_separate",
+                               "separate_launches_per_step") if k in leg}
     out["roofline"] = roof
     out["clocks"] = {"sm_mhz": c.get("sm_mhz"), "sm_max_mhz": c.get("sm_max_mhz"), "reasons": c.get("reasons", [])}
     if leg.get("e2e"):
@@ -695,6 +739,8 @@ def main():
     with_cpu = (not args.no_cpu) and world == 1
     if args.workload in BACKWARD:
         main_res = run_backward(wl, args, rank, world, device, peaks)
+    elif args.workload == "inner_batched":
+        main_res = run_batched(args, rank, world, device, peaks)
     elif args.workload == "decode_fp8":
         main_res = run_decode_fp8(wl, args, rank, world, device, peaks)
     else:
@@ -703,7 +749,7 @@ def main():
     also = []
     full_legs = {args.workload: main_res}
     if not args.only and world == 1:
-        for name in ("fwd32k", "decode", "restore", "inner_self", "inner_gen", "fwd_seq", "bwd_chunk", "bwd32k", "bwd_seq", "decode_fp8"):
+        for name in ("fwd32k", "decode", "restore", "inner_self", "inner_gen", "inner_batched", "fwd_seq", "bwd_chunk", "bwd32k", "bwd_seq", "decode_fp8"):
             if name == args.workload:
                 continue
             torch.cuda.empty_cache()
@@ -714,6 +760,8 @@ def main():
             a2.sustained = args.sustained and name in ("fwd32k", "decode")  # the legs with a stated target
             if name in BACKWARD:
                 leg = run_backward(w2, a2, rank, world, device, peaks)
+            elif name == "inner_batched":
+                leg = run_batched(a2, rank, world, device, peaks)
             elif name == "decode_fp8":
                 leg = run_decode_fp8(w2, a2, rank, world, device, peaks)
             else:
@@ -724,6 +772,8 @@ def main():
     if rank == 0:
         if args.workload in BACKWARD:
             metric, unit, value = "attention_backward_TFLOP_per_s", "TFLOP/s", world * main_res["tflops"]
+        elif args.workload == "inner_batched":
+            metric, unit, value = "attention_forward_TFLOP_per_s", "TFLOP/s", world * main_res["tflops"]
         elif wl.decode:
             metric, unit, value = "decode_kv_GB_per_s", "GB/s", main_res["gb_per_s"]
         else:

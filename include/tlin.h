@@ -93,6 +93,40 @@ int tlin_attn_forward_prefixes(const void* q, const void* k, const void* v, void
 int tlin_attn_forward_cache(const void* q, const void* k_cache, const void* v_cache, void* out, float* lse,
                             int B, int H, int Ncap, int n_keys, int W, int d, int causal_window, tlin_stream_t stream);
 
+/* A table of attention problems as ONE launch.  Besides the two N-proportional attentions, a block holds layers whose
+ * cost does not grow with N (Appendix A: H self-attention layers over the W_oh summary tokens, cost H*D*W_oh^2, and per
+ * generation layer a cross-attention to them plus the causal window, (H+1)*D*W_og*W_oh + (H+2)*D*W_og^2).  Each is a
+ * small problem on which a launch of its own spends a large share of its time starting and finishing; problems that do
+ * not depend on each other (context layer i and generation layer i both read C_{i-1}; the layers of different
+ * requests; the chunks of a sliding-window training pass, Section 5.1, with arbitrary prefix lengths) go into one
+ * table and one launch.  Every problem is computed exactly as tlin_attn_forward would compute it.
+ *   problems: HOST array of n_problems entries (1 <= n_problems); the pointers inside are DEVICE pointers.
+ *   All problems share the head size d (64 or 128: tensor-core path only) and are bf16.
+ *   kv_rows: rows per (b,h) of the k, v allocation when it is larger than n_keys (a key prefix read in place, as in
+ *   tlin_attn_forward_prefixes / tlin_attn_forward_cache), else 0.  Problems may share k and v.
+ * The CTAs take contiguous runs of whole (problem, b*h, 256-row query tile) units, balanced by the key tiles each unit
+ * has to visit; keys are never split, so no workspace is used and the result does not depend on the table's neighbours.
+ * Long-context problems with few query rows (W <= 1024 over tens of thousands of keys) are better served by
+ * tlin_attn_forward, which splits the key range.  Tables of more than 24 problems are issued as several launches. */
+typedef struct {
+    const void* q;          /* [BH, n_queries, d] */
+    const void* k;          /* [BH, kv_rows or n_keys, d] */
+    const void* v;
+    void* out;              /* [BH, n_queries, d] */
+    float* lse;             /* [BH, n_queries] or NULL */
+    int32_t BH;             /* number of (batch, head) pairs of this problem */
+    int32_t n_keys;         /* N */
+    int32_t kv_rows;        /* 0, or rows per (b,h) of the k/v allocation (>= n_keys) */
+    int32_t n_queries;      /* W */
+    int32_t causal_window;  /* as in tlin_attn_forward; requires n_keys >= n_queries */
+    int32_t reserved;       /* 0 */
+} tlin_problem;
+int tlin_attn_forward_batched(const tlin_problem* problems, int n_problems, int d, tlin_stream_t stream);
+/* The split of a table's units among the CTAs of one launch (n_problems <= 24): starts[c] = first unit of CTA c,
+ * starts[*n_ctas] = number of units; unit order = problem, then b*h, then query tile pair.  starts has room for
+ * num_sms + 1 entries (num_sms <= 0: 148).  Pure host arithmetic. */
+int tlin_plan_batched(const tlin_problem* problems, int n_problems, int num_sms, int64_t* starts, int32_t* n_ctas);
+
 /* Same as tlin_attn_forward with HOST input/output buffers (ideally pinned).  *_h are HOST
  * pointers; *_d are DEVICE staging buffers of the same shapes, supplied by the caller.  Copies
  * q,k,v host->device, runs the forward, copies out (and lse if lse_h != NULL) device->host, all on
@@ -128,6 +162,30 @@ int tlin_decode_step(const void* q_new, const void* k_new, const void* v_new,
 int tlin_decode_step_ragged(const void* q_new, const void* k_new, const void* v_new,
                             void* k_cache, void* v_cache, void* out, float* lse,
                             int B, int H, int Ncap, const int32_t* pos, int max_pos, int d, tlin_stream_t stream);
+
+/* A table of cached decode steps as ONE launch.  In a cache-hit step (Appendix A) the N-proportional term is the new
+ * token against the history, served by tlin_decode_step; what remains are short rows: per generation layer the new
+ * token against the W_oh cached summary tokens C_i, (H+1)*D*W_oh in all, and against the window so far.  For one
+ * token the layers follow one another, but the rows of different sequences, of different requests, or of layers whose
+ * inputs are ready are independent; each is a launch-bound problem of its own shape, and a table runs them in one
+ * launch: one CTA per (problem, b*h), the whole key range, the result written directly (no split, no workspace).
+ *   problems: HOST array; pointers inside are DEVICE pointers, bf16, layouts as in tlin_decode_step with B*H = BH.
+ *   pos: valid cache rows on entry.  With k_new, v_new given the new row is copied to row pos (bit-exact) and the
+ *   query attends over rows [0, pos]; with k_new = v_new = NULL nothing is written and the query attends over rows
+ *   [0, pos) (a cross-attention to a finished cache; pos >= 1).  0 <= pos < Ncap (pos <= Ncap without append).
+ *   d in {64,128}.  Meant for short caches: a long one keeps a single CTA per (b*h) busy for its whole length.
+ * Tables of more than 48 problems are issued as several launches. */
+typedef struct {
+    const void* q_new;      /* [BH,1,d] */
+    const void* k_new;      /* [BH,1,d] or NULL */
+    const void* v_new;      /* [BH,1,d] or NULL (together with k_new) */
+    void* k_cache;          /* [BH,Ncap,d] */
+    void* v_cache;
+    void* out;              /* [BH,1,d] */
+    float* lse;             /* [BH] or NULL */
+    int32_t BH, Ncap, pos, reserved;
+} tlin_decode_problem;
+int tlin_decode_step_batched(const tlin_decode_problem* problems, int n_problems, int d, tlin_stream_t stream);
 
 /* tlin_decode_step over an 8-bit cache (not in the paper; it halves the cache memory of Section 5.2 and the bytes a step
  * streams).  k_cache, v_cache [B,H,Ncap,d] hold one byte per element: E4M3 codes of the 8-bit floating point format

@@ -33,6 +33,18 @@ class FwdPlan(ctypes.Structure):
                 ("n_keys", ctypes.c_int32), ("n_queries", ctypes.c_int32)]
 
 
+class Problem(ctypes.Structure):
+    _fields_ = [("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("out", ctypes.c_void_p),
+                ("lse", ctypes.c_void_p), ("BH", ctypes.c_int32), ("n_keys", ctypes.c_int32), ("kv_rows", ctypes.c_int32),
+                ("n_queries", ctypes.c_int32), ("causal_window", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class DecodeProblem(ctypes.Structure):
+    _fields_ = [("q_new", ctypes.c_void_p), ("k_new", ctypes.c_void_p), ("v_new", ctypes.c_void_p), ("k_cache", ctypes.c_void_p),
+                ("v_cache", ctypes.c_void_p), ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("BH", ctypes.c_int32),
+                ("Ncap", ctypes.c_int32), ("pos", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
 class DecodePlan(ctypes.Structure):
     _fields_ = [("splits", ctypes.c_int32), ("keys_per_split", ctypes.c_int32), ("n_ctas", ctypes.c_int32),
                 ("workspace_bytes", ctypes.c_int64)]
@@ -46,11 +58,14 @@ SIGNATURES = {
     "tlin_attn_forward_f32": (_i, [_vp] * 5 + [_i] * 6 + [_vp]),
     "tlin_attn_forward_prefixes": (_i, [_vp] * 5 + [_i] * 6 + [_vp, _i, _vp]),
     "tlin_attn_forward_host": (_i, [_vp] * 10 + [_i] * 6 + [_vp]),
+    "tlin_attn_forward_batched": (_i, [_vp, _i, _i, _vp]),
+    "tlin_plan_batched": (_i, [_vp, _i, _i, _vp, _vp]),
     "tlin_attn_forward_cache": (_i, [_vp] * 5 + [_i] * 7 + [_vp]),
     "tlin_attn_backward": (_i, [_vp] * 9 + [_i] * 6 + [_vp]),
     "tlin_attn_backward_f32": (_i, [_vp] * 9 + [_i] * 6 + [_vp]),
     "tlin_decode_step": (_i, [_vp] * 7 + [_i] * 5 + [_vp]),
     "tlin_decode_step_host": (_i, [_vp] * 12 + [_i] * 5 + [_vp]),
+    "tlin_decode_step_batched": (_i, [_vp, _i, _i, _vp]),
     "tlin_decode_step_static": (_i, [_vp] * 7 + [_i] * 5 + [_vp]),
     "tlin_decode_step_ragged": (_i, [_vp] * 7 + [_i] * 3 + [_vp, _i, _i, _vp]),
     "tlin_decode_step_fp8": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
@@ -221,6 +236,46 @@ def tlin_attn_forward_cache(q, k_cache, v_cache, n_keys, out=None, lse=None, cau
     return out, lse
 
 
+def make_problem_table(problems):
+    """ctypes array of Problem from dicts/tuples (q, k, v, out, lse, n_keys, causal_window): q [B,H,W,d] (or [BH,W,d]),
+    k, v [B,H,rows,d] with rows >= n_keys (n_keys None: all rows)."""
+    arr = (Problem * len(problems))()
+    keep = []
+    for i, (q, k, v, out, lse, n_keys, causal) in enumerate(problems):
+        d = q.shape[-1]
+        W = q.shape[-2]
+        bh = q.numel() // (W * d)
+        rows = k.shape[-2]
+        n_keys = rows if n_keys is None else int(n_keys)
+        for t, name in ((q, "q"), (k, "k"), (v, "v"), (out, "out")):
+            if not t.is_cuda or t.dtype != torch.bfloat16 or not t.is_contiguous():
+                raise ValueError(f"problem {i}: {name} must be a contiguous bf16 CUDA tensor")
+        if k.numel() != bh * rows * d or v.shape != k.shape or out.shape != q.shape:
+            raise ValueError(f"problem {i}: shape mismatch")
+        if lse is not None and (lse.dtype != torch.float32 or lse.numel() != bh * W or not lse.is_contiguous()):
+            raise ValueError(f"problem {i}: lse must be contiguous fp32 of {bh * W} elements")
+        arr[i] = Problem(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), None if lse is None else lse.data_ptr(),
+                         bh, n_keys, rows if rows != n_keys else 0, W, int(causal), 0)
+        keep.append((q, k, v, out, lse))
+    return arr, keep
+
+
+def tlin_attn_forward_batched(problems, stream=None):
+    """One launch for a list of problems (q, k, v, out, lse, n_keys, causal_window) sharing one head size."""
+    arr, _keep = make_problem_table(problems)
+    d = problems[0][0].shape[-1]
+    _check(lib().tlin_attn_forward_batched(ctypes.cast(arr, ctypes.c_void_p), len(problems), d, _stream(stream)), "tlin_attn_forward_batched")
+
+
+def tlin_plan_batched(problem_array, num_sms=0):
+    """(starts list of n_ctas + 1 entries) for a ctypes Problem array."""
+    starts = (ctypes.c_int64 * 200)()
+    n = ctypes.c_int32(0)
+    _check(lib().tlin_plan_batched(ctypes.cast(problem_array, ctypes.c_void_p), len(problem_array), num_sms,
+                                   ctypes.cast(starts, ctypes.c_void_p), ctypes.cast(ctypes.pointer(n), ctypes.c_void_p)), "tlin_plan_batched")
+    return [int(starts[i]) for i in range(n.value + 1)]
+
+
 def tlin_attn_forward_f32(q, k, v, out=None, lse=None, causal_window=1, stream=None):
     """fp32 forward (CUDA-core kernel)."""
     B, H, W, d = q.shape
@@ -340,6 +395,28 @@ def tlin_decode_step_ragged(q_new, k_new, v_new, k_cache, v_cache, pos, max_pos,
                                          _ptr(out), _ptr(lse), B, H, Ncap, _ptr(pos), int(max_pos), d, _stream(stream)),
            "tlin_decode_step_ragged")
     return out, lse
+
+
+def tlin_decode_step_batched(problems, stream=None):
+    """One launch for a list of decode problems (q_new, k_new or None, v_new or None, k_cache, v_cache, pos, out, lse)."""
+    arr = (DecodeProblem * len(problems))()
+    for i, (q_new, k_new, v_new, k_cache, v_cache, pos, out, lse) in enumerate(problems):
+        d = k_cache.shape[-1]
+        Ncap = k_cache.shape[-2]
+        bh = k_cache.numel() // (Ncap * d)
+        for t, name in ((q_new, "q_new"), (out, "out")) + (((k_new, "k_new"), (v_new, "v_new")) if k_new is not None else ()):
+            if not t.is_cuda or t.dtype != torch.bfloat16 or not t.is_contiguous() or t.numel() != bh * d:
+                raise ValueError(f"problem {i}: {name} must be contiguous bf16 [BH,1,d]")
+        for t, name in ((k_cache, "k_cache"), (v_cache, "v_cache")):
+            if not t.is_cuda or t.dtype != torch.bfloat16 or not t.is_contiguous() or t.numel() != bh * Ncap * d:
+                raise ValueError(f"problem {i}: {name} must be contiguous bf16 [BH,Ncap,d]")
+        if lse is not None and (lse.dtype != torch.float32 or lse.numel() != bh or not lse.is_contiguous()):
+            raise ValueError(f"problem {i}: lse must be contiguous fp32 [BH]")
+        arr[i] = DecodeProblem(q_new.data_ptr(), None if k_new is None else k_new.data_ptr(), None if v_new is None else v_new.data_ptr(),
+                               k_cache.data_ptr(), v_cache.data_ptr(), out.data_ptr(), None if lse is None else lse.data_ptr(),
+                               bh, Ncap, int(pos), 0)
+    d = problems[0][3].shape[-1]
+    _check(lib().tlin_decode_step_batched(ctypes.cast(arr, ctypes.c_void_p), len(problems), d, _stream(stream)), "tlin_decode_step_batched")
 
 
 def tlin_decode_step_static(q_new, k_new, v_new, k_cache, v_cache, pos, out, lse, stream=None):

@@ -151,6 +151,36 @@ extern "C" int tlin_attn_forward_cache(const void* q, const void* k_cache, const
     return forward_common(q, k_cache, v_cache, out, lse, B, H, n_keys, W, d, causal_window, 0, (cudaStream_t)stream, Ncap);
 }
 
+extern "C" int tlin_attn_forward_batched(const tlin_problem* problems, int n_problems, int d, tlin_stream_t stream) {
+    t_launches = 0;
+    if (!problems || n_problems <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return TLIN_ERR_UNSUPPORTED;
+    // every problem of every chunk is checked before the first launch
+    int64_t starts[kMaxGroups + 1];
+    int32_t n_ctas = 0;
+    for (int first = 0; first < n_problems; first += kMaxBatch) {
+        const int n = n_problems - first < kMaxBatch ? n_problems - first : kMaxBatch;
+        const int rc = tlin_plan_batched(problems + first, n, 0, starts, &n_ctas);
+        if (rc != TLIN_OK) return rc;
+    }
+    int sms = 0;
+    int rc = device_info(&sms);
+    if (rc != TLIN_OK) return rc;
+    for (int first = 0; first < n_problems; first += kMaxBatch) {
+        const int n = n_problems - first < kMaxBatch ? n_problems - first : kMaxBatch;
+        rc = tlin_plan_batched(problems + first, n, sms, starts, &n_ctas);
+        if (rc != TLIN_OK) return rc;
+        if (log_plans())
+            fprintf(stderr, "libtlin: batched forward, problems %d..%d of %d, d=%d -> %lld units on %d ctas\n", first, first + n - 1,
+                    n_problems, d, (long long)starts[n_ctas], n_ctas);
+        long long st[kMaxGroups + 1];
+        for (int g = 0; g <= n_ctas; ++g) st[g] = starts[g];
+        rc = launch_fwd_tc_batched(problems + first, n, d, st, n_ctas, (cudaStream_t)stream);
+        if (rc != TLIN_OK) return rc;
+    }
+    return TLIN_OK;
+}
+
 extern "C" size_t tlin_workspace_bytes_forward_prefixes(int B, int H, int W, int d, int C, const int32_t* n_keys, int causal_window) {
     size_t need = 0;
     if (!n_keys) return 0;
@@ -259,6 +289,32 @@ extern "C" int tlin_decode_step(const void* q_new, const void* k_new, const void
     if (!w.ptr || w.bytes < (size_t)plan.workspace_bytes) return TLIN_ERR_WORKSPACE;
     return launch_decode(q_new, k_new, v_new, k_cache, v_cache, out, lse, B, H, Ncap, pos, nullptr, d, plan,
                          (float*)w.ptr, (cudaStream_t)stream);
+}
+
+extern "C" int tlin_decode_step_batched(const tlin_decode_problem* problems, int n_problems, int d, tlin_stream_t stream) {
+    t_launches = 0;
+    if (!problems || n_problems <= 0 || d <= 0) return TLIN_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return TLIN_ERR_UNSUPPORTED;
+    for (int i = 0; i < n_problems; ++i) {          // every problem is checked before the first launch
+        const tlin_decode_problem& pb = problems[i];
+        if (!pb.q_new || !pb.k_cache || !pb.v_cache || !pb.out) return TLIN_ERR_INVALID_ARG;
+        if ((pb.k_new == nullptr) != (pb.v_new == nullptr)) return TLIN_ERR_INVALID_ARG;
+        if (pb.BH <= 0 || pb.Ncap <= 0) return TLIN_ERR_INVALID_ARG;
+        if (pb.k_new ? (pb.pos < 0 || pb.pos >= pb.Ncap) : (pb.pos < 1 || pb.pos > pb.Ncap)) return TLIN_ERR_INVALID_ARG;
+        if (!aligned16(pb.q_new) || !aligned16(pb.k_new) || !aligned16(pb.v_new) || !aligned16(pb.k_cache) ||
+            !aligned16(pb.v_cache) || !aligned16(pb.out)) return TLIN_ERR_INVALID_ARG;
+        if (pb.lse && (reinterpret_cast<uintptr_t>(pb.lse) & 3u)) return TLIN_ERR_INVALID_ARG;
+    }
+    int sms = 0;
+    int rc = device_info(&sms);
+    if (rc != TLIN_OK) return rc;
+    const int per = decode_table_max_problems();
+    for (int first = 0; first < n_problems; first += per) {
+        const int n = n_problems - first < per ? n_problems - first : per;
+        rc = launch_decode_table(problems + first, n, d, (cudaStream_t)stream);
+        if (rc != TLIN_OK) return rc;
+    }
+    return TLIN_OK;
 }
 
 extern "C" int tlin_decode_step_fp8(const void* q_new, const void* k_new, const void* v_new,

@@ -12,6 +12,7 @@
 #include <cuda_fp16.h>
 #include <math_constants.h>
 #include <mutex>
+#include <string.h>
 
 namespace tlin {
 namespace {
@@ -63,51 +64,21 @@ __device__ __forceinline__ void combine(float& m, float& l, float (&a)[8], float
     m = mn;
 }
 
+// One query row of one (b,h) over keys [j0, j1) of its cache, by all threads of the CTA: the row `pos` (the token being
+// appended in this launch, or -1) is taken from k_new / v_new instead of the cache.  Returns, in threads 0..D-1, column
+// c = threadIdx.x of the un-normalised result `a`, the row sum `ll` and the running maximum `mm` (log2 units).
 template <int D>
-__global__ void __launch_bounds__(kWarps * 32, kDecodeCtasPerSM)
-decode_splitk_kernel(const uint4* __restrict__ q_new, const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
-                     uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
-                     float* __restrict__ part_o, float* __restrict__ part_lse,
-                     int Ncap, int pos_all, const int* __restrict__ pos_per_seq, int H, int* __restrict__ status,
-                     int splits, int kps, float scale_log2e) {
+__device__ __forceinline__ void attend_key_range(const uint4* __restrict__ q_row, const uint4* __restrict__ kn, const uint4* __restrict__ vn,
+                                                 const uint4* __restrict__ kc, const uint4* __restrict__ vc, int j0, int j1, int pos,
+                                                 float scale_log2e, float& a, float& ll, float& mm) {
     constexpr int LPR = D / 8;           // lanes (16-byte chunks) per row
     constexpr int RPW = 32 / LPR;        // rows per warp-load
     constexpr int ROWS_PER_IT = kWarps * RPW * kUnroll;
-    const int bh = blockIdx.x / splits, sp = blockIdx.x - bh * splits;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int sub = lane % LPR, rsel = lane / LPR;
-    // one position for the whole batch, or one per sequence read from device memory (ragged batch)
-    int pos = pos_all;
-    if (pos_per_seq != nullptr) {
-        pos = pos_per_seq[bh / H];
-        if (pos < 0 || pos >= Ncap || pos > pos_all) {   // pos_all is the caller's bound, which sized the splits; the host
-                                                          // cannot see the entries: report, and leave this (b,h) alone
-            if (threadIdx.x == 0) {
-                atomicExch(status, (int)TLIN_ERR_INVALID_ARG);
-                part_lse[(int64_t)bh * splits + sp] = -CUDART_INF_F;
-            }
-            if (threadIdx.x < D) part_o[((int64_t)bh * splits + sp) * D + threadIdx.x] = 0.f;
-            return;
-        }
-    }
-    const int L = pos + 1;
-    const int j0 = sp * kps, j1 = min(L, j0 + kps);
-
-    const uint4* kc = k_cache + (int64_t)bh * Ncap * LPR;
-    const uint4* vc = v_cache + (int64_t)bh * Ncap * LPR;
-    const uint4* kn = k_new + (int64_t)bh * LPR;
-    const uint4* vn = v_new + (int64_t)bh * LPR;
-
-    // append (bit-exact copy) by the CTA whose range holds row `pos`; nobody reads that row from the
-    // cache in this launch -- the lanes below take it from k_new / v_new.
-    if (pos >= j0 && pos < j1 && warp == 0 && lane < LPR) {
-        k_cache[((int64_t)bh * Ncap + pos) * LPR + lane] = kn[lane];
-        v_cache[((int64_t)bh * Ncap + pos) * LPR + lane] = vn[lane];
-    }
-
     float qf[8];
     {
-        const uint4 qv = q_new[(int64_t)bh * LPR + sub];
+        const uint4 qv = q_row[sub];
         qf[0] = bf_lo(qv.x) * scale_log2e; qf[1] = bf_hi(qv.x) * scale_log2e;
         qf[2] = bf_lo(qv.y) * scale_log2e; qf[3] = bf_hi(qv.y) * scale_log2e;
         qf[4] = bf_lo(qv.z) * scale_log2e; qf[5] = bf_hi(qv.z) * scale_log2e;
@@ -178,22 +149,108 @@ decode_splitk_kernel(const uint4* __restrict__ q_new, const uint4* __restrict__ 
         if (sub == 0) { sm_m[warp] = m; sm_l[warp] = l; }
     }
     __syncthreads();
+    a = 0.f; ll = 0.f; mm = -CUDART_INF_F;
     if (threadIdx.x < D) {
         const int c = threadIdx.x;
-        float mm = -CUDART_INF_F;
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) mm = fmaxf(mm, sm_m[w]);
         const float ms = mm == -CUDART_INF_F ? 0.f : mm;
-        float ll = 0.f, a = 0.f;
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) {
             const float c1 = exp2f(sm_m[w] - ms);
             ll += sm_l[w] * c1;
             a += sm_a[w][c] * c1;
         }
+    }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kWarps * 32, kDecodeCtasPerSM)
+decode_splitk_kernel(const uint4* __restrict__ q_new, const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+                     uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
+                     float* __restrict__ part_o, float* __restrict__ part_lse,
+                     int Ncap, int pos_all, const int* __restrict__ pos_per_seq, int H, int* __restrict__ status,
+                     int splits, int kps, float scale_log2e) {
+    constexpr int LPR = D / 8;           // lanes (16-byte chunks) per row
+    const int bh = blockIdx.x / splits, sp = blockIdx.x - bh * splits;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // one position for the whole batch, or one per sequence read from device memory (ragged batch)
+    int pos = pos_all;
+    if (pos_per_seq != nullptr) {
+        pos = pos_per_seq[bh / H];
+        if (pos < 0 || pos >= Ncap || pos > pos_all) {   // pos_all is the caller's bound, which sized the splits; the host
+                                                          // cannot see the entries: report, and leave this (b,h) alone
+            if (threadIdx.x == 0) {
+                atomicExch(status, (int)TLIN_ERR_INVALID_ARG);
+                part_lse[(int64_t)bh * splits + sp] = -CUDART_INF_F;
+            }
+            if (threadIdx.x < D) part_o[((int64_t)bh * splits + sp) * D + threadIdx.x] = 0.f;
+            return;
+        }
+    }
+    const int L = pos + 1;
+    const int j0 = sp * kps, j1 = min(L, j0 + kps);
+
+    const uint4* kc = k_cache + (int64_t)bh * Ncap * LPR;
+    const uint4* vc = v_cache + (int64_t)bh * Ncap * LPR;
+    const uint4* kn = k_new + (int64_t)bh * LPR;
+    const uint4* vn = v_new + (int64_t)bh * LPR;
+
+    // append (bit-exact copy) by the CTA whose range holds row `pos`; nobody reads that row from the
+    // cache in this launch -- the lanes below take it from k_new / v_new.
+    if (pos >= j0 && pos < j1 && warp == 0 && lane < LPR) {
+        k_cache[((int64_t)bh * Ncap + pos) * LPR + lane] = kn[lane];
+        v_cache[((int64_t)bh * Ncap + pos) * LPR + lane] = vn[lane];
+    }
+
+    float a, ll, mm;
+    attend_key_range<D>(q_new + (int64_t)bh * LPR, kn, vn, kc, vc, j0, j1, pos, scale_log2e, a, ll, mm);
+    if (threadIdx.x < D) {
+        const int c = threadIdx.x;
         const int64_t slot = (int64_t)bh * splits + sp;
         part_o[slot * D + c] = ll > 0.f ? a / ll : 0.f;
         if (c == 0) part_lse[slot] = ll > 0.f ? (mm + log2f(ll)) * kLn2 : -CUDART_INF_F;
+    }
+}
+
+// A table of decode problems as one launch: one CTA per (problem, b*h), whole key range, result written directly (no
+// split, no second kernel).  Meant for the per-layer caches of a block, which are short (Appendix A, cache hit: the
+// (H+1) D W_oh term -- one row against the W_oh summary tokens of a layer -- and the row inside the window).
+struct DecodeProblemDev {
+    const uint4* q_new; const uint4* k_new; const uint4* v_new;   // k_new == null: attend only, nothing is appended
+    uint4* k_cache; uint4* v_cache;
+    __nv_bfloat16* out; float* lse;
+    int cta0, Ncap, pos;
+};
+constexpr int kMaxDecodeBatch = 48;
+struct DecodeTable { DecodeProblemDev prob[kMaxDecodeBatch]; int n; };
+
+template <int D>
+__global__ void __launch_bounds__(kWarps * 32, kDecodeCtasPerSM)
+decode_table_kernel(const __grid_constant__ DecodeTable tbl, float scale_log2e) {
+    constexpr int LPR = D / 8;
+    int pi = 0;
+    while (pi + 1 < tbl.n && (int)blockIdx.x >= tbl.prob[pi + 1].cta0) ++pi;
+    const DecodeProblemDev& pr = tbl.prob[pi];
+    const int bh = blockIdx.x - pr.cta0;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool append = pr.k_new != nullptr;
+    const int pos = append ? pr.pos : -1;              // row taken from k_new / v_new instead of the cache
+    const int L = append ? pr.pos + 1 : pr.pos;
+    const uint4* kc = pr.k_cache + (int64_t)bh * pr.Ncap * LPR;
+    const uint4* vc = pr.v_cache + (int64_t)bh * pr.Ncap * LPR;
+    const uint4* kn = append ? pr.k_new + (int64_t)bh * LPR : kc;
+    const uint4* vn = append ? pr.v_new + (int64_t)bh * LPR : vc;
+    if (append && warp == 0 && lane < LPR) {
+        pr.k_cache[((int64_t)bh * pr.Ncap + pos) * LPR + lane] = kn[lane];
+        pr.v_cache[((int64_t)bh * pr.Ncap + pos) * LPR + lane] = vn[lane];
+    }
+    float a, ll, mm;
+    attend_key_range<D>(pr.q_new + (int64_t)bh * LPR, kn, vn, kc, vc, 0, L, pos, scale_log2e, a, ll, mm);
+    if (threadIdx.x < D) {
+        const int c = threadIdx.x;
+        pr.out[(int64_t)bh * D + c] = __float2bfloat16_rn(ll > 0.f ? a / ll : 0.f);
+        if (pr.lse != nullptr && c == 0) pr.lse[bh] = ll > 0.f ? (mm + log2f(ll)) * kLn2 : -CUDART_INF_F;
     }
 }
 
@@ -458,7 +515,37 @@ int launch_fp8_d(const void* q_new, const void* k_new, const void* v_new, void* 
     return TLIN_OK;
 }
 
+template <int D>
+int launch_table_d(const tlin_decode_problem* problems, int n, cudaStream_t st) {
+    DecodeTable tbl;
+    memset(&tbl, 0, sizeof(tbl));
+    tbl.n = n;
+    long long ctas = 0;
+    for (int i = 0; i < n; ++i) {
+        const tlin_decode_problem& pb = problems[i];
+        DecodeProblemDev& pd = tbl.prob[i];
+        pd.q_new = (const uint4*)pb.q_new; pd.k_new = (const uint4*)pb.k_new; pd.v_new = (const uint4*)pb.v_new;
+        pd.k_cache = (uint4*)pb.k_cache; pd.v_cache = (uint4*)pb.v_cache;
+        pd.out = (__nv_bfloat16*)pb.out; pd.lse = pb.lse;
+        pd.cta0 = (int)ctas; pd.Ncap = pb.Ncap; pd.pos = pb.pos;
+        ctas += pb.BH;
+    }
+    if (ctas > 0x7fffffffLL) return TLIN_ERR_UNSUPPORTED;
+    decode_table_kernel<D><<<(unsigned)ctas, kWarps * 32, 0, st>>>(tbl, kLog2e / sqrtf((float)D));
+    TLIN_CUDA_CHECK(cudaGetLastError());
+    count_launch();
+    return TLIN_OK;
+}
+
 }  // namespace
+
+int decode_table_max_problems() { return kMaxDecodeBatch; }
+int launch_decode_table(const tlin_decode_problem* problems, int n, int d, cudaStream_t st) {
+    if (n <= 0 || n > kMaxDecodeBatch) return TLIN_ERR_INVALID_ARG;
+    if (d == 128) return launch_table_d<128>(problems, n, st);
+    if (d == 64) return launch_table_d<64>(problems, n, st);
+    return TLIN_ERR_UNSUPPORTED;
+}
 
 int launch_decode_fp8(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                       const float* k_scale, const float* v_scale, void* out, float* lse, int B, int H, int Ncap, int pos,

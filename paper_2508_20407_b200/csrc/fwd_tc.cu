@@ -22,6 +22,7 @@
 #include "tc_common.cuh"
 #include <math_constants.h>
 #include <mutex>
+#include <string.h>
 
 namespace tlin {
 namespace {
@@ -76,6 +77,23 @@ struct Cfg {
     static constexpr uint32_t kColS = 0, kColO = 256;
 };
 
+// One problem of a batched launch as the kernel sees it (the field names N, W, causal, key_tiles are the ones the
+// helpers shared with the single-problem kernel read).
+struct ProblemDev {
+    void* out;            // [BH, W, D] bf16
+    float* lse;           // [BH, W] or null
+    long long unit0;      // first unit of this problem in the launch's list: unit = unit0 + bh * q_tiles + q tile pair
+    int N, W, causal, key_tiles, q_tiles;
+};
+// What a launch reads its tensors through: three tensor maps, or a table of them with the problems' shapes.
+template <bool kBatched> struct KernelMaps;
+template <> struct KernelMaps<false> { CUtensorMap q, k, v; };
+template <> struct KernelMaps<true> {
+    CUtensorMap q[kMaxBatch], k[kMaxBatch], v[kMaxBatch];
+    ProblemDev prob[kMaxBatch];
+    int n;
+};
+
 struct Params {
     void* out;            // [B*H, W, D] bf16
     float* lse;           // [B*H, W] or null
@@ -88,10 +106,42 @@ struct Params {
     float scale_log2e;
 };
 
-template <int D>
+// Walks the units of a batched launch: whole problems, in table order.
+struct BatchWalker {
+    long long u, u1;
+    const ProblemDev* prob;
+    int n, pi;
+    __device__ BatchWalker(const KernelMaps<true>& m, const GroupStarts& starts)
+        : u(starts.u[blockIdx.x]), u1(starts.u[blockIdx.x + 1]), prob(m.prob), n(m.n), pi(0) {}
+    __device__ bool next(Segment& s) {
+        if (u >= u1) return false;
+        while (pi + 1 < n && u >= prob[pi + 1].unit0) ++pi;
+        const long long r = u - prob[pi].unit0;
+        s.bh = (int)(r / prob[pi].q_tiles);
+        s.qt = (int)(r - (long long)s.bh * prob[pi].q_tiles);
+        s.t_begin = 0;
+        s.t_end = prob[pi].key_tiles;
+        s.prob = pi;
+        ++u;
+        return true;
+    }
+};
+template <bool kBatched>
+__device__ __forceinline__ auto make_walker(const KernelMaps<kBatched>& m, const Params& p, const GroupStarts& starts) {
+    if constexpr (kBatched) return BatchWalker(m, starts);
+    else return SegmentWalker(p, starts);
+}
+// shape (N, W, causal, key_tiles) and result pointers of the problem a segment belongs to
+template <bool kBatched>
+__device__ __forceinline__ decltype(auto) problem_of(const KernelMaps<kBatched>& m, const Params& p, const Segment& s) {
+    if constexpr (kBatched) return (m.prob[s.prob]);
+    else return (p);
+}
+
+template <int D, bool kBatched>
 __global__ void __launch_bounds__(kThreads, 1)
-fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-              const __grid_constant__ CUtensorMap map_v, const Params p, const __grid_constant__ GroupStarts starts) {
+fwd_tc_kernel(const __grid_constant__ KernelMaps<kBatched> maps, const __grid_constant__ Params p,
+              const __grid_constant__ GroupStarts starts) {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -132,10 +182,12 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         tmem_alloc(tmem_slot, 512);
         tmem_relinquish();
     }
-    if (warp == kProducerWarp && lane == 0) {
-        prefetch_tensormap(&map_q);
-        prefetch_tensormap(&map_k);
-        prefetch_tensormap(&map_v);
+    if constexpr (!kBatched) {
+        if (warp == kProducerWarp && lane == 0) {
+            prefetch_tensormap(&maps.q);
+            prefetch_tensormap(&maps.k);
+            prefetch_tensormap(&maps.v);
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -152,11 +204,17 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             uint32_t it = 0;           // ring counter
             uint32_t seg_idx = 0;
             bool ok = true;
-            SegmentWalker walk(p, starts);
+            auto walk = make_walker<kBatched>(maps, p, starts);
             Segment s;
             while (ok && walk.next(s)) {
+                const auto& pr = problem_of<kBatched>(maps, p, s);
+                const CUtensorMap* map_q_p;
+                const CUtensorMap* map_k_p;
+                const CUtensorMap* map_v_p;
+                if constexpr (kBatched) { map_q_p = &maps.q[s.prob]; map_k_p = &maps.k[s.prob]; map_v_p = &maps.v[s.prob]; }
+                else { map_q_p = &maps.q; map_k_p = &maps.k; map_v_p = &maps.v; }
                 const int row0 = s.qt * kTileM;
-                const int c0 = seg_count(s, tiles_allowed(p, row0, 0)), c1 = seg_count(s, tiles_allowed(p, row0, 1));
+                const int c0 = seg_count(s, tiles_allowed(pr, row0, 0)), c1 = seg_count(s, tiles_allowed(pr, row0, 1));
                 const int cnt = c0 > c1 ? c0 : c1;
                 if (cnt == 0) continue;
                 if (seg_idx > 0) ok = mbar_wait(q_empty, (seg_idx - 1) & 1, abort_p);
@@ -164,7 +222,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 mbar_arrive_expect_tx(q_full, 2 * C::kTileBytes);
                 for (int i = 0; i < 2; ++i)
                     for (int b = 0; b < C::kBoxes; ++b)
-                        tma_load_3d(sQ + i * C::kTileBytes + b * (kQTile * 128), &map_q, q_full, b * 64, row0 + i * kQTile, s.bh);
+                        tma_load_3d(sQ + i * C::kTileBytes + b * (kQTile * 128), map_q_p, q_full, b * 64, row0 + i * kQTile, s.bh);
                 for (int j = 0; j < cnt && ok; ++j) {
                     const int t = s.t_begin + j;
                     for (int kv = 0; kv < 2 && ok; ++kv) {
@@ -174,7 +232,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                         mbar_arrive_expect_tx(&kv_full[slot], C::kTileBytes);
                         uint8_t* dst = sRing + slot * C::kTileBytes;
                         for (int b = 0; b < C::kBoxes; ++b)
-                            tma_load_3d(dst + b * (kQTile * 128), kv == 0 ? &map_k : &map_v, &kv_full[slot], b * 64, t * kTileN, s.bh);
+                            tma_load_3d(dst + b * (kQTile * 128), kv == 0 ? map_k_p : map_v_p, &kv_full[slot], b * 64, t * kTileN, s.bh);
                         ++it;
                     }
                 }
@@ -233,11 +291,12 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 }
                 if (half == 1) commit_elected(&pv_done[i]);
             };
-            SegmentWalker walk(p, starts);
+            auto walk = make_walker<kBatched>(maps, p, starts);
             Segment s;
             while (ok && walk.next(s)) {
+                const auto& pr = problem_of<kBatched>(maps, p, s);
                 const int row0 = s.qt * kTileM;
-                const int c0 = seg_count(s, tiles_allowed(p, row0, 0)), c1 = seg_count(s, tiles_allowed(p, row0, 1));
+                const int c0 = seg_count(s, tiles_allowed(pr, row0, 0)), c1 = seg_count(s, tiles_allowed(pr, row0, 1));
                 const int cnt = c0 > c1 ? c0 : c1;
                 if (cnt == 0) continue;
                 const int cq[2] = {c0, c1};
@@ -304,18 +363,20 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         const uint32_t tO = tmem_base + lane_addr + C::kColO + i * D;
         uint32_t n = 0;     // tiles processed by this warpgroup (phase counter of s_full/p_full/pv_done)
         bool ok = true;
-        SegmentWalker walk(p, starts);
-        const int bh_first = (int)(walk.u / p.key_tiles);  // (b,h) of this CTA's first unit (used under schedule 0 only)
+        auto walk = make_walker<kBatched>(maps, p, starts);
+        int bh_first = 0;                                  // (b,h) of this CTA's first unit (used under schedule 0 only)
+        if constexpr (!kBatched) bh_first = (int)(walk.u / p.key_tiles);
         Segment s;
         while (ok && walk.next(s)) {
+            const auto& pr = problem_of<kBatched>(maps, p, s);
             const int row0 = s.qt * kTileM;
             const int row = row0 + i * kQTile + r;         // row inside W (may lie beyond W: computed, never stored)
-            const int allowed_i = tiles_allowed(p, row0, i);
+            const int allowed_i = tiles_allowed(pr, row0, i);
             // keys visible to this row, and to the first row of this warp (the smallest in the warp)
-            const long long lim_row_ll = p.causal ? (long long)p.N - p.W + row + 1 : (long long)p.N;
-            const int lim_row = (int)(lim_row_ll < p.N ? lim_row_ll : p.N);
-            const long long lim_warp_ll = p.causal ? (long long)p.N - p.W + (row - lane) + 1 : (long long)p.N;
-            const int lim_warp = (int)(lim_warp_ll < p.N ? lim_warp_ll : p.N);
+            const long long lim_row_ll = pr.causal ? (long long)pr.N - pr.W + row + 1 : (long long)pr.N;
+            const int lim_row = (int)(lim_row_ll < pr.N ? lim_row_ll : pr.N);
+            const long long lim_warp_ll = pr.causal ? (long long)pr.N - pr.W + (row - lane) + 1 : (long long)pr.N;
+            const int lim_warp = (int)(lim_warp_ll < pr.N ? lim_warp_ll : pr.N);
             const int cnt_i = seg_count(s, allowed_i);
             float m_ref = -CUDART_INF_F;
             uint64_t l2[2] = {0ull, 0ull};          // four partial row sums as two packed fp32 pairs
@@ -413,7 +474,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             if (!ok) break;
             if (allowed_i == 0) continue;                  // this Q tile does not exist: nothing to write
             // ---------------------------------------------------------------- epilogue of the segment
-            const bool whole = s.t_begin == 0 && s.t_end == p.key_tiles;
+            const bool whole = kBatched || (s.t_begin == 0 && s.t_end == p.key_tiles);
             if (cnt_i > 0) {
                 ok = mbar_wait(&pv_done[i], (n - 1) & 1, abort_p);
                 ok = __all_sync(0xffffffffu, ok);
@@ -429,7 +490,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             }
             const float inv_l = l > 0.f ? 1.f / l : 0.f;
             const float lse_val = l > 0.f ? (m_ref + log2f(l)) * kLn2 : -CUDART_INF_F;
-            const bool store = row < p.W;
+            const bool store = row < pr.W;
             // partial result -> workspace slot (0: first segment of this CTA's range, 1: a later one)
             float* pbase = p.ws + ((long long)blockIdx.x * 2 + (s.bh == bh_first ? 0 : 1)) * (long long)kTileM * (D + 1);
             // A thread holds one row.  Stored straight from the registers a warp's store would touch 32 different lines, so
@@ -438,7 +499,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             uint8_t* stage = sStage + warp * (32 * 128);
             const int row_warp = row - lane;                   // row of lane 0
             if (whole) {
-                __nv_bfloat16* owarp = reinterpret_cast<__nv_bfloat16*>(p.out) + ((long long)s.bh * p.W + row_warp) * D;
+                __nv_bfloat16* owarp = reinterpret_cast<__nv_bfloat16*>(pr.out) + ((long long)s.bh * pr.W + row_warp) * D;
 #pragma unroll
                 for (int h = 0; h < D / 64; ++h) {             // 64 bf16 columns per pass
 #pragma unroll
@@ -466,7 +527,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     for (int it = 0; it < 8; ++it) {
                         const int rrow = it * 4 + (lane >> 3), piece = lane & 7;
                         const uint4 w = *reinterpret_cast<const uint4*>(stage + rrow * 128 + ((piece ^ (rrow & 7)) << 4));
-                        if (row_warp + rrow < p.W) *reinterpret_cast<uint4*>(owarp + (long long)rrow * D + h * 64 + piece * 8) = w;
+                        if (row_warp + rrow < pr.W) *reinterpret_cast<uint4*>(owarp + (long long)rrow * D + h * 64 + piece * 8) = w;
                     }
                     __syncwarp();
                 }
@@ -505,7 +566,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 }
             }
             if (whole) {
-                if (store && p.lse != nullptr) p.lse[(long long)s.bh * p.W + row] = lse_val;
+                if (store && pr.lse != nullptr) pr.lse[(long long)s.bh * pr.W + row] = lse_val;
             } else {
                 pbase[(long long)kTileM * D + i * kQTile + r] = lse_val;
             }
@@ -619,10 +680,10 @@ int launch_d(const void* q, const void* k, const void* v, void* out, float* lse,
              int causal, const tlin_fwd_plan& plan, float* ws, long long kv_rows_alloc, cudaStream_t st) {
     using C = Cfg<D>;
     const long long bh = (long long)B * H;
-    CUtensorMap mq, mk, mv;
-    int rc = make_map(&mq, q, D, W, bh);
-    if (rc == TLIN_OK) rc = make_map(&mk, k, D, N, bh, kQTile, kv_rows_alloc);
-    if (rc == TLIN_OK) rc = make_map(&mv, v, D, N, bh, kQTile, kv_rows_alloc);
+    KernelMaps<false> maps;
+    int rc = make_map(&maps.q, q, D, W, bh);
+    if (rc == TLIN_OK) rc = make_map(&maps.k, k, D, N, bh, kQTile, kv_rows_alloc);
+    if (rc == TLIN_OK) rc = make_map(&maps.v, v, D, N, bh, kQTile, kv_rows_alloc);
     if (rc != TLIN_OK) return rc;
     Params p;
     p.out = out; p.lse = lse; p.ws = ws; p.status = status_word();
@@ -631,11 +692,11 @@ int launch_d(const void* q, const void* k, const void* v, void* out, float* lse,
     p.N = N; p.W = W; p.causal = causal; p.schedule = plan.schedule;
     p.scale_log2e = kLog2e / sqrtf((float)D);
     static bool smem_allowed[64] = {};
-    TLIN_CUDA_CHECK(allow_dynamic_smem(fwd_tc_kernel<D>, C::kSmemBytes, smem_allowed));
+    TLIN_CUDA_CHECK(allow_dynamic_smem(fwd_tc_kernel<D, false>, C::kSmemBytes, smem_allowed));
     if (plan.n_groups > kMaxGroups) return TLIN_ERR_UNSUPPORTED;
     GroupStarts starts;
     fwd_group_starts(plan, &starts);
-    fwd_tc_kernel<D><<<plan.n_ctas, kThreads, C::kSmemBytes, st>>>(mq, mk, mv, p, starts);
+    fwd_tc_kernel<D, false><<<plan.n_ctas, kThreads, C::kSmemBytes, st>>>(maps, p, starts);
     TLIN_CUDA_CHECK(cudaGetLastError());
     count_launch();
     if (plan.uses_workspace) {
@@ -646,7 +707,54 @@ int launch_d(const void* q, const void* k, const void* v, void* out, float* lse,
     return TLIN_OK;
 }
 
+// A table of problems as one launch: every CTA walks a contiguous run of whole (problem, b*h, query tile pair) units.
+template <int D>
+int launch_batched_d(const tlin_problem* problems, int n, const long long* starts_in, int n_ctas, cudaStream_t st) {
+    using C = Cfg<D>;
+    static_assert(sizeof(KernelMaps<true>) + sizeof(Params) + sizeof(GroupStarts) < 32000, "launch parameters exceed the limit");
+    KernelMaps<true> maps;
+    memset(&maps, 0, sizeof(maps));
+    maps.n = n;
+    long long unit = 0;
+    for (int i = 0; i < n; ++i) {
+        const tlin_problem& pb = problems[i];
+        const long long kv_rows = pb.kv_rows > 0 ? pb.kv_rows : pb.n_keys;
+        int rc = make_map(&maps.q[i], pb.q, D, pb.n_queries, pb.BH);
+        if (rc == TLIN_OK) rc = make_map(&maps.k[i], pb.k, D, pb.n_keys, pb.BH, kQTile, kv_rows);
+        if (rc == TLIN_OK) rc = make_map(&maps.v[i], pb.v, D, pb.n_keys, pb.BH, kQTile, kv_rows);
+        if (rc != TLIN_OK) return rc;
+        ProblemDev& pd = maps.prob[i];
+        pd.out = pb.out; pd.lse = pb.lse; pd.unit0 = unit;
+        pd.N = pb.n_keys; pd.W = pb.n_queries; pd.causal = pb.causal_window;
+        pd.key_tiles = (pb.n_keys + kTileN - 1) / kTileN;
+        pd.q_tiles = (pb.n_queries + kTileM - 1) / kTileM;
+        unit += (long long)pb.BH * pd.q_tiles;
+    }
+    Params p;
+    memset(&p, 0, sizeof(p));
+    p.status = status_word();
+    if (!p.status) return TLIN_ERR_CUDA;
+    p.total_units = unit; p.n_groups = n_ctas; p.q_tiles = 1; p.key_tiles = 1; p.schedule = 1;
+    p.scale_log2e = kLog2e / sqrtf((float)D);
+    if (n_ctas > kMaxGroups) return TLIN_ERR_UNSUPPORTED;
+    GroupStarts starts;
+    for (int g = 0; g <= n_ctas; ++g) starts.u[g] = starts_in[g];
+    static bool smem_allowed[64] = {};
+    TLIN_CUDA_CHECK(allow_dynamic_smem(fwd_tc_kernel<D, true>, C::kSmemBytes, smem_allowed));
+    fwd_tc_kernel<D, true><<<n_ctas, kThreads, C::kSmemBytes, st>>>(maps, p, starts);
+    TLIN_CUDA_CHECK(cudaGetLastError());
+    count_launch();
+    return TLIN_OK;
+}
+
 }  // namespace
+
+int launch_fwd_tc_batched(const tlin_problem* problems, int n, int d, const long long* starts, int n_ctas, cudaStream_t st) {
+    if (n <= 0 || n > kMaxBatch) return TLIN_ERR_INVALID_ARG;
+    if (d == 128) return launch_batched_d<128>(problems, n, starts, n_ctas, st);
+    if (d == 64) return launch_batched_d<64>(problems, n, starts, n_ctas, st);
+    return TLIN_ERR_UNSUPPORTED;
+}
 
 int launch_fwd_tc(const void* q, const void* k, const void* v, void* out, float* lse,
                   int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& plan,

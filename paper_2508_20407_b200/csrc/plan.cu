@@ -92,6 +92,78 @@ void tlin::fwd_group_starts(const tlin_fwd_plan& plan, GroupStarts* starts) {
     starts->u[G] = U;
 }
 
+// Contiguous runs of units, one per CTA, every run non-empty: the costliest run as cheap as contiguous runs allow, and
+// within that as close as possible to equal shares of the total (run c starting where the cost before it reaches
+// c/n of the total).
+void tlin::balanced_run_starts(const long long* prefix, long long U, int G, long long* starts) {
+    const long long total = prefix[U];
+    long long biggest = 0;
+    for (long long x = 0; x < U; ++x) biggest = std::max(biggest, prefix[x + 1] - prefix[x]);
+    auto last_le = [&](long long v) { return (long long)(std::upper_bound(prefix, prefix + U + 1, v) - prefix) - 1; };   // largest x with prefix[x] <= v
+    auto first_ge = [&](long long v) { return (long long)(std::lower_bound(prefix, prefix + U + 1, v) - prefix); };       // smallest x with prefix[x] >= v
+    auto feasible = [&](long long cap) {
+        long long pos = 0;
+        for (int g = 0; g < G && pos < U; ++g) pos = last_le(prefix[pos] + cap);
+        return pos >= U;
+    };
+    long long cap = std::max(biggest, (total + G - 1) / G), hi = (total + G - 1) / G + biggest;
+    while (cap < hi) {
+        const long long mid = (cap + hi) / 2;
+        if (feasible(mid)) hi = mid; else cap = mid + 1;
+    }
+    std::vector<long long> earliest((size_t)G + 1);
+    earliest[G] = U;
+    for (int g = G - 1; g >= 0; --g) earliest[g] = first_ge(prefix[earliest[g + 1]] - cap);
+    starts[0] = 0;
+    for (int g = 0; g + 1 < G; ++g) {
+        const long long from = starts[g];
+        const long long lo = std::max(earliest[g + 1], from), up = last_le(prefix[from] + cap);
+        const long long want = first_ge((long long)(((unsigned long long)(g + 1) * (unsigned long long)total) / (unsigned)G));
+        long long x = std::min(std::max(want, lo), up);
+        // no run is empty (G <= U): at least one unit for this CTA, and one left for each of the CTAs after it
+        x = std::max(x, from + 1);
+        x = std::min(x, U - (G - 1 - g));
+        starts[g + 1] = x;
+    }
+    starts[G] = U;
+}
+
+static int check_problem(const tlin_problem& pb) {
+    if (!pb.q || !pb.k || !pb.v || !pb.out) return TLIN_ERR_INVALID_ARG;
+    if (pb.BH <= 0 || pb.n_keys <= 0 || pb.n_queries <= 0) return TLIN_ERR_INVALID_ARG;
+    if (pb.causal_window != 0 && pb.causal_window != 1) return TLIN_ERR_INVALID_ARG;
+    if (pb.causal_window && pb.n_keys < pb.n_queries) return TLIN_ERR_INVALID_ARG;
+    if (pb.kv_rows != 0 && pb.kv_rows < pb.n_keys) return TLIN_ERR_INVALID_ARG;
+    const uintptr_t all = (uintptr_t)pb.q | (uintptr_t)pb.k | (uintptr_t)pb.v | (uintptr_t)pb.out;
+    if (all & 15u) return TLIN_ERR_INVALID_ARG;
+    if (pb.lse && ((uintptr_t)pb.lse & 3u)) return TLIN_ERR_INVALID_ARG;
+    return TLIN_OK;
+}
+
+extern "C" int tlin_plan_batched(const tlin_problem* problems, int n_problems, int num_sms, int64_t* starts, int32_t* n_ctas) {
+    if (!problems || !starts || !n_ctas || n_problems <= 0 || n_problems > kMaxBatch) return TLIN_ERR_INVALID_ARG;
+    if (num_sms <= 0) num_sms = kDefaultSMs;
+    if (num_sms > kMaxGroups) num_sms = kMaxGroups;
+    std::vector<long long> prefix(1, 0);
+    for (int i = 0; i < n_problems; ++i) {
+        const tlin_problem& pb = problems[i];
+        const int rc = check_problem(pb);
+        if (rc != TLIN_OK) return rc;
+        const int key_tiles = (pb.n_keys + kTileN - 1) / kTileN, q_tiles = (pb.n_queries + 255) / 256;
+        if ((long long)pb.BH * pb.n_queries > 0x7fffffffLL) return TLIN_ERR_UNSUPPORTED;
+        for (int bh = 0; bh < pb.BH; ++bh)
+            for (int qt = 0; qt < q_tiles; ++qt)
+                prefix.push_back(prefix.back() + (pb.causal_window ? fwd_problem_cost(pb.n_keys, pb.n_queries, key_tiles, qt) : key_tiles + 2));
+    }
+    const long long U = (long long)prefix.size() - 1;
+    const int G = (int)std::min<long long>(num_sms, U);
+    std::vector<long long> st((size_t)G + 1);
+    balanced_run_starts(prefix.data(), U, G, st.data());
+    for (int g = 0; g <= G; ++g) starts[g] = st[g];
+    *n_ctas = G;
+    return TLIN_OK;
+}
+
 extern "C" int64_t tlin_plan_group_start(const tlin_fwd_plan* plan, int g) {
     if (!plan || plan->n_groups <= 0) return 0;
     if (g <= 0) return 0;

@@ -17,7 +17,7 @@ constexpr int kTileM = 2 * kQTile;          // query rows per CTA
 // Work of one CTA as a list of segments: a (b,h), a pair of Q tiles (256 query rows) and a range of key tiles.
 // Schedule 0: CTA = (group, q-tile pair); the group's unit range [u, u1) over (b,h,key tile) is cut at the (b,h)
 // borders.  Schedule 1: the units are whole (b,h,q-tile pair) problems and a CTA takes a contiguous run of them.
-struct Segment { int bh, qt, t_begin, t_end; };
+struct Segment { int bh, qt, t_begin, t_end, prob; };    // prob: index into the problem table of a batched launch (else 0)
 
 // The first unit of every group comes from the host as a launch parameter (GroupStarts, in the constant bank).
 struct SegmentWalker {
@@ -32,6 +32,7 @@ struct SegmentWalker {
     }
     __device__ bool next(Segment& s) {
         if (u >= u1) return false;
+        s.prob = 0;
         if (schedule != 0) {
             s.bh = (int)(u / q_tiles);
             s.qt = (int)(u - (long long)s.bh * q_tiles);

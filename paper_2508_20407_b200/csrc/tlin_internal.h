@@ -95,6 +95,13 @@ __host__ __device__ inline long long bwd_first_unit_of_share(int N, int W, int c
     return bh * T + t;
 }
 
+// Batched forward (a table of small problems in one launch).  Units are whole (problem, b*h, 256-row query tile pair)
+// problems in table order; a CTA takes a contiguous run of them, the runs balanced by cost (allowed key tiles + 2) with
+// the costliest run as cheap as contiguous runs allow.  prefix[x] = cost of the first x units (prefix.size() = units + 1);
+// fills starts[0 .. n_ctas], every CTA non-empty (n_ctas <= units).
+constexpr int kMaxBatch = 24;          // problems per launch of the batched kernel (its table travels as a launch parameter)
+void balanced_run_starts(const long long* prefix, long long units, int n_ctas, long long* starts);
+
 #define TLIN_CUDA_CHECK(expr)                                                              \
     do {                                                                                   \
         cudaError_t e__ = (expr);                                                          \
@@ -113,6 +120,7 @@ int launch_fwd_simt_f32(const float* q, const float* k, const float* v, float* o
 int launch_fwd_tc(const void* q, const void* k, const void* v, void* out, float* lse,
                   int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& plan,
                   float* ws, long long kv_rows_alloc, cudaStream_t st);   // kv_rows_alloc: rows per (b,h) of k, v (0 = N)
+int launch_fwd_tc_batched(const tlin_problem* problems, int n, int d, const long long* starts, int n_ctas, cudaStream_t st);
 int launch_decode(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                   void* out, float* lse, int B, int H, int Ncap, int pos, const int* pos_per_seq, int d,
                   const tlin_decode_plan& plan, float* ws, cudaStream_t st);
@@ -124,6 +132,8 @@ int launch_bwd_tc(const void* q, const void* k, const void* v, const void* out, 
                   void* dq, void* dk, void* dv, int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& plan,
                   float* ws, int num_sms, cudaStream_t st);
 size_t bwd_tc_workspace_bytes(long long B, long long H, long long W, int d, const tlin_fwd_plan& plan);
+int decode_table_max_problems();
+int launch_decode_table(const tlin_decode_problem* problems, int n, int d, cudaStream_t st);
 int launch_decode_fp8(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
                       const float* k_scale, const float* v_scale, void* out, float* lse, int B, int H, int Ncap, int pos,
                       int d, const tlin_decode_plan& plan, float* ws, cudaStream_t st);

@@ -267,3 +267,82 @@ def test_backward_key_tile_shares_cover_everything_and_balance_the_steps():
         mean = sum(loads) / G
         assert max(loads) <= mean + Qt and min(loads) >= mean - Qt             # within one key tile's full cost of the mean
     assert L.tlin_plan_backward_share_start(1, 1, 10, 20, 1, 0, 4) == -1       # N < W with the window rule
+
+
+def _problem_array(specs):
+    """ctypes Problem array from (BH, n_keys, n_queries, causal) with dummy aligned pointers (never dereferenced)."""
+    arr = (tl.Problem * len(specs))()
+    for i, (bh, n, w, causal) in enumerate(specs):
+        arr[i] = tl.Problem(16, 32, 48, 64, None, bh, n, 0, w, causal, 0)
+    return arr
+
+
+def _unit_costs(specs):
+    costs = []
+    for (bh, n, w, causal) in specs:
+        key_tiles, q_tiles = -(-n // 128), -(-w // 256)
+        per_qt = []
+        for qt in range(q_tiles):
+            if causal:
+                rows_end = min(w, (qt + 1) * 256)
+                per_qt.append(min(key_tiles, -(-(n - w + rows_end) // 128)) + 2)
+            else:
+                per_qt.append(key_tiles + 2)
+        costs.extend(per_qt * bh)
+    return costs
+
+
+@pytest.mark.parametrize("specs", [
+    [(32, 1024, 1024, 0), (32, 2048, 1024, 1)],                     # an inner context layer and an inner generation layer
+    [(3, 100, 40, 0), (3, 333, 40, 0), (3, 1000, 40, 0)],            # three key prefixes of one sequence
+    [(1, 128, 128, 1)],                                               # a single unit
+    [(8, 4096, 4096, 1), (2, 300, 5000, 0), (40, 64, 64, 1)],         # very uneven units
+    [(1, 256, 256, 1)] * 24,
+])
+def test_batched_plan_gives_every_cta_a_contiguous_non_empty_run_with_the_cheapest_possible_maximum(specs):
+    costs = _unit_costs(specs)
+    U = len(costs)
+    starts = tl.tlin_plan_batched(_problem_array(specs))
+    G = len(starts) - 1
+    assert G == min(148, U) and starts[0] == 0 and starts[-1] == U
+    assert all(b > a for a, b in zip(starts, starts[1:]))
+    runs = [sum(costs[a:b]) for a, b in zip(starts, starts[1:])]
+    # the cheapest possible maximum over all splits into G contiguous non-empty runs, by bisection with a greedy check
+    def fits(cap):
+        g, acc = 1, 0
+        for c in costs:
+            if c > cap:
+                return False
+            if acc + c > cap:
+                g, acc = g + 1, 0
+            acc += c
+        return g <= G
+    lo, hi = max(costs), sum(costs)
+    while lo < hi:
+        mid = (lo + hi) // 2
+        lo, hi = (lo, mid) if fits(mid) else (mid + 1, hi)
+    assert max(runs) == lo
+
+
+def test_batched_plan_rejects_bad_problems_on_the_host():
+    L = tl.lib()
+    out = (ctypes.c_int64 * 200)()
+    n = ctypes.c_int32()
+    call = lambda arr, count: L.tlin_plan_batched(ctypes.cast(arr, ctypes.c_void_p), count, 0, ctypes.cast(out, ctypes.c_void_p),
+                                                  ctypes.cast(ctypes.pointer(n), ctypes.c_void_p))
+    ok = _problem_array([(2, 300, 100, 1)])
+    assert call(ok, 1) == 0
+    assert call(ok, 0) == tl.ERR_INVALID_ARG
+    assert call(_problem_array([(2, 50, 100, 1)]), 1) == tl.ERR_INVALID_ARG          # window rule with N < W
+    assert call(_problem_array([(0, 300, 100, 0)]), 1) == tl.ERR_INVALID_ARG
+    bad = _problem_array([(2, 300, 100, 0)])
+    bad[0].kv_rows = 200                                                             # allocation smaller than the keys used
+    assert call(bad, 1) == tl.ERR_INVALID_ARG
+    bad = _problem_array([(2, 300, 100, 0)])
+    bad[0].q = 24                                                                    # misaligned
+    assert call(bad, 1) == tl.ERR_INVALID_ARG
+    assert call(_problem_array([(1, 128, 128, 0)] * 25), 25) == tl.ERR_INVALID_ARG    # more than one launch's table
+    assert L.tlin_attn_forward_batched(ctypes.cast(ok, ctypes.c_void_p), 1, 36, None) == tl.ERR_UNSUPPORTED
+    assert L.tlin_attn_forward_batched(None, 1, 64, None) == tl.ERR_INVALID_ARG
+    assert L.tlin_attn_forward_cache(ctypes.c_void_p(16), ctypes.c_void_p(16), ctypes.c_void_p(16), ctypes.c_void_p(16), None,
+                                     1, 1, 100, 101, 8, 64, 0, None) == tl.ERR_INVALID_ARG

@@ -346,3 +346,39 @@ def test_window_slide_cycle_on_the_cache_in_place(B, H, d, hist, W_og, W_oh, ext
     assert (kc[:, :, hist + total:] == -7.0).all() and (vc[:, :, hist + total:] == -7.0).all()
     with pytest.raises(tl.TlinError):
         tl.tlin_attn_forward_cache(q_sum, kc, vc, kc.shape[2] + 1, causal_window=0)      # more rows than the cache has
+
+
+@pytest.mark.parametrize("d,n_problems", [(128, 5), (64, 3), (128, 50)])
+def test_batched_decode_table_every_problem_against_the_oracle(d, n_problems):
+    """A table of short cached steps in one launch (per-layer rows of a cache-hit step, Appendix A): problems of different
+    cache lengths and head counts, some appending the new token, some attending to a finished cache only."""
+    rng = torch.Generator(device="cpu").manual_seed(1000 + d + n_problems)
+    problems, host = [], []
+    for i in range(n_problems):
+        bh = int(torch.randint(1, 7, (1,), generator=rng))
+        pos = int(torch.randint(1, 1400 if i % 3 else 40, (1,), generator=rng))
+        append = i % 2 == 0
+        ncap = pos + 3
+        kc = torch.randn((1, bh, ncap, d), generator=rng).to(torch.bfloat16)
+        vc = torch.randn((1, bh, ncap, d), generator=rng).to(torch.bfloat16)
+        kc[:, :, pos:] = -7.0
+        vc[:, :, pos:] = -7.0
+        qn, kn, vn = (torch.randn((1, bh, 1, d), generator=rng).to(torch.bfloat16) for _ in range(3))
+        out = torch.empty((1, bh, 1, d), dtype=torch.bfloat16, device=DEV)
+        lse = torch.empty((1, bh), dtype=torch.float32, device=DEV)
+        host.append((qn, kn, vn, kc, vc, pos, append))
+        problems.append((qn.to(DEV), kn.to(DEV) if append else None, vn.to(DEV) if append else None, kc.to(DEV), vc.to(DEV), pos, out, lse))
+    tl.tlin_decode_step_batched(problems)
+    torch.cuda.synchronize()
+    assert tl.tlin_get_status() == 0 and tl.tlin_last_launch_count() == -(-n_problems // 48)
+    for i, ((qn, kn, vn, kc, vc, pos, append), pr) in enumerate(zip(host, problems)):
+        out, lse, kc_d, vc_d = pr[6], pr[7], pr[3], pr[4]
+        if append:
+            ref, ref_lse = oracle.decode_step(qn, kn, vn, kc, vc, pos)                     # updates kc, vc in place
+        else:
+            ref, ref_lse = oracle.attn_forward(qn, kc[:, :, :pos].contiguous(), vc[:, :, :pos].contiguous(), 0)
+        parity.check(out.float().cpu().numpy(), lse.cpu().numpy(), ref.reshape(out.shape), ref_lse.reshape(lse.shape), "bf16", f"table problem {i}")
+        assert torch.equal(kc_d.cpu(), kc) and torch.equal(vc_d.cpu(), vc)               # appended row bit-exact, the rest untouched
+    with pytest.raises(tl.TlinError):
+        bad = list(problems[0]); bad[5] = problems[0][3].shape[2]                          # pos beyond the cache
+        tl.tlin_decode_step_batched([tuple(bad)])

@@ -346,9 +346,13 @@ def test_full_size_tensor_core_path_agrees_with_the_cuda_core_path_everywhere(na
     q, k, v = synth.forward_inputs(wl, device=DEV)
     a, la = run_impl(2, tl.tlin_attn_forward, q, k, v, causal_window=1)
     b, lb = run_impl(1, tl.tlin_attn_forward, q, k, v, causal_window=1)
-    # both results are rounded to bf16 (8 significant bits): two last places of the larger value, plus a floor
-    excess = (a.float() - b.float()).abs() - (2.0 ** -6) * torch.maximum(a.float().abs(), b.float().abs())
-    assert float(excess.max()) <= 2e-3
+    # both sides are rounded to bf16, so besides the absolute gate of the oracle comparison two values may sit one last
+    # place (2^-7 relative) apart; the peaked rows of the long configuration reach magnitudes of several units
+    af, bf = a.float(), b.float()
+    excess = (af - bf).abs() - (2.0 ** -7) * torch.maximum(af.abs(), bf.abs())
+    assert float(excess.max()) <= 2e-2
+    assert float((af - bf).abs().mean()) <= 2e-3
+    assert float((af - bf).norm() / bf.norm()) <= 2e-2
     assert float((la - lb).abs().max()) <= 1e-3
 
 
@@ -404,3 +408,64 @@ def test_chunk_scheduled_forward_ragged_prefixes_without_mask():
         parity.check(out[c].float().cpu().numpy(), lse[c].cpu().numpy(), ref, ref_lse, "bf16", f"prefix {n_keys[c]}")
     with pytest.raises(tl.TlinError):
         tl.tlin_attn_forward_prefixes(q, k, v, [100, 333, 1001], causal_window=0)      # beyond the key tensor
+
+
+def _batched_case(d, specs, seed):
+    """specs: (B, H, rows, n_keys, W, causal); k, v hold `rows` rows per head of which the first n_keys are used."""
+    problems, refs = [], []
+    for i, (B, H, rows, n_keys, W, causal) in enumerate(specs):
+        wl = synth.Workload(f"tab{i}", B, H, d, rows, W, seed=seed + i, causal_window=causal)
+        q, k, v = synth.forward_inputs(wl, device=DEV)
+        out_g = Guarded(q.shape, torch.bfloat16, DEV)
+        lse_g = Guarded((B, H, W), torch.float32, DEV)
+        problems.append((q, k, v, out_g.t, lse_g.t, n_keys, causal))
+        refs.append((out_g, lse_g))
+    return problems, refs
+
+
+@pytest.mark.parametrize("d,specs", [
+    (128, [(1, 6, 300, 300, 300, 0), (1, 6, 700, 700, 300, 1), (2, 2, 1000, 100, 40, 0), (2, 2, 1000, 333, 40, 0),
+           (2, 2, 1000, 1000, 40, 0), (1, 3, 520, 520, 520, 1), (1, 1, 77, 77, 1, 1)]),
+    (64, [(2, 5, 1111, 1111, 200, 1), (1, 2, 129, 100, 600, 0), (3, 1, 2049, 2049, 129, 1)]),
+    (128, [(1, 1, 64 + 8 * i, 64 + 8 * i, 30 + i, i % 2) for i in range(27)]),      # more than one launch's table
+])
+def test_batched_forward_every_problem_against_the_oracle(d, specs):
+    """A table of independent problems of different shapes and masks as one launch (inner layers of a block, key
+    prefixes of one sequence read in place): each problem equals the oracle, guard regions around every output stay
+    untouched, and a problem that a call of its own would also run unsplit comes out bit-identical."""
+    if not TC_AVAILABLE:
+        pytest.skip("tensor path not built")
+    problems, guards = _batched_case(d, specs, seed=900 + d)
+    tl.tlin_attn_forward_batched(problems)
+    torch.cuda.synchronize()
+    assert tl.tlin_get_status() == 0
+    assert tl.tlin_last_launch_count() == -(-len(specs) // 24)
+    for i, ((q, k, v, out, lse, n_keys, causal), (og, lg)) in enumerate(zip(problems, guards)):
+        og.check(f"problem {i} out")
+        lg.check(f"problem {i} lse")
+        ks, vs = k[:, :, :n_keys].contiguous(), v[:, :, :n_keys].contiguous()
+        ref, ref_lse = oracle.attn_forward(q.cpu(), ks.cpu(), vs.cpu(), causal)
+        parity.check(out.float().cpu().numpy(), lse.cpu().numpy(), ref, ref_lse, "bf16", f"batched problem {i} {specs[i]}")
+        B, H, W = q.shape[0], q.shape[1], q.shape[2]
+        if tl.tlin_plan_forward(B, H, n_keys, W, d, causal).schedule == 1:
+            single, single_lse = run_impl(2, tl.tlin_attn_forward, q, ks, vs, causal_window=causal)
+            assert torch.equal(single, out) and torch.equal(single_lse, lse), f"problem {i}: differs from its own call"
+
+
+def test_batched_forward_runs_a_sliding_window_pass_with_arbitrary_prefixes_in_one_launch():
+    # Section 5.1: every chunk of W_og tokens attends to everything up to its own end; here as one table over one k, v
+    if not TC_AVAILABLE:
+        pytest.skip("tensor path not built")
+    C, B, H, W, d = 6, 2, 3, 160, 128
+    L = C * W
+    wl = synth.Workload("chunks1", B, H, d, L, L, seed=47, causal_window=1)
+    q_all, k, v = synth.forward_inputs(wl, device=DEV)
+    q = q_all.view(B, H, C, W, d).permute(2, 0, 1, 3, 4).contiguous()
+    out = torch.empty_like(q)
+    lse = torch.empty((C, B, H, W), dtype=torch.float32, device=DEV)
+    tl.tlin_attn_forward_batched([(q[c], k, v, out[c], lse[c], (c + 1) * W, 1) for c in range(C)])
+    torch.cuda.synchronize()
+    assert tl.tlin_get_status() == 0 and tl.tlin_last_launch_count() == 1
+    ref, ref_lse = oracle.attn_forward(q_all.cpu(), k.cpu(), v.cpu(), 1)         # plain causal attention over the whole sequence
+    got = out.permute(1, 2, 0, 3, 4).reshape(B, H, L, d)
+    parity.check(got.float().cpu().numpy(), lse.permute(1, 2, 0, 3).reshape(B, H, L).cpu().numpy(), ref, ref_lse, "bf16", "chunks in one launch")
