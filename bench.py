@@ -200,8 +200,8 @@ L2_BYTES = 126e6
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from one-pass ncu captures of these
 # very workloads.  To be set to None whenever the kernel changes.
-FWD_TRAFFIC = {"cfg4_vlong": (2168.65e6 + 20.05e6, "ncu, full workload, fwd_tc_kernel<128>"),
-               "cfg3_long": (544.75e6 + 10.74e6, "ncu, full workload, fwd_tc_kernel<128>")}
+FWD_TRAFFIC = {"cfg4_vlong": (2191.82e6 + 20.53e6, "ncu, full workload, fwd_tc_kernel<128, 0>"),
+               "cfg3_long": (544.79e6 + 10.41e6, "ncu, full workload, fwd_tc_kernel<128, 0>")}
 # decode: captured on a smaller cache (B8 H32, 4096 rows: 537.35 MB read + 3.9 MB written for 537.3 MB of cache) and
 # scaled by the cached rows of the timed steps; the kernel streams every cached byte once at any size
 DECODE_TRAFFIC_RATIO = (537.35 + 3.9) / 537.3
@@ -546,8 +546,30 @@ def run_batched(args, rank, world, device, peaks):
     roof = dict(bound="tensor", achieved=tflops, peak=peaks["bf16_tflops"], unit="TFLOP/s", frac=tflops / peaks["bf16_tflops"],
                 traffic=None, algorithmic_bytes=sum(fwd_bytes(wl) for wl in wls), peak_source=peaks["source"] + " (burst)",
                 kernel="forward, two problems in one launch", roofline_ms=flop / (peaks["bf16_tflops"] * 1e12) * 1e3)
+    # The same two layers for four requests of 8 heads each (eight problems): alone, a problem of 32 units leaves most of
+    # the 148 SMs idle, which is where one launch for the table pays.
+    few = []
+    for r in range(4):
+        for wl in wls:
+            w8 = synth.Workload(f"{wl.name}_h8_r{r}", 1, 8, wl.d, wl.N, wl.W, seed=wl.seed + 100 + r, causal_window=wl.causal_window)
+            q, k, v = synth.forward_inputs(w8, device=device)
+            few.append((w8, q, k, v, torch.empty_like(q), torch.empty((1, 8, w8.W), dtype=torch.float32, device=device)))
+    table8 = [(q, k, v, out, lse, None, wl.causal_window) for (wl, q, k, v, out, lse) in few]
+
+    def step_batched8(_):
+        tl.tlin_attn_forward_batched(table8)
+
+    def step_separate8(_):
+        for (wl, q, k, v, out, lse) in few:
+            tl.tlin_attn_forward(q, k, v, out, lse, wl.causal_window)
+
+    ms_b8, _ = time_steps(step_batched8, args.steps, args.warmup, world, device, None, flush)
+    ms_s8, _ = time_steps(step_separate8, args.steps, args.warmup, world, device, None, flush)
+    ms_b8 /= args.steps
+    ms_s8 /= args.steps
     return dict(workload="inner_self + inner_gen as one table", ms_per_step=ms_b, tflops=tflops, roofline=roof, e2e=None, clocks=clocks,
                 separate_calls_ms_per_step=ms_s, batched_over_separate=ms_b / ms_s,
+                eight_problems_of_8_heads=dict(batched_ms=ms_b8, separate_calls_ms=ms_s8, batched_over_separate=ms_b8 / ms_s8),
                 l2="a %.0f MB buffer is overwritten before every timed step (L2 flush), steps timed one by one" % (flush.numel() / 1e6),
                 gpu_launches=int(sum(launches["batched"][args.warmup:args.warmup + args.steps])),
                 launches_per_step=launches["batched"][-1], separate_launches_per_step=launches["separate"][-1])
@@ -680,7 +702,7 @@ def compact_leg(leg):
     c = leg.get("clocks") or {}
     out = {k: leg[k] for k in ("workload", "shape", "ms_per_step", "tflops", "gb_per_s", "tokens_per_s", "decode_tokens_per_s", "steps",
                                "gpu_launches", "launches_per_step", "separate_calls_ms_per_step", "batched_over_separate",
-                               "separate_launches_per_step") if k in leg}
+                               "separate_launches_per_step", "eight_problems_of_8_heads") if k in leg}
     out["roofline"] = roof
     out["clocks"] = {"sm_mhz": c.get("sm_mhz"), "sm_max_mhz": c.get("sm_max_mhz"), "reasons": c.get("reasons", [])}
     if leg.get("e2e"):
@@ -804,6 +826,8 @@ def main():
             "also": also,
             "tflops": main_res.get("tflops"),
             "gpu_launches": main_res["gpu_launches"], "launches_per_step": main_res["launches_per_step"],
+            **{k: main_res[k] for k in ("separate_calls_ms_per_step", "batched_over_separate", "separate_launches_per_step",
+                                        "eight_problems_of_8_heads") if k in main_res},
             "cpu_baseline": main_res.get("cpu_baseline"), "e2e": main_res["e2e"], "clocks": main_res["clocks"],
             "roofline": main_res["roofline"], "targets": targets,
         }
