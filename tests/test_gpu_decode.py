@@ -5,6 +5,7 @@ import torch
 
 import oracle
 import parity
+from guards import Guarded
 from paper_2508_20407_b200 import binding as tl
 from paper_2508_20407_b200 import synth
 
@@ -24,15 +25,24 @@ def test_decode_steps_elementwise_and_cache_bookkeeping(B, H, d, N0, T):
     kc[:, :, N0:N0 + T] = -7.0
     vc[:, :, N0:N0 + T] = -7.0
     kc_h, vc_h = kc.cpu(), vc.cpu()
+    # out, lse and the split workspace sit between filled guard regions, in buffers of exactly the documented sizes
+    out_g, lse_g = Guarded((B, H, 1, d), torch.bfloat16, DEV), Guarded((B, H), torch.float32, DEV)
+    ws_g = Guarded((tl.workspace_bytes_decode(B, H, kc.shape[2], d),), torch.uint8, DEV)
+    saved = tl._workspace_tensor
+    tl.set_workspace(ws_g.t)
     for t in range(T):
-        out, lse = tl.tlin_decode_step(qn[t], kn[t], vn[t], kc, vc, N0 + t)
+        out, lse = tl.tlin_decode_step(qn[t], kn[t], vn[t], kc, vc, N0 + t, out_g.t, lse_g.t)
         torch.cuda.synchronize()
         assert tl.tlin_get_status() == 0 and tl.tlin_last_launch_count() >= 1
+        assert tl._workspace_tensor is ws_g.t
+        for g, name in ((out_g, "out"), (lse_g, "lse"), (ws_g, "workspace")):
+            g.check(f"decode step {t} {name}")
         ref, ref_lse = oracle.decode_step(qn[t].cpu(), kn[t].cpu(), vn[t].cpu(), kc_h, vc_h, N0 + t)
         parity.check(out.float().cpu().numpy(), lse.cpu().numpy(), ref, ref_lse, "bf16", f"decode step {t}")
         # bit-exact bookkeeping: appended rows equal the new tokens, everything above is untouched
         assert torch.equal(kc.cpu(), kc_h) and torch.equal(vc.cpu(), vc_h)
         assert (kc[:, :, N0 + t + 1:] == -7.0).all() and (vc[:, :, N0 + t + 1:] == -7.0).all()
+    tl.set_workspace(saved)
 
 
 def test_decode_equals_rows_of_the_forward_oracle():
