@@ -567,7 +567,21 @@ def run_batched(args, rank, world, device, peaks):
     ms_s8, _ = time_steps(step_separate8, args.steps, args.warmup, world, device, None, flush)
     ms_b8 /= args.steps
     ms_s8 /= args.steps
+    # Cache-hit analogue (Appendix A: per generation layer one row against the W_oh cached summary tokens and the window so
+    # far): three layers' rows, B8 H32, caches of 1024 + 64 rows with the new token appended, as one table against three
+    # tlin_decode_step calls (two kernels each).
+    rows = []
+    for li in range(3):
+        dwl = synth.Workload(f"layer{li}_hit", 8, 32, 128, 1024 + 63, 1, seed=40 + li, decode=True)
+        (kc, vc), (qn, kn, vn) = synth.decode_inputs(dwl, device=device)
+        rows.append((qn[0], kn[0], vn[0], kc, vc, dwl.N, torch.empty_like(qn[0]), torch.empty((8, 32), dtype=torch.float32, device=device)))
+    tl.ensure_workspace(tl.workspace_bytes_decode(8, 32, 1024 + 64, 128), device)
+    ms_dt, _ = time_steps(lambda _i: tl.tlin_decode_step_batched(rows), args.steps, args.warmup, world, device, None, flush)
+    ms_ds, _ = time_steps(lambda _i: [tl.tlin_decode_step(*r[:6], r[6], r[7]) for r in rows], args.steps, args.warmup, world, device, None, flush)
+    decode_table = dict(batched_ms=ms_dt / args.steps, separate_calls_ms=ms_ds / args.steps, batched_over_separate=ms_dt / ms_ds,
+                        what="three problems of B8 H32 d128, 1087 cached rows + the appended row: one launch against six")
     return dict(workload="inner_self + inner_gen as one table", ms_per_step=ms_b, tflops=tflops, roofline=roof, e2e=None, clocks=clocks,
+                decode_table=decode_table,
                 separate_calls_ms_per_step=ms_s, batched_over_separate=ms_b / ms_s,
                 eight_problems_of_8_heads=dict(batched_ms=ms_b8, separate_calls_ms=ms_s8, batched_over_separate=ms_b8 / ms_s8),
                 l2="a %.0f MB buffer is overwritten before every timed step (L2 flush), steps timed one by one" % (flush.numel() / 1e6),
@@ -702,7 +716,7 @@ def compact_leg(leg):
     c = leg.get("clocks") or {}
     out = {k: leg[k] for k in ("workload", "shape", "ms_per_step", "tflops", "gb_per_s", "tokens_per_s", "decode_tokens_per_s", "steps",
                                "gpu_launches", "launches_per_step", "separate_calls_ms_per_step", "batched_over_separate",
-                               "separate_launches_per_step", "eight_problems_of_8_heads") if k in leg}
+                               "separate_launches_per_step", "eight_problems_of_8_heads", "decode_table") if k in leg}
     out["roofline"] = roof
     out["clocks"] = {"sm_mhz": c.get("sm_mhz"), "sm_max_mhz": c.get("sm_max_mhz"), "reasons": c.get("reasons", [])}
     if leg.get("e2e"):
@@ -827,7 +841,7 @@ def main():
             "tflops": main_res.get("tflops"),
             "gpu_launches": main_res["gpu_launches"], "launches_per_step": main_res["launches_per_step"],
             **{k: main_res[k] for k in ("separate_calls_ms_per_step", "batched_over_separate", "separate_launches_per_step",
-                                        "eight_problems_of_8_heads") if k in main_res},
+                                        "eight_problems_of_8_heads", "decode_table") if k in main_res},
             "cpu_baseline": main_res.get("cpu_baseline"), "e2e": main_res["e2e"], "clocks": main_res["clocks"],
             "roofline": main_res["roofline"], "targets": targets,
         }
