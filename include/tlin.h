@@ -69,8 +69,10 @@ int tlin_attn_forward_f32(const float* q, const float* k, const float* v, float*
  *   q   [C,B,H,W,d]   the W queries of each chunk        k,v [B,H,L,d]   shared; n_keys[c] <= L (HOST array of C ints)
  *   out [C,B,H,W,d]   lse [C,B,H,W] (may be NULL)
  * causal_window as in tlin_attn_forward, applied per chunk with N = n_keys[c] (with n_keys[c] = (c+1)*W and
- * causal_window = 1 chunk c is the c-th window of the training pass).  The chunks are issued as C launches of the forward
- * kernel on `stream`, each with its own plan, reading k and v in place (row stride L); nothing is copied.
+ * causal_window = 1 chunk c is the c-th window of the training pass).  k and v are read in place (row stride L); nothing is
+ * copied.  When the chunks hold enough whole (chunk, b*h, 256-row query tile) problems to fill the SMs (at least two per SM,
+ * C <= 24, d in {64,128}) they are issued as ONE launch (the table form of tlin_attn_forward_batched); otherwise as C
+ * launches of the forward kernel on `stream`, each with its own plan and free to split its key range.
  * bf16, head sizes as for tlin_attn_forward.  Workspace: tlin_workspace_bytes_forward_prefixes (the largest of the
  * chunks' needs).  tlin_attn_forward_batched runs such a list, and any other, as one launch. */
 int tlin_attn_forward_prefixes(const void* q, const void* k, const void* v, void* out, float* lse,

@@ -133,6 +133,21 @@ extern "C" int tlin_attn_forward_prefixes(const void* q, const void* k, const vo
     for (int c = 0; c < C; ++c)      // every chunk is checked before the first one is launched
         if (n_keys[c] <= 0 || n_keys[c] > L || (causal_window && n_keys[c] < W)) return TLIN_ERR_INVALID_ARG;
     const size_t q_chunk = (size_t)B * H * W * d * 2, lse_chunk = (size_t)B * H * W;
+    // Enough whole (chunk, b*h, query tile) problems to fill the SMs: all chunks as one table launch (keys never split, so no
+    // workspace).  Fewer: one launch per chunk, each free to split its key range.
+    if ((d == 64 || d == 128) && forward_impl() != 1 && C <= kMaxBatch && (long long)B * H <= 0x7fffffffLL) {
+        int sms = 0;
+        if (device_info(&sms) == TLIN_OK && (long long)C * B * H * ((W + 255) / 256) >= 2LL * sms) {
+            tlin_problem tbl[kMaxBatch];
+            for (int c = 0; c < C; ++c) {
+                tbl[c].q = (const char*)q + c * q_chunk; tbl[c].k = k; tbl[c].v = v;
+                tbl[c].out = (char*)out + c * q_chunk; tbl[c].lse = lse ? lse + c * lse_chunk : nullptr;
+                tbl[c].BH = B * H; tbl[c].n_keys = n_keys[c]; tbl[c].kv_rows = n_keys[c] == L ? 0 : L;
+                tbl[c].n_queries = W; tbl[c].causal_window = causal_window; tbl[c].reserved = 0;
+            }
+            return tlin_attn_forward_batched(tbl, C, d, stream);
+        }
+    }
     int total = 0;                 // a chunked call counts the launches of all its chunks
     for (int c = 0; c < C; ++c) {
         const int rc = forward_common((const char*)q + c * q_chunk, k, v, (char*)out + c * q_chunk, lse ? lse + c * lse_chunk : nullptr,

@@ -469,3 +469,28 @@ def test_batched_forward_runs_a_sliding_window_pass_with_arbitrary_prefixes_in_o
     ref, ref_lse = oracle.attn_forward(q_all.cpu(), k.cpu(), v.cpu(), 1)         # plain causal attention over the whole sequence
     got = out.permute(1, 2, 0, 3, 4).reshape(B, H, L, d)
     parity.check(got.float().cpu().numpy(), lse.permute(1, 2, 0, 3).reshape(B, H, L).cpu().numpy(), ref, ref_lse, "bf16", "chunks in one launch")
+
+
+def test_chunk_scheduled_forward_with_many_units_is_one_launch():
+    # enough (chunk, b*h, query tile) problems to fill the SMs: the prefixes entry point issues all chunks as one table launch
+    if not TC_AVAILABLE:
+        pytest.skip("tensor path not built")
+    C, B, H, W, d = 4, 2, 40, 200, 64
+    L = C * W + 37                                   # the last chunk does not reach the end of k, v
+    wl = synth.Workload("chunks_table", B, H, d, L, C * W, seed=49, causal_window=1)
+    q_all, k, v = synth.forward_inputs(wl, device=DEV)
+    q = q_all.view(B, H, C, W, d).permute(2, 0, 1, 3, 4).contiguous()
+    n_keys = [(c + 1) * W for c in range(C)]
+    out, lse = tl.tlin_attn_forward_prefixes(q, k, v, n_keys, causal_window=1)
+    torch.cuda.synchronize()
+    assert tl.tlin_get_status() == 0 and tl.tlin_last_launch_count() == 1
+    for c in (0, C - 1):
+        for (b, h) in ((0, 0), (B - 1, H - 1)):
+            sl = lambda t: t[b:b + 1, h:h + 1].contiguous().cpu()
+            ref, ref_lse = oracle.attn_forward(sl(q[c]), sl(k[:, :, :n_keys[c]]), sl(v[:, :, :n_keys[c]]), 1)
+            parity.check(sl(out[c]).float().numpy(), sl(lse[c]).numpy(), ref, ref_lse, "bf16", f"chunk {c} head {(b, h)}")
+    # every chunk equals its own call bit for bit when that call does not split the keys either
+    for c in range(C):
+        if tl.tlin_plan_forward(B, H, n_keys[c], W, d, 1).schedule == 1:
+            o1, l1 = run_impl(2, tl.tlin_attn_forward, q[c], k[:, :, :n_keys[c]].contiguous(), v[:, :, :n_keys[c]].contiguous(), causal_window=1)
+            assert torch.equal(o1, out[c]) and torch.equal(l1, lse[c])
