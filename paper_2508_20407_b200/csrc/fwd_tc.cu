@@ -313,17 +313,28 @@ fwd_tc_kernel(const __grid_constant__ KernelMaps<kBatched> maps, const __grid_co
                 if (cnt == 1) commit_elected(q_empty);      // the segment's last use of Q is issued: its successor may load
                 ++it;
                 for (int j = 0; j < cnt && ok; ++j) {
-                    const uint32_t v_slot = it % C::kSlots;
-                    ok = __all_sync(0xffffffffu, mbar_wait(&kv_full[v_slot], (it / C::kSlots) & 1, abort_p));
-                    if (!ok) break;
+                    const uint32_t v_slot = it % C::kSlots, v_par = (it / C::kSlots) & 1;
                     ++it;
                     const bool have_next = j + 1 < cnt;
-                    uint32_t nk_slot = 0;
+                    uint32_t nk_slot = 0, nk_par = 0;
                     if (have_next) {
                         nk_slot = it % C::kSlots;
-                        ok = __all_sync(0xffffffffu, mbar_wait(&kv_full[nk_slot], (it / C::kSlots) & 1, abort_p));
-                        if (!ok) break;
+                        nk_par = (it / C::kSlots) & 1;
                         ++it;
+                    }
+                    // both tiles are usually there already: ask both barriers at once (the two answers travel together), and
+                    // wait one after the other only if one is missing
+                    {
+                        const bool v_there = mbar_try_wait(&kv_full[v_slot], v_par);
+                        const bool k_there = have_next ? mbar_try_wait(&kv_full[nk_slot], nk_par) : true;
+                        if (!__all_sync(0xffffffffu, v_there && k_there)) {
+                            ok = __all_sync(0xffffffffu, mbar_wait(&kv_full[v_slot], v_par, abort_p));
+                            if (!ok) break;
+                            if (have_next) {
+                                ok = __all_sync(0xffffffffu, mbar_wait(&kv_full[nk_slot], nk_par, abort_p));
+                                if (!ok) break;
+                            }
+                        }
                     }
                     tc_fence_after();
                     for (int i = 0; i < 2 && ok; ++i) {
