@@ -715,7 +715,9 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const int row = row0 + i * kQTile + r;
             const int a0 = tiles_allowed(p, row0, 0), a1 = tiles_allowed(p, row0, 1);
             const int c0 = seg_count(s, a0), c1 = seg_count(s, a1);
-            if ((c0 > c1 ? c0 : c1) == 0) continue;           // the MMA warp skips this segment too
+            // No tile of the segment is visible to either Q tile: the MMA warp and the producer skip it and it takes no
+            // barrier phase, but its partial slot is still read by the reduce kernel and has to hold zeros.
+            const bool skipped = (c0 > c1 ? c0 : c1) == 0;
             const int allowed_i = i == 0 ? a0 : a1, cnt_i = i == 0 ? c0 : c1;
             const long long lim_row_ll = p.causal ? (long long)p.N - p.W + row + 1 : (long long)p.N;
             const int lim_row = (int)(lim_row_ll < p.N ? lim_row_ll : p.N);
@@ -768,7 +770,8 @@ bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 ++n;
             }
             if (!ok) break;
-            const uint32_t my_seg = seg_idx++;
+            const uint32_t my_seg = seg_idx;
+            if (!skipped) ++seg_idx;
             if (allowed_i == 0) continue;                      // this Q tile does not exist
             // ---------------------------------------------------------------- dQ of the segment
             if (cnt_i > 0) {
