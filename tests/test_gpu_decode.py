@@ -104,6 +104,30 @@ def test_cfg5_full_size_sampled_heads_and_steps():
         assert torch.equal(kc[b, h].cpu(), host[(b, h)][0][0, 0]) and torch.equal(vc[b, h].cpu(), host[(b, h)][1][0, 0])
 
 
+def _every_head_agrees(out, lse, ref_out, ref_lse, what, lse_gate=1e-3):
+    """Two kernel families on the same inputs, both storing bf16: per (b,h) relative L2 <= 1e-2 (rounding of 128 bf16
+    values gives about 2e-3) and |lse difference| <= lse_gate."""
+    a, b = out.float().flatten(2), ref_out.float().flatten(2)                 # [B,H,d]
+    assert torch.isfinite(a).all() and torch.isfinite(lse).all(), what
+    rel = ((a - b).pow(2).sum(-1) / b.pow(2).sum(-1).clamp_min(1e-30)).sqrt()
+    assert float(rel.max()) <= 1e-2, f"{what}: worst (b,h) rel L2 {float(rel.max()):.3e} at {int(rel.argmax())}"
+    dl = (lse.flatten() - ref_lse.flatten()).abs()
+    assert float(dl.max()) <= lse_gate, f"{what}: lse differs by {float(dl.max()):.3e} at {int(dl.argmax())}"
+
+
+def test_cfg5_every_head_against_the_forward_kernels_on_the_cache():
+    """The oracle recomputes three heads of cfg5; here every (b,h) of a step is compared with the forward entry point run
+    on the same cache (one query row, all cached rows, no mask): a different kernel family, different split of the keys."""
+    wl = synth.WORKLOADS["cfg5_decode"]
+    (kc, vc), (qn, kn, vn) = synth.decode_inputs(wl, device=DEV, steps=3)
+    for t in range(3):
+        out, lse = tl.tlin_decode_step(qn[t], kn[t], vn[t], kc, vc, wl.N + t)
+        ref_out, ref_lse = tl.tlin_attn_forward_cache(qn[t], kc, vc, wl.N + t + 1, causal_window=0)
+        torch.cuda.synchronize()
+        assert tl.tlin_get_status() == 0
+        _every_head_agrees(out, lse, ref_out, ref_lse, f"cfg5 step {t}")
+
+
 def test_ragged_decode_one_length_per_sequence():
     """Sequences of one batch at different cache lengths (positions read from device memory): every sequence
     equals the oracle's step at its own length; appended rows are bit-exact; nothing else in the caches moves."""
@@ -289,6 +313,35 @@ def test_fp8_decode_at_the_cfg5_size_on_sampled_heads():
             parity.check(sl(out).float().numpy(), sl(lse).numpy(), ref, ref_lse, "bf16", f"8-bit cfg5 step {t} head {(b, h)}")
     for (b, h) in heads:
         assert torch.equal(kc[b, h].cpu(), host[(b, h)][0][0, 0]) and torch.equal(vc[b, h].cpu(), host[(b, h)][1][0, 0])
+
+
+def test_fp8_decode_at_the_cfg5_size_every_head_against_the_bf16_kernels():
+    """Every (b,h) of an 8-bit step against the forward entry point on the same cache after torch has turned the codes into
+    bf16 values (code * scale, rounded to bf16).  That rounding moves every key by up to 2^-9 of itself, and with keys
+    as large as these (codes up to 448, scales up to 0.012) the scores of the few keys that carry a row move by a few 1e-3:
+    the lse gate of this comparison is 1e-2, the output gate the usual one."""
+    wl = synth.WORKLOADS["cfg5_decode"]
+    B, H, d, N = wl.B, wl.H, wl.d, wl.N
+    g = torch.Generator(device=DEV).manual_seed(78)
+    def codes():
+        c = torch.randint(0, 254, (B, H, N + 8, d), generator=g, device=DEV, dtype=torch.int16)
+        return (c + (c >= 127).to(torch.int16)).to(torch.uint8).contiguous()       # every finite code, no NaN code
+    kc, vc = codes(), codes()
+    ks = (torch.rand(B, H, generator=g, device=DEV) * 0.01 + 0.002).float()
+    vs = (torch.rand(B, H, generator=g, device=DEV) * 0.01 + 0.002).float()
+    q, kn, vn = (torch.randn(B, H, 1, d, generator=g, device=DEV).to(torch.bfloat16) for _ in range(3))
+    out, lse = tl.tlin_decode_step_fp8(q, kn, vn, kc, vc, ks, vs, N)
+    torch.cuda.synchronize()
+    assert tl.tlin_get_status() == 0
+    def values(c, scale):       # [B,H,N+1,d] bf16, a (b,h) at a time to bound the fp32 temporaries
+        v = torch.empty((B, H, N + 1, d), dtype=torch.bfloat16, device=DEV)
+        for b in range(B):
+            v[b] = (c[b, :, :N + 1].view(torch.float8_e4m3fn).float() * scale[b].view(H, 1, 1)).to(torch.bfloat16)
+        return v
+    kb, vb = values(kc, ks), values(vc, vs)
+    ref_out, ref_lse = tl.tlin_attn_forward_cache(q, kb, vb, N + 1, causal_window=0)
+    torch.cuda.synchronize()
+    _every_head_agrees(out, lse, ref_out, ref_lse, "8-bit cfg5 step", lse_gate=1e-2)
 
 
 @pytest.mark.parametrize("B,H,d,hist,W_og,W_oh,extra", [(2, 3, 128, 300, 64, 48, 5), (1, 2, 64, 1000, 130, 40, 3), (1, 2, 72, 90, 20, 8, 2)])
