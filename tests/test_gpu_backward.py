@@ -96,6 +96,14 @@ def test_backward_elementwise(B, H, N, W, d, causal, impl):
     run_case(B, H, N, W, d, causal, seed=300 + N + W, impl=impl, guarded=True)
 
 
+@pytest.mark.parametrize("seed", [21, 22, 23])
+def test_backward_random_shapes_against_the_oracle(seed):
+    # seeded shapes nobody picked by hand (the forward tests' generator, smaller: the fp64 chain rule costs more)
+    from test_gpu_forward import random_shapes
+    for (B, H, N, W, d, causal) in random_shapes(seed, 6, budget=1.5e9):
+        run_case(B, H, N, W, d, causal, seed=seed * 1000 + N + W, impl=0, guarded=True)
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 def test_backward_cfg1_tiny(impl):
     wl = synth.WORKLOADS["cfg1_tiny"]

@@ -119,6 +119,45 @@ def partials_per_head(plan):
     return counts
 
 
+def random_shapes(seed, count, budget=4e9):
+    """Seeded shapes that no one picked by hand: tile edges +-1, window rule on and off, few and many (b,h), key ranges that
+    are split between CTAs and ones that are not; B*H*W*N*d bounded so that the oracle stays within a second per shape."""
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < count:
+        d = int(rng.choice([64, 128]))
+        causal = int(rng.integers(0, 2))
+        kind = int(rng.integers(0, 4))
+        if kind == 0:       # long keys, few queries
+            W, N, BH = int(rng.integers(1, 700)), int(rng.integers(700, 9000)), int(rng.integers(1, 5))
+        elif kind == 1:     # square-ish
+            W = int(rng.integers(1, 1400)); N, BH = W + int(rng.integers(0, 400)), int(rng.integers(1, 7))
+        elif kind == 2:     # tile edges
+            W = max(1, 128 * int(rng.integers(1, 9)) + int(rng.integers(-1, 2)))
+            N, BH = max(1, 128 * int(rng.integers(1, 30)) + int(rng.integers(-1, 2))), int(rng.integers(1, 9))
+        else:               # many queries, few keys
+            W, N, BH = int(rng.integers(300, 3000)), int(rng.integers(1, 700)), int(rng.integers(1, 6))
+        if causal and N < W:
+            N = W
+        while BH > 1 and BH * W * N * d > budget:
+            BH -= 1
+        if BH * W * N * d > budget:
+            continue
+        B = 2 if BH % 2 == 0 and rng.integers(0, 2) else 1
+        out.append((B, BH // B, N, W, d, causal))
+    return out
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13, 14])
+def test_forward_random_shapes_against_the_oracle(seed):
+    if not TC_AVAILABLE:
+        pytest.skip("tensor path not built")
+    for (B, H, N, W, d, causal) in random_shapes(seed, 10):
+        wl = synth.Workload(f"random B{B} H{H} N{N} W{W} d{d} causal{causal}", B, H, d, N, W, seed=seed * 1000 + N + W,
+                            causal_window=causal)
+        guarded_compare(wl, 2)
+
+
 def test_awkward_shapes_reach_both_branches_of_the_split_merge():
     # the merge kernel combines up to 8 partial results per row from registers and more than 8 in a loop: the shapes
     # above must keep exercising both, whatever the planner turns into
