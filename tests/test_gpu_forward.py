@@ -158,6 +158,22 @@ def test_forward_random_shapes_against_the_oracle(seed):
         guarded_compare(wl, 2)
 
 
+@pytest.mark.parametrize("seed", [15, 16])
+def test_forward_random_shapes_cuda_core_kernels_and_fp32(seed):
+    # the same generator through the kernels that serve every other head size, in bf16 and in fp32 (the paper's d = 36 included)
+    rng = np.random.default_rng(seed)
+    for (B, H, N, W, d, causal) in random_shapes(seed, 8, budget=1e9):
+        d16 = int(rng.choice([8, 40, 64, 96, 128, 200, 256]))
+        d32 = int(rng.choice([4, 36, 64, 100, 128, 256]))
+        N, W = min(N, 3000), min(W, 1000)
+        if causal and N < W:
+            N = W
+        guarded_compare(synth.Workload(f"random B{B} H{H} N{N} W{W} d{d16} causal{causal}", B, H, d16, N, W, seed=seed * 1000 + N,
+                                       causal_window=causal), 1)
+        full_compare(synth.Workload(f"random f32 B{B} H{H} N{N} W{W} d{d32} causal{causal}", B, H, d32, N, W, seed=seed * 1000 + W,
+                                    causal_window=causal), 0, kind="f32")
+
+
 def test_awkward_shapes_reach_both_branches_of_the_split_merge():
     # the merge kernel combines up to 8 partial results per row from registers and more than 8 in a loop: the shapes
     # above must keep exercising both, whatever the planner turns into
