@@ -87,6 +87,7 @@ SIGNATURES = {
     "tlin_status_string": (ctypes.c_char_p, [_i]),
     "tlin_version": (ctypes.c_char_p, []),
     "tlin_set_forward_impl": (_i, [_i]),
+    "tlin_set_backward_impl": (_i, [_i]),
     "tlin_last_launch_count": (_i, []),
 }
 
@@ -493,6 +494,12 @@ def tlin_debug_wait_expires(limit_cycles: int, waited=None, stream=None) -> None
 
 def tlin_set_forward_impl(impl: int) -> int:
     return int(lib().tlin_set_forward_impl(impl))
+
+
+def tlin_set_backward_impl(impl: int) -> int:
+    """0: the library chooses, 1: two kernels (dK/dV, then dQ; bitwise repeatable), 2: one kernel (d = 128; dQ summed by
+    reductions in L2, repeatable up to the order of fp32 additions).  Returns the previous setting."""
+    return int(lib().tlin_set_backward_impl(int(impl)))
 
 
 def tlin_last_launch_count() -> int:

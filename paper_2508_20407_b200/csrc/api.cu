@@ -12,6 +12,7 @@ constexpr int kMaxDevices = 64;
 std::mutex g_mu;
 Workspace g_ws[kMaxDevices] = {};          // one registered workspace per device (indexed by the current device)
 std::atomic<int> g_impl{0};
+std::atomic<int> g_bwd_impl{0};
 thread_local int t_launches = 0;
 __device__ int g_status_word = 0;
 
@@ -81,6 +82,7 @@ int* status_word() {
 }
 void count_launch(int n) { t_launches += n; }
 int forward_impl() { return g_impl.load(); }
+int backward_impl() { return g_bwd_impl.load(); }
 
 }  // namespace tlin
 
@@ -250,6 +252,10 @@ static int backward_common(const void* q, const void* k, const void* v, const vo
         if (!w.ptr || w.bytes < bwd_workspace_bytes(B, H, W, d)) return TLIN_ERR_WORKSPACE;
         return launch_bwd_simt(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, d, causal_window, is_f32, (float*)w.ptr, sms, st);
     }
+    if (d == 128 && backward_impl() == 2) {
+        if (!w.ptr || w.bytes < bwd_fused_workspace_bytes(B, H, W, d)) return TLIN_ERR_WORKSPACE;
+        return launch_bwd_fused(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, d, causal_window, (float*)w.ptr, sms, st);
+    }
     tlin_fwd_plan plan;
     rc = tlin_plan_forward(B, H, N, W, d, causal_window, 0, sms, &plan);   // the dQ kernel follows the forward's plan
     if (rc != TLIN_OK) return rc;
@@ -278,6 +284,10 @@ extern "C" size_t tlin_workspace_bytes_backward(int B, int H, int N, int W, int 
         if (causal && N < W) continue;
         if (tlin_plan_forward(B, H, N, W, d, causal, 0, 0, &plan) != TLIN_OK || !plan.tensor_path) continue;
         const size_t t = bwd_tc_workspace_bytes(B, H, W, d, plan);
+        if (t > need) need = t;
+    }
+    if (d == 128) {
+        const size_t t = bwd_fused_workspace_bytes(B, H, W, d);
         if (t > need) need = t;
     }
     return need;
@@ -460,6 +470,11 @@ extern "C" const char* tlin_version(void) { return "libtlin 0.1 (sm_100a)"; }
 extern "C" int tlin_set_forward_impl(int impl) {
     if (impl < 0 || impl > 2) return TLIN_ERR_INVALID_ARG;
     return g_impl.exchange(impl);
+}
+
+extern "C" int tlin_set_backward_impl(int impl) {
+    if (impl < 0 || impl > 2) return TLIN_ERR_INVALID_ARG;
+    return g_bwd_impl.exchange(impl);
 }
 
 extern "C" int tlin_last_launch_count(void) { return t_launches; }

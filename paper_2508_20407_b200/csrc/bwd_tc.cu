@@ -5,7 +5,7 @@
 //   p = exp(q k^T / sqrt(d) - lse)    dp = dout v^T    ds = p * (dp - delta) / sqrt(d),  delta_i = dout_i . out_i
 //   dv = p^T dout      dk = ds^T q      dq = ds k
 //
-// Two kernels, neither with atomics, both recomputing p from the saved lse:
+// Two kernels, neither with atomics, both recomputing p from the saved lse (the default):
 //
 // bwd_dkdv_tc_kernel   A CTA owns one 128-key tile of a (b,h) at a time and walks the 128-row query tiles that may
 //   see it.  Scores are computed TRANSPOSED (S^T = K Q^T, dP^T = V dout^T: TMEM lane = key, column = query) so that
@@ -19,6 +19,12 @@
 //   thread per row) and streams 128-key tiles; per tile S = Q K^T -> p (kept in registers), then dP = dout V^T into
 //   the same TMEM columns -> dS (bf16, in place) -> dQ += dS K with K read MN-major.  The work is scheduled like the
 //   forward (groups that split the key range write fp32 partial dQ to the workspace; a small kernel adds them).
+//
+// bwd_fused_tc_kernel  (d = 128, on request)  The dK/dV kernel with a third accumulating product per chain step,
+//   dQ^T_x = K^T dS^T_x (K read MN-major, dS^T_x also written to shared memory as the B operand) into the chain's dead
+//   dP^T_x columns, which the chain's threads read back and add to an fp32 dQ buffer with reductions in L2; a small kernel
+//   scales and rounds it.  Five matrix products instead of seven, but 32 KB of reductions per chain step, and an SM gets
+//   about 25 bytes per clock of those: measured within +-10 % of the two kernels.
 //
 // A preparation kernel writes lse*log2(e) and delta per query row, padded to a multiple of 128 rows per (b,h) with
 // +inf / 0: a padded row then gives p = 0 without any test.
@@ -398,6 +404,387 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(&pds_full[wg]);
+            }
+            if (!ok) break;
+            // ---------------------------------------------------------------- dK, dV of this key tile
+            ok = __all_sync(0xffffffffu, mbar_wait(acc_full, n & 1, abort_p));
+            if (!ok) break;
+            tc_fence_after();
+            // Each thread holds half a row (D/2 columns) of dK and of dV.  Written straight from the registers a warp's store
+            // would touch 32 different lines; the warp passes its 32 x D bytes through shared memory (16-byte pieces, piece
+            // index xor row so that neither side has bank conflicts beyond the minimum) and stores whole lines instead.
+            constexpr int kPieces = D / 16;                    // 16-byte pieces per half row
+            constexpr int kRowsPerStore = 32 / kPieces;
+            uint8_t* stage = smem + C::kOffStage + warp * (32 * D);
+            const int key_warp = t * kTileN + (warp & 3) * 32;     // key of lane 0
+#pragma unroll
+            for (int which = 0; which < 2; ++which) {
+                const uint32_t tA = tmem_base + lane_addr + (which == 0 ? C::kColDK : C::kColDV) + wg * (D / 2);
+                const float f = which == 0 ? p.scale : 1.f;
+#pragma unroll
+                for (int c = 0; c < D / 64; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tA + c * 32, o);
+#pragma unroll
+                    for (int v4 = 0; v4 < 4; ++v4) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(o[v4 * 8 + 0]) * f, __uint_as_float(o[v4 * 8 + 1]) * f);
+                        w.y = pack_bf16x2(__uint_as_float(o[v4 * 8 + 2]) * f, __uint_as_float(o[v4 * 8 + 3]) * f);
+                        w.z = pack_bf16x2(__uint_as_float(o[v4 * 8 + 4]) * f, __uint_as_float(o[v4 * 8 + 5]) * f);
+                        w.w = pack_bf16x2(__uint_as_float(o[v4 * 8 + 6]) * f, __uint_as_float(o[v4 * 8 + 7]) * f);
+                        const int piece = c * 4 + v4;
+                        *reinterpret_cast<uint4*>(stage + lane * D + ((piece ^ (lane & (kPieces - 1))) << 4)) = w;
+                    }
+                }
+                __syncwarp();
+                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(which == 0 ? p.dk : p.dv) +
+                                     ((long long)bh * p.N + key_warp) * D + wg * (D / 2);
+#pragma unroll
+                for (int it = 0; it < 32 / kRowsPerStore; ++it) {
+                    const int rrow = it * kRowsPerStore + lane / kPieces, piece = lane % kPieces;
+                    const uint4 w = *reinterpret_cast<const uint4*>(stage + rrow * D + ((piece ^ (rrow & (kPieces - 1))) << 4));
+                    if (key_warp + rrow < p.N) *reinterpret_cast<uint4*>(dst + (long long)rrow * D + piece * 8) = w;
+                }
+                __syncwarp();
+            }
+            tc_fence_before();
+            mbar_arrive(acc_empty);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, base_ok ? (int)TLIN_ERR_TIMEOUT : (int)TLIN_ERR_CUDA);
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ------------------------------------------------------------------------------------------ dK / dV / dQ in one kernel
+// The dK/dV kernel with a third accumulating product per chain step: dQ^T_x = K^T dS^T_x goes into the chain's dead dP^T_x
+// columns (dS^T_x now sits beside P^T_x over S^T_x), is read back by the chain's threads and added to an fp32 dQ buffer in the
+// workspace with reductions in L2.  Scores are computed once: five matrix products per (query, key) pair instead of seven.
+template <int D>
+__global__ void __launch_bounds__(ACfg<D>::kThreads, 1)
+bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do, const BwdParams p) {
+    using C = ACfg<D>;
+    static_assert(D == 128, "the transposed dQ accumulator needs M = d = 128");
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint8_t* sKV = smem + C::kOffKV;          // K, V
+    uint8_t* sRing = smem + C::kOffRing;      // [kSlots][Q 64 rows | dout 64 rows]
+    float* sStats = reinterpret_cast<float*>(smem + C::kOffStats);   // [kSlots][lse2 64 | delta 64]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kOffBars);
+    uint64_t* kv_full = bars + 0;
+    uint64_t* kv_empty = bars + 1;
+    uint64_t* sdp_full = bars + 2;    // [2] S^T_x and dP^T_x of a step are in TMEM
+    uint64_t* pds_full = bars + 4;    // [2] the chain's threads have stored P^T_x and dS^T_x
+    uint64_t* acc_full = bars + 6;    // dK, dV of the key tile are complete
+    uint64_t* acc_empty = bars + 7;   // all threads have read them
+    uint64_t* slot_full = bars + 8;   // [kSlots]
+    uint64_t* slot_empty = slot_full + C::kSlots;
+    uint64_t* dqt_full = bars + C::kNumBars;        // [2] dQ^T_x of a chain step is in TMEM
+    uint64_t* dq_drained = dqt_full + 2;            // [2] the chain's threads hold it in registers: its columns are free
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::kNumBars + 4);
+    int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool base_ok = (smem_u32(smem) & 1023u) == 0;   // the swizzled tiles need 1024-byte alignment
+
+    if (threadIdx.x == 0) {
+        *abort_flag = base_ok ? 0 : 1;
+        mbar_init(kv_full, 1);
+        mbar_init(kv_empty, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sdp_full[i], 1);
+            mbar_init(&pds_full[i], 128);
+            mbar_init(&dqt_full[i], 1);
+            mbar_init(&dq_drained[i], 128);
+        }
+        for (int i = 0; i < C::kSlots; ++i) {
+            mbar_init(&slot_full[i], 1);
+            mbar_init(&slot_empty[i], 1);
+        }
+        mbar_init(acc_full, 1);
+        mbar_init(acc_empty, 256);
+        fence_mbar_init();
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(tmem_slot, 512);
+        tmem_relinquish();
+    }
+    if (warp == kProducerWarp && lane == 0) {
+        prefetch_tensormap(&map_q);
+        prefetch_tensormap(&map_k);
+        prefetch_tensormap(&map_v);
+        prefetch_tensormap(&map_do);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    volatile int* abort_p = abort_flag;
+
+    // The CTAs share the (b,h,key tile) units by cost (query tiles a key tile has to visit), not by count: with the
+    // window rule the last key tiles of a (b,h) are cheaper, down to one step.
+    const long long u_begin = bwd_first_unit_of_share(p.N, p.W, p.causal, p.total_units, p.key_tiles, blockIdx.x, gridDim.x);
+    const long long u_end = bwd_first_unit_of_share(p.N, p.W, p.causal, p.total_units, p.key_tiles, blockIdx.x + 1, gridDim.x);
+
+    if (warp == kProducerWarp) {
+        // ------------------------------------------------------------------ TMA producer: Q / dout / row statistics ring
+        // The ring runs ahead of the key tiles: the first chain steps of the next key tile are loaded while the
+        // current one is still being worked on.
+        if (lane == 0) {
+            bool ok = base_ok;
+            uint32_t hh = 0;                // chain steps (64 queries each) issued
+            for (long long u = u_begin; u < u_end && ok; ++u) {
+                const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
+                const int row_first = first_q_tile(p, t) * kQTile, row_end = p.q_tiles128 * kQTile;
+                for (int row = row_first; row < row_end && ok; row += 64, ++hh) {
+                    const uint32_t slot = hh % C::kSlots, round = hh / C::kSlots;
+                    ok = mbar_wait(&slot_empty[slot], (round & 1) ^ 1, abort_p);
+                    if (!ok) break;
+                    uint8_t* dst = sRing + slot * C::kSlotBytes;
+                    mbar_arrive_expect_tx(&slot_full[slot], C::kSlotBytes + 512);
+                    for (int x = 0; x < C::kBoxes; ++x) {
+                        tma_load_3d(dst + x * (64 * 128), &map_q, &slot_full[slot], x * 64, row, bh);
+                        tma_load_3d(dst + C::kHalfBytes + x * (64 * 128), &map_do, &slot_full[slot], x * 64, row, bh);
+                    }
+                    bulk_load_1d(sStats + slot * 128, p.lse2 + (long long)bh * p.Wpad + row, 256, &slot_full[slot]);
+                    bulk_load_1d(sStats + slot * 128 + 64, p.delta + (long long)bh * p.Wpad + row, 256, &slot_full[slot]);
+                }
+            }
+            if (!ok && base_ok) {
+                int dummy = 0;              // leave no copy in flight: the barriers armed last must complete (bounded)
+                for (uint32_t back = 1; back <= (uint32_t)C::kSlots && back <= hh; ++back) {
+                    const uint32_t id = hh - back;
+                    mbar_wait(&slot_full[id % C::kSlots], (id / C::kSlots) & 1, &dummy, 200000000LL);
+                }
+            }
+        }
+    } else if (warp == kKvWarp) {
+        // ------------------------------------------------------------------ TMA producer: K, V of the key tiles
+        if (lane == 0) {
+            bool ok = base_ok;
+            uint32_t n = 0;
+            for (long long u = u_begin; u < u_end && ok; ++u, ++n) {
+                const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
+                if (u + 1 < u_end) {        // K, V have one buffer: the next tile's rows come as far as L2 meanwhile
+                    const int bh_n = (int)((u + 1) / p.key_tiles), t_n = (int)(u + 1 - (long long)bh_n * p.key_tiles);
+                    for (int x = 0; x < C::kBoxes; ++x) {
+                        tma_prefetch_l2_3d(&map_k, x * 64, t_n * kTileN, bh_n);
+                        tma_prefetch_l2_3d(&map_v, x * 64, t_n * kTileN, bh_n);
+                    }
+                }
+                ok = mbar_wait(kv_empty, (n & 1) ^ 1, abort_p);
+                if (!ok) break;
+                mbar_arrive_expect_tx(kv_full, 2 * C::kTileBytes);
+                for (int x = 0; x < C::kBoxes; ++x) {
+                    tma_load_3d(sKV + x * (kQTile * 128), &map_k, kv_full, x * 64, t * kTileN, bh);
+                    tma_load_3d(sKV + C::kTileBytes + x * (kQTile * 128), &map_v, kv_full, x * 64, t * kTileN, bh);
+                }
+            }
+            if (!ok && base_ok && n > 0) {
+                int dummy = 0;
+                mbar_wait(kv_full, (n - 1) & 1, &dummy, 200000000LL);
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------------ MMA issuer (all lanes walk, one issues)
+        const uint32_t idesc_st = make_idesc_bf16(kQTile, 64, 0, 0);         // S^T, dP^T of a chain: M = keys, N = 64 queries
+        const uint32_t idesc_acc = make_idesc_bf16(kQTile, D, 0, 1);         // dV, dK: A in TMEM, B MN-major
+        const uint32_t idesc_dqt = make_idesc_bf16(D, 64, 1, 1);             // dQ^T_x = K^T dS^T_x: M = d, N = 64 queries, K = keys; both MN-major
+        const uint64_t kmaj = make_smem_desc_sw128(smem_u32(smem), 16, 1024);
+        const uint64_t mnmaj = make_smem_desc_sw128(smem_u32(smem), 64 * 128, 1024);   // 64-row tiles: 8 KB between column blocks
+        const uint32_t desc_hi = (uint32_t)(kmaj >> 32);
+        const uint32_t kmaj_lo = (uint32_t)kmaj, mnmaj_lo = (uint32_t)mnmaj;
+        const uint32_t mnmaj128_lo = (uint32_t)make_smem_desc_sw128(smem_u32(smem), kQTile * 128, 1024);   // 128-row tile: 16 KB between column blocks
+        const uint32_t ds_off = (uint32_t)(C::kOffStage >> 4);              // dS^T_x tiles: chain x at + x * 16 KB
+        const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
+        const uint32_t tDK = tmem_u + C::kColDK, tDV = tmem_u + C::kColDV;
+        const uint32_t k_off = (uint32_t)(C::kOffKV >> 4), v_off = (uint32_t)((C::kOffKV + C::kTileBytes) >> 4);
+        // [S^T_x | dP^T_x] = [K Q_x^T | V dout_x^T]: A a 128-row K-major tile, B the 64-row K-major tile of the slot
+        auto issue_sdp = [&](int x, uint32_t slot) {
+            const uint32_t q_off = (uint32_t)((C::kOffRing + slot * C::kSlotBytes) >> 4), do_off = q_off + (uint32_t)(C::kHalfBytes >> 4);
+            const uint32_t d = tmem_u + C::kColR + x * 128;
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t a16 = ((kk >> 2) * (kQTile * 128) + (kk & 3) * 32) >> 4, b16 = ((kk >> 2) * (64 * 128) + (kk & 3) * 32) >> 4;
+                if (elect_one()) mma_ss_parts(d, kmaj_lo + k_off + a16, kmaj_lo + q_off + b16, desc_hi, idesc_st, kk > 0);
+            }
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t a16 = ((kk >> 2) * (kQTile * 128) + (kk & 3) * 32) >> 4, b16 = ((kk >> 2) * (64 * 128) + (kk & 3) * 32) >> 4;
+                if (elect_one()) mma_ss_parts(d + 64, kmaj_lo + v_off + a16, kmaj_lo + do_off + b16, desc_hi, idesc_st, kk > 0);
+            }
+            commit_elected(&sdp_full[x]);
+        };
+        // dV += P^T_x dout_x, dK += dS^T_x Q_x: A in TMEM (64 queries = 32 columns), B the slot's 64-row tile read MN-major
+        auto issue_acc = [&](int x, uint32_t slot, bool accumulate) {
+            const uint32_t q_off = (uint32_t)((C::kOffRing + slot * C::kSlotBytes) >> 4), do_off = q_off + (uint32_t)(C::kHalfBytes >> 4);
+            const uint32_t a = tmem_u + C::kColR + x * 128;
+            // dQ^T_x (d x 64 queries, over the dead dP^T_x columns) = K^T (the K tile read MN-major) dS^T_x (shared memory,
+            // MN-major); first, so that the chain's threads can take it away while dV and dK are in the pipe
+#pragma unroll
+            for (int kk = 0; kk < kTileN / 16; ++kk)
+                if (elect_one()) mma_ss_parts(a + 64, mnmaj128_lo + k_off + kk * (2048 >> 4), mnmaj_lo + ds_off + x * (16384 >> 4) + kk * (2048 >> 4),
+                                              desc_hi, idesc_dqt, kk > 0 ? 1u : 0u);
+            commit_elected(&dqt_full[x]);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                if (elect_one()) mma_ts_parts(tDV, a + kk * 8, mnmaj_lo + do_off + kk * (2048 >> 4), desc_hi, idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                if (elect_one()) mma_ts_parts(tDK, a + 32 + kk * 8, mnmaj_lo + q_off + kk * (2048 >> 4), desc_hi, idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+            commit_elected(&slot_empty[slot]);
+        };
+        bool ok = base_ok;
+        uint32_t g = 0, n = 0;              // 128-query steps done, key tiles done; chain x of step g uses ring entry 2g + x
+        int t = (int)(u_begin % p.key_tiles);
+        for (long long u = u_begin; u < u_end && ok; ++u, ++n, t = t + 1 == p.key_tiles ? 0 : t + 1) {
+            const int steps = p.q_tiles128 - first_q_tile(p, t);
+            ok = __all_sync(0xffffffffu, mbar_wait(kv_full, n & 1, abort_p));
+            if (!ok) break;
+            for (int x = 0; x < 2 && ok; ++x) {
+                const uint32_t hh = 2 * g + x;
+                ok = __all_sync(0xffffffffu, mbar_wait(&slot_full[hh % C::kSlots], (hh / C::kSlots) & 1, abort_p));
+                if (!ok) break;
+                if (g > 0) {                                // dP^T_x is written over the chain's previous dQ^T_x
+                    ok = __all_sync(0xffffffffu, mbar_wait(&dq_drained[x], (g - 1) & 1, abort_p));
+                    if (!ok) break;
+                }
+                issue_sdp(x, hh % C::kSlots);
+            }
+            if (!ok) break;
+            for (int s = 0; s < steps && ok; ++s, ++g) {
+                const bool have_next = s + 1 < steps;
+                for (int x = 0; x < 2 && ok; ++x) {
+                    const uint32_t hh = 2 * g + x;
+                    ok = __all_sync(0xffffffffu, mbar_wait(&pds_full[x], g & 1, abort_p));
+                    if (!ok) break;
+                    if (s == 0 && x == 0 && n > 0) {        // the previous key tile's dK, dV must have been read out
+                        ok = __all_sync(0xffffffffu, mbar_wait(acc_empty, (n - 1) & 1, abort_p));
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+                    issue_acc(x, hh % C::kSlots, s > 0 || x > 0);
+                }
+                if (!ok) break;
+                if (!have_next) commit_elected(kv_empty);   // K (read by the dQ^T products) and V are free for the next key tile
+                // the next score products of a chain overwrite its dQ^T_x: they follow its drain, which runs while the
+                // other chain's products are in the pipe
+                for (int x = 0; x < 2 && ok && have_next; ++x) {
+                    const uint32_t hn = 2 * g + x + 2;
+                    ok = __all_sync(0xffffffffu, mbar_wait(&slot_full[hn % C::kSlots], (hn / C::kSlots) & 1, abort_p));
+                    if (!ok) break;
+                    ok = __all_sync(0xffffffffu, mbar_wait(&dq_drained[x], g & 1, abort_p));
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_sdp(x, hn % C::kSlots);
+                }
+                if (!ok) break;
+            }
+            if (!ok) break;
+            commit_elected(acc_full);
+        }
+    } else if (warp < 8) {
+        // ------------------------------------------------------------------ elementwise threads
+        const int wg = warp >> 2;                              // chain: which 64 queries of every tile
+        const int r = (warp & 3) * 32 + lane;                  // key row inside the tile == TMEM lane
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_base + lane_addr + C::kColR + wg * 128;
+        const uint32_t tDP = tS + 64;
+        bool ok = base_ok;
+        uint32_t g = 0, n = 0;
+        int bh = (int)(u_begin / p.key_tiles), t = (int)(u_begin - (long long)bh * p.key_tiles);
+        for (long long u = u_begin; u < u_end && ok; ++u, ++n, ++t) {
+            if (t == p.key_tiles) {
+                t = 0;
+                ++bh;
+            }
+            const int key = t * kTileN + r;
+            const int i_first = first_q_tile(p, t);
+            const long long shift = (long long)p.N - p.W;       // query q may use key k iff q >= k - shift
+            const int q_min = p.causal ? (int)((long long)key - shift) : -0x7fffffff;
+            const int q_min_warp = p.causal ? (int)((long long)key - lane + 31 - shift) : -0x7fffffff;   // largest in the warp
+            for (int i = i_first; i < p.q_tiles128; ++i, ++g) {
+                const uint32_t hh = 2 * g + wg, slot = hh % C::kSlots;
+                const float* st = sStats + slot * 128;
+                const int q0 = i * kQTile + wg * 64;              // first query of this thread's columns
+                ok = __all_sync(0xffffffffu, mbar_wait(&sdp_full[wg], g & 1, abort_p));
+                if (!ok) break;
+                // already complete (the MMAs waited for it); observing it here orders the bulk-copied lse2 / delta
+                // before this thread's reads
+                ok = __all_sync(0xffffffffu, mbar_wait(&slot_full[slot], (hh / C::kSlots) & 1, abort_p));
+                if (!ok) break;
+                tc_fence_after();
+                const bool masked = q0 < q_min_warp;              // warp-uniform: some element of some lane is masked
+                // all of S^T_x comes into registers first: dS^T_x goes into the second half of its columns
+                uint32_t sv[2][32];
+                tmem_ld32_async(tS, sv[0]);
+                tmem_ld32_async(tS + 32, sv[1]);
+                tmem_wait_ld(sv[0]);
+                tmem_wait_ld(sv[1]);
+                uint8_t* ds_row = smem + C::kOffStage + wg * 16384 + r * 128;       // this key's row of the dS^T_x tile
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t dv_[32];
+                    tmem_ld32(tDP + h * 32, dv_);
+                    uint32_t pk[16], dk_[16];
+#pragma unroll
+                    for (int c = 0; c < 32; c += 4) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(st + h * 32 + c);
+                        const float4 d4 = *reinterpret_cast<const float4*>(st + 64 + h * 32 + c);
+                        const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dlv[4] = {d4.x, d4.y, d4.z, d4.w};
+                        float pe[4], de[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            pe[e] = ex2(fmaf(__uint_as_float(sv[h][c + e]), p.scale_log2e, -lv[e]));
+                            if (masked && q0 + h * 32 + c + e < q_min) pe[e] = 0.f;
+                            de[e] = pe[e] * (__uint_as_float(dv_[c + e]) - dlv[e]);
+                        }
+                        pk[c / 2] = pack_bf16x2(pe[0], pe[1]);
+                        pk[c / 2 + 1] = pack_bf16x2(pe[2], pe[3]);
+                        dk_[c / 2] = pack_bf16x2(de[0], de[1]);
+                        dk_[c / 2 + 1] = pack_bf16x2(de[2], de[3]);
+                    }
+                    // bf16 P^T_x over the first 32 columns of S^T_x, dS^T_x over the next 32 (all of S^T_x is in registers)
+                    tmem_st16(tS + h * 16, pk);
+                    tmem_st16(tS + 32 + h * 16, dk_);
+                    // and dS^T_x once more as the B operand of the dQ^T product: row = key, 64 queries = 128 bytes, 16-byte
+                    // pieces at (piece xor row mod 8), the layout the 128-byte swizzle of the descriptors expects
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4)
+                        *reinterpret_cast<uint4*>(ds_row + (((h * 4 + c4) ^ (r & 7)) << 4)) =
+                            make_uint4(dk_[c4 * 4], dk_[c4 * 4 + 1], dk_[c4 * 4 + 2], dk_[c4 * 4 + 3]);
+                }
+                tc_wait_st();
+                fence_proxy_async_smem();             // the tile was written with ordinary stores and is read by the MMA
+                tc_fence_before();
+                mbar_arrive(&pds_full[wg]);
+                // ------------------------------------------------------------ dQ^T_x of this step -> fp32 dQ (L2 reductions)
+                ok = __all_sync(0xffffffffu, mbar_wait(&dqt_full[wg], g & 1, abort_p));
+                if (!ok) break;
+                tc_fence_after();
+                // TMEM lane = column of dQ (this thread: r), TMEM column = query.  Once the values are in registers the columns
+                // are free for the chain's next score products.
+                uint32_t o[2][32];
+                tmem_ld32_async(tDP, o[0]);
+                tmem_ld32_async(tDP + 32, o[1]);
+                tmem_wait_ld(o[0]);
+                tmem_wait_ld(o[1]);
+                tc_fence_before();
+                mbar_arrive(&dq_drained[wg]);
+                // for one query the 32 lanes of a warp hold 32 consecutive floats of its row of the fp32 dQ buffer: one
+                // reduction instruction adds 128 consecutive bytes in L2
+                {
+                    float* drow = p.ws + ((long long)bh * p.Wpad + q0) * D + r;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) atomicAdd(drow + (long long)(h * 32 + e) * D, __uint_as_float(o[h][e]));
+                }
             }
             if (!ok) break;
             // ---------------------------------------------------------------- dK, dV of this key tile
@@ -924,7 +1311,87 @@ int launch_d(const void* q, const void* k, const void* v, const void* out, const
     return TLIN_OK;
 }
 
+// fp32 dQ sums (rows padded to 128 per (b,h)) -> scaled bf16 dQ; 8 elements per thread
+template <int D>
+__global__ void __launch_bounds__(256)
+bwd_dq_convert_kernel(const float* __restrict__ dq32, __nv_bfloat16* __restrict__ dq, int W, int Wpad, long long rows, float scale) {
+    constexpr int TPR = D / 8;              // threads per row
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    const long long row = idx / TPR;
+    const int piece = (int)(idx - row * TPR);
+    if (row >= rows) return;
+    const long long bh = row / W;
+    const int i = (int)(row - bh * W);
+    const float4* src = reinterpret_cast<const float4*>(dq32 + (bh * Wpad + i) * D + piece * 8);
+    const float4 a = src[0], b = src[1];
+    uint4 w;
+    w.x = pack_bf16x2(a.x * scale, a.y * scale);
+    w.y = pack_bf16x2(a.z * scale, a.w * scale);
+    w.z = pack_bf16x2(b.x * scale, b.y * scale);
+    w.w = pack_bf16x2(b.z * scale, b.w * scale);
+    *reinterpret_cast<uint4*>(dq + row * D + piece * 8) = w;
+}
+
+// One kernel for dK, dV and dQ (five matrix products per pair; dQ summed in fp32 by reductions in L2, then rounded).
+int launch_fused_128(const void* q, const void* k, const void* v, const void* out, const float* lse, const void* dout,
+                     void* dq, void* dk, void* dv, int B, int H, int N, int W, int causal, float* ws, int num_sms, cudaStream_t st) {
+    constexpr int D = 128;
+    const long long bh = (long long)B * H;
+    const int Wpad = (W + kQTile - 1) / kQTile * kQTile;
+    CUtensorMap mk, mv, mq64, mdo64;
+    int rc = make_map(&mk, k, D, N, bh);
+    if (rc == TLIN_OK) rc = make_map(&mv, v, D, N, bh);
+    if (rc == TLIN_OK) rc = make_map(&mq64, q, D, W, bh, 64);
+    if (rc == TLIN_OK) rc = make_map(&mdo64, dout, D, W, bh, 64);
+    if (rc != TLIN_OK) return rc;
+    BwdParams p;
+    float* lse2 = ws;
+    float* delta = ws + bh * Wpad;
+    float* dq32 = ws + 2 * bh * Wpad;
+    p.lse2 = lse2; p.delta = delta; p.dq = dq; p.dk = dk; p.dv = dv;
+    p.ws = dq32;
+    p.status = status_word();
+    if (!p.status) return TLIN_ERR_CUDA;
+    p.key_tiles = (N + kTileN - 1) / kTileN;
+    p.q_tiles128 = Wpad / kQTile;
+    p.N = N; p.W = W; p.Wpad = Wpad; p.causal = causal;
+    p.scale = 1.f / sqrtf((float)D);
+    p.scale_log2e = kLog2e * p.scale;
+    p.wide_stores = 0;
+    p.total_units = bh * p.key_tiles;
+    p.n_groups = 0; p.q_tiles = 0; p.schedule = 0;
+    static bool smem_allowed[64] = {};
+    constexpr int kSmem = ACfg<D>::kSmemBytes + 32;             // four more barriers than the dK/dV kernel
+    TLIN_CUDA_CHECK(allow_dynamic_smem(bwd_fused_tc_kernel<D>, kSmem, smem_allowed));
+    const long long rows_padded = bh * Wpad;
+    bwd_prep_kernel<D><<<(unsigned)((rows_padded + prep_rows_per_block<D>() - 1) / prep_rows_per_block<D>()), 256, 0, st>>>(
+        (const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse, lse2, delta, W, Wpad, rows_padded);
+    TLIN_CUDA_CHECK(cudaGetLastError());
+    TLIN_CUDA_CHECK(cudaMemsetAsync(dq32, 0, (size_t)rows_padded * D * sizeof(float), st));
+    const long long ctas = p.total_units < num_sms ? p.total_units : num_sms;
+    bwd_fused_tc_kernel<D><<<(unsigned)ctas, ACfg<D>::kThreads, kSmem, st>>>(mq64, mk, mv, mdo64, p);
+    TLIN_CUDA_CHECK(cudaGetLastError());
+    const long long rows = bh * W, threads = rows * (D / 8);
+    bwd_dq_convert_kernel<D><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(dq32, (__nv_bfloat16*)dq, W, Wpad, rows, p.scale);
+    TLIN_CUDA_CHECK(cudaGetLastError());
+    count_launch(3);
+    return TLIN_OK;
+}
+
 }  // namespace
+
+// row statistics (lse2, delta, padded) + the fp32 dQ sums, rows padded to 128 per (b,h)
+size_t bwd_fused_workspace_bytes(long long B, long long H, long long W, int d) {
+    const long long bh = B * H, Wpad = (W + tc::kQTile - 1) / tc::kQTile * tc::kQTile;
+    return (size_t)(2 * bh * Wpad + bh * Wpad * d) * sizeof(float);
+}
+
+int launch_bwd_fused(const void* q, const void* k, const void* v, const void* out, const float* lse, const void* dout,
+                     void* dq, void* dk, void* dv, int B, int H, int N, int W, int d, int causal, float* ws, int num_sms, cudaStream_t st) {
+    if (d != 128) return TLIN_ERR_UNSUPPORTED;
+    if ((long long)B * H * W > 0x7fffffffLL || (long long)B * H > 0x7fffffffLL) return TLIN_ERR_UNSUPPORTED;
+    return launch_fused_128(q, k, v, out, lse, dout, dq, dk, dv, B, H, N, W, causal, ws, num_sms, st);
+}
 
 // row statistics (lse2, delta, padded) + the dQ kernel's partial slots
 size_t bwd_tc_workspace_bytes(long long B, long long H, long long W, int d, const tlin_fwd_plan& plan) {

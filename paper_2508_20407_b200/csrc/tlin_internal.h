@@ -132,6 +132,11 @@ int launch_bwd_tc(const void* q, const void* k, const void* v, const void* out, 
                   void* dq, void* dk, void* dv, int B, int H, int N, int W, int d, int causal, const tlin_fwd_plan& plan,
                   float* ws, int num_sms, cudaStream_t st);
 size_t bwd_tc_workspace_bytes(long long B, long long H, long long W, int d, const tlin_fwd_plan& plan);
+// dK, dV and dQ in one tensor-core kernel (d = 128): scores computed once, dQ summed in an fp32 buffer of the workspace
+int launch_bwd_fused(const void* q, const void* k, const void* v, const void* out, const float* lse, const void* dout,
+                     void* dq, void* dk, void* dv, int B, int H, int N, int W, int d, int causal, float* ws, int num_sms, cudaStream_t st);
+size_t bwd_fused_workspace_bytes(long long B, long long H, long long W, int d);
+int backward_impl();
 int decode_table_max_problems();
 int launch_decode_table(const tlin_decode_problem* problems, int n, int d, cudaStream_t st);
 int launch_decode_fp8(const void* q_new, const void* k_new, const void* v_new, void* k_cache, void* v_cache,

@@ -228,6 +228,8 @@ def test_backward_workspace_covers_row_statistics_and_partial_sums():
             plan = tl.tlin_plan_forward(B, H, N, W, d, causal)
             tc = 4 * (2 * B * H * wpad + (plan.n_ctas * 2 * 256 * d if plan.uses_workspace else 0))
             need = max(need, tc)
+        if d == 128:        # the one-kernel arrangement: row statistics plus an fp32 dQ buffer on padded rows
+            need = max(need, 4 * B * H * wpad * (d + 2))
         assert got == need, (B, H, N, W, d, got, need)
     assert tl.workspace_bytes_backward(0, 1, 1, 1, 64) == 0
 

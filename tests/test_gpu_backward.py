@@ -25,11 +25,12 @@ REL_L2, REL_MAX, ABS_FLOOR = 2e-2, 2e-2, 1e-5
 IMPLS = [0, 1]      # 0: tensor-core kernels, 1: CUDA-core kernels (the same switch as the forward's)
 
 
-def grads(q, k, v, dout, causal, impl=0, guarded=False):
+def grads(q, k, v, dout, causal, impl=0, guarded=False, arrangement=0):
     """Gradients through the C-ABI.  guarded: dq, dk, dv and the workspace sit inside buffers of exactly the documented
-    sizes with filled guard regions on both sides, which must come back untouched."""
+    sizes with filled guard regions on both sides, which must come back untouched.  arrangement: tlin_set_backward_impl."""
     out, lse = tl.tlin_attn_forward(q, k, v, causal_window=causal)
     prev = tl.tlin_set_forward_impl(impl)
+    prev_arr = tl.tlin_set_backward_impl(arrangement)
     saved = tl._workspace_tensor
     gs = []
     try:
@@ -49,6 +50,7 @@ def grads(q, k, v, dout, causal, impl=0, guarded=False):
             assert tl._workspace_tensor is gw.t
     finally:
         tl.tlin_set_forward_impl(prev)
+        tl.tlin_set_backward_impl(prev_arr)
         if guarded:
             tl.set_workspace(saved)
     for g, name in gs:
@@ -67,16 +69,16 @@ def compare(got, ref, what):
     return e
 
 
-def run_case(B, H, N, W, d, causal, seed, peaky=False, impl=0, guarded=False):
+def run_case(B, H, N, W, d, causal, seed, peaky=False, impl=0, guarded=False, arrangement=0):
     wl = synth.Workload("bwd", B, H, d, N, W, seed=seed, causal_window=causal)
     q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
     if peaky:
         q = (q.float() * 6.0).to(torch.bfloat16)
     g = torch.Generator(device="cpu").manual_seed(seed + 7)
     dout = torch.randn(q.shape, generator=g, dtype=torch.float32).to(torch.bfloat16).to(DEV)
-    dq, dk, dv = grads(q, k, v, dout, causal, impl, guarded)
+    dq, dk, dv = grads(q, k, v, dout, causal, impl, guarded, arrangement)
     rq, rk, rv = oracle.attn_backward(q.cpu(), k.cpu(), v.cpu(), dout.cpu(), causal)
-    tag = f"B{B} H{H} N{N} W{W} d{d} causal{causal} impl{impl}"
+    tag = f"B{B} H{H} N{N} W{W} d{d} causal{causal} impl{impl} arrangement{arrangement}"
     compare(dq, rq, tag + " dq")
     compare(dk, rk, tag + " dk")
     compare(dv, rv, tag + " dv")
@@ -102,6 +104,37 @@ def test_backward_random_shapes_against_the_oracle(seed):
     from test_gpu_forward import random_shapes
     for (B, H, N, W, d, causal) in random_shapes(seed, 6, budget=1.5e9):
         run_case(B, H, N, W, d, causal, seed=seed * 1000 + N + W, impl=0, guarded=True)
+
+
+# the one-kernel arrangement (d = 128): the same element-by-element gates, guarded buffers, poisoned workspace
+ONE_KERNEL = [s for s in SHAPES if s[4] == 128] + [(1, 2, 40000, 300, 128, 1), (1, 1, 30000, 1024, 128, 0), (2, 40, 1600, 1500, 128, 1),
+                                                   (1, 1, 2048, 512, 128, 1), (1, 3, 2560, 768, 128, 1), (1, 5, 4000, 1000, 128, 1)]
+
+
+@pytest.mark.parametrize("B,H,N,W,d,causal", ONE_KERNEL)
+def test_backward_one_kernel_arrangement(B, H, N, W, d, causal):
+    assert tl.workspace_bytes_backward(B, H, N, W, d) >= B * H * (-(-W // 128) * 128) * (d + 2) * 4
+    run_case(B, H, N, W, d, causal, seed=600 + N + W, impl=0, guarded=True, arrangement=2)
+
+
+def test_backward_one_kernel_arrangement_repeats_dk_dv_bitwise_and_dq_within_fp32_addition_order():
+    wl = synth.Workload("bwd", 1, 2, 128, 30000, 300, seed=9, causal_window=1)
+    q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
+    dout = torch.randn(q.shape, device=DEV).to(torch.bfloat16)
+    a = grads(q, k, v, dout, 1, 0, arrangement=2)
+    b = grads(q, k, v, dout, 1, 0, arrangement=2)
+    assert torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])
+    diff = (a[0].float() - b[0].float()).abs()
+    assert float(diff.max()) <= 2.0 ** -7 * float(a[0].float().abs().max())
+    two = grads(q, k, v, dout, 1, 0, arrangement=1)
+    assert torch.equal(a[1], two[1]) and torch.equal(a[2], two[2])      # dK, dV: the same products in the same order
+
+
+def test_backward_arrangement_switch_rejects_other_values_and_other_head_sizes_keep_two_kernels():
+    assert tl.tlin_set_backward_impl(0) in (0, 1, 2)
+    assert tl.tlin_set_backward_impl(3) < 0 and tl.tlin_set_backward_impl(-1) < 0
+    run_case(1, 2, 515, 130, 64, 1, seed=4, impl=0, guarded=True, arrangement=2)     # d = 64
+    assert tl.tlin_last_launch_count() >= 3
 
 
 @pytest.mark.parametrize("impl", IMPLS)
@@ -330,7 +363,9 @@ def test_backward_both_kernel_families_agree_on_every_head_of_the_training_chunk
     dout = torch.randn(q.shape, generator=g, dtype=torch.float32).to(torch.bfloat16).to(DEV)
     tc = grads(q, k, v, dout, wl.causal_window, 0)
     cc = grads(q, k, v, dout, wl.causal_window, 1)
-    for a, b, name in zip(tc, cc, ("dq", "dk", "dv")):
+    one = grads(q, k, v, dout, wl.causal_window, 0, arrangement=2)
+    assert torch.equal(one[1], tc[1]) and torch.equal(one[2], tc[2])
+    for a, b, name in list(zip(tc, cc, ("dq", "dk", "dv"))) + [(one[0], cc[0], "dq (one kernel)")]:
         a, b = a.float(), b.float()
         assert torch.isfinite(a).all() and torch.isfinite(b).all(), name
         diff = (a - b).abs()
