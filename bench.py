@@ -377,22 +377,29 @@ def run_backward(wl, args, rank, world, device, peaks):
     ms_step = ms / args.steps
     flop = 10.0 * wl.B * wl.H * allowed_pairs(wl) * wl.d
     tflops = flop / (ms_step * 1e-3) / 1e12
-    # the one-kernel arrangement beside it (scores computed once, dQ by reductions in L2): same call, same timing
-    one_kernel = None
+    # the headline is the library's own choice of arrangement (tlin_set_backward_impl(0)); both arrangements beside it,
+    # same call, same timing
+    chosen = tl.tlin_backward_arrangement(wl.B, wl.H, wl.N, wl.W, wl.d)
+    one_kernel = two_kernels = None
     if wl.d == 128:
-        prev = tl.tlin_set_backward_impl(2)
-        try:
-            n_counted = len(launches)
-            ms1, _ = time_steps(step, args.steps, args.warmup, world, device, None, flush)
-            del launches[n_counted:]
-        finally:
-            tl.tlin_set_backward_impl(prev)
-        one_kernel = dict(ms_per_step=ms1 / args.steps, tflops=flop / (ms1 / args.steps * 1e-3) / 1e12,
-                          note="tlin_set_backward_impl(2): five matrix products instead of seven, dQ summed by fp32 reductions in L2")
+        n_counted = len(launches)
+        for mode in (1, 2):
+            prev = tl.tlin_set_backward_impl(mode)
+            try:
+                ms1, _ = time_steps(step, args.steps, args.warmup, world, device, None, flush)
+            finally:
+                tl.tlin_set_backward_impl(prev)
+            rec = dict(ms_per_step=ms1 / args.steps, tflops=flop / (ms1 / args.steps * 1e-3) / 1e12)
+            if mode == 1:
+                two_kernels = dict(rec, note="tlin_set_backward_impl(1): dK/dV kernel, then dQ kernel; seven matrix products, bitwise repeatable")
+            else:
+                one_kernel = dict(rec, note="tlin_set_backward_impl(2): five matrix products instead of seven, dQ summed by fp32 reductions in L2")
+        del launches[n_counted:]
     roof = dict(bound="tensor", achieved=tflops, peak=peaks["bf16_tflops"], unit="TFLOP/s", frac=tflops / peaks["bf16_tflops"],
                 traffic=None, algorithmic_bytes=nbytes, peak_source=peaks["source"] + " (burst)",
-                kernel="backward (row statistics, dK/dV kernel, dQ kernel, dQ partial sums)",
-                executed_over_counted_flops=1.4, roofline_ms=flop / (peaks["bf16_tflops"] * 1e12) * 1e3)
+                kernel=("backward (row statistics, dK/dV kernel, dQ kernel, dQ partial sums)" if chosen != 2 else
+                        "backward (row statistics, one dK/dV/dQ kernel with fp32 reductions, dQ rounding)"),
+                executed_over_counted_flops=1.4 if chosen != 2 else 1.0, roofline_ms=flop / (peaks["bf16_tflops"] * 1e12) * 1e3)
     if "bf16_tflops_sustained" in peaks:
         roof["frac_of_sustained_peak"] = tflops / peaks["bf16_tflops_sustained"]
     roof["nominal"] = dict(peak=NOMINAL_BF16_TFLOPS, unit="TFLOP/s", frac=tflops / NOMINAL_BF16_TFLOPS, note="datasheet dense bf16, context only")
@@ -400,7 +407,7 @@ def run_backward(wl, args, rank, world, device, peaks):
                "inputs+outputs %.0f MB: a %.0f MB buffer is overwritten before every timed call (L2 flush), calls timed one by one"
                % (nbytes / 1e6, flush.numel() / 1e6))
     return dict(workload=wl.name + " backward", shape=dict(B=wl.B, H=wl.H, N=wl.N, W=wl.W, d=wl.d, causal_window=wl.causal_window),
-                l2=l2_note, ms_per_step=ms_step, tflops=tflops, roofline=roof, e2e=None, clocks=clocks, one_kernel=one_kernel,
+                l2=l2_note, ms_per_step=ms_step, tflops=tflops, roofline=roof, e2e=None, clocks=clocks, arrangement=chosen, two_kernels=two_kernels, one_kernel=one_kernel,
                 gpu_launches=int(sum(launches[args.warmup:])), launches_per_step=launches[-1] if launches else 0)
 
 
@@ -728,7 +735,7 @@ def compact_leg(leg):
     c = leg.get("clocks") or {}
     out = {k: leg[k] for k in ("workload", "shape", "ms_per_step", "tflops", "gb_per_s", "tokens_per_s", "decode_tokens_per_s", "steps",
                                "gpu_launches", "launches_per_step", "separate_calls_ms_per_step", "batched_over_separate",
-                               "separate_launches_per_step", "eight_problems_of_8_heads", "decode_table", "one_kernel") if k in leg and leg[k] is not None}
+                               "separate_launches_per_step", "eight_problems_of_8_heads", "decode_table", "arrangement", "two_kernels", "one_kernel") if k in leg and leg[k] is not None}
     out["roofline"] = roof
     out["clocks"] = {"sm_mhz": c.get("sm_mhz"), "sm_max_mhz": c.get("sm_max_mhz"), "reasons": c.get("reasons", [])}
     if leg.get("e2e"):
@@ -853,7 +860,7 @@ def main():
             "tflops": main_res.get("tflops"),
             "gpu_launches": main_res["gpu_launches"], "launches_per_step": main_res["launches_per_step"],
             **{k: main_res[k] for k in ("separate_calls_ms_per_step", "batched_over_separate", "separate_launches_per_step",
-                                        "eight_problems_of_8_heads", "decode_table", "one_kernel") if k in main_res and main_res[k] is not None},
+                                        "eight_problems_of_8_heads", "decode_table", "arrangement", "two_kernels", "one_kernel") if k in main_res and main_res[k] is not None},
             "cpu_baseline": main_res.get("cpu_baseline"), "e2e": main_res["e2e"], "clocks": main_res["clocks"],
             "roofline": main_res["roofline"], "targets": targets,
         }

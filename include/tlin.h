@@ -236,8 +236,8 @@ int tlin_decode_step_static(const void* q_new, const void* k_new, const void* v_
  * out and lse are what tlin_attn_forward returned for the same q, k, v and causal_window (lse is
  * required here); dout is the loss gradient with respect to out; the loss must not depend on lse.
  * dq, dk, dv are overwritten (keys that no query may use get zeros).
- * bf16: d in {64,128} runs on the tensor cores (two kernels that recompute p, no atomics, bitwise repeatable; or, on request,
- * one kernel at d = 128: tlin_set_backward_impl); any other
+ * bf16: d in {64,128} runs on the tensor cores (two kernels that recompute p, no atomics, bitwise repeatable; or one kernel
+ * at d = 128 with dq summed by fp32 reductions, which small calls get by default: tlin_set_backward_impl); any other
  * d that is a multiple of 8 up to 256 runs on the CUDA-core kernels (dq summed with fp32 atomics).  f32: d a multiple
  * of 4 up to 256 (covers the paper's d = 36), CUDA-core kernels.
  * Needs a workspace of tlin_workspace_bytes_backward bytes (row sums, partial or accumulated dq in fp32).
@@ -353,16 +353,19 @@ const char* tlin_version(void);
 int tlin_set_forward_impl(int impl);
 /* How the tensor-core kernels of tlin_attn_backward (bf16, d = 64 or 128) are arranged; the chain rule of the Section 3
  * attention formula is the same in both (the paper gives no gradient algorithm of its own):
- *   1 (and 0, the default) = two kernels, dK/dV and then dQ, each recomputing the scores: seven matrix products per (query,
- *       key) pair, no atomics, bitwise repeatable;
- *   2 = one kernel (d = 128 only; other head sizes keep the two kernels): scores computed once, five matrix products per pair;
- *       the dQ contribution of every (128-key, 64-query) block is added to an fp32 buffer in the workspace by reductions
- *       in L2 and rounded to bf16 at the end, so dQ repeats only up to the order of those fp32 additions (dK, dV stay
- *       bitwise repeatable); needs B*H*ceil(W/128)*128*(d+2)*4 bytes of workspace, which tlin_workspace_bytes_backward
- *       includes.  Measured on B200 it is within +-10 % of the two kernels (faster on small and medium calls, slower on the
- *       largest), because the reductions, not the matrix products, bound its step.
- * Returns the old value; TLIN_ERR_INVALID_ARG for another argument. */
+ *   1 = two kernels, dK/dV and then dQ, each recomputing the scores: seven matrix products per (query, key) pair, no atomics,
+ *       bitwise repeatable;
+ *   2 = one kernel (d = 128 only; d = 64 keeps the two kernels): scores computed once, five matrix products per pair; the dQ
+ *       contribution of every (128-key, 64-query) block is added to an fp32 buffer in the workspace by reductions in L2 and
+ *       rounded to bf16 at the end, so dQ repeats only up to the order of those fp32 additions (dK, dV stay bitwise
+ *       repeatable); needs B*H*ceil(W/128)*128*(d+2)*4 bytes of workspace, which tlin_workspace_bytes_backward includes;
+ *   0 (the default) = the library chooses: arrangement 2 at d = 128 while that fp32 dQ buffer is at most 16 MiB (it then
+ *       stays in L2 beside the streaming inputs and the call is 2 to 13 % faster on B200), arrangement 1 otherwise (the
+ *       reductions, not the matrix products, bound arrangement 2, and with a larger buffer it is up to 15 % slower).
+ * Set 1 where bitwise repeatable gradients are needed.  Returns the old value; TLIN_ERR_INVALID_ARG for another argument.
+ * tlin_backward_arrangement: the arrangement (1 or 2) a call with these sizes gets under the current setting; host-only. */
 int tlin_set_backward_impl(int impl);
+int tlin_backward_arrangement(int B, int H, int N, int W, int d);
 /* Number of kernels launched by the last tlin_* compute call on this thread. */
 int tlin_last_launch_count(void);
 

@@ -88,6 +88,7 @@ SIGNATURES = {
     "tlin_version": (ctypes.c_char_p, []),
     "tlin_set_forward_impl": (_i, [_i]),
     "tlin_set_backward_impl": (_i, [_i]),
+    "tlin_backward_arrangement": (_i, [_i, _i, _i, _i, _i]),
     "tlin_last_launch_count": (_i, []),
 }
 
@@ -497,9 +498,15 @@ def tlin_set_forward_impl(impl: int) -> int:
 
 
 def tlin_set_backward_impl(impl: int) -> int:
-    """0: the library chooses, 1: two kernels (dK/dV, then dQ; bitwise repeatable), 2: one kernel (d = 128; dQ summed by
-    reductions in L2, repeatable up to the order of fp32 additions).  Returns the previous setting."""
+    """0: the library chooses (one kernel while the fp32 dQ buffer is at most 16 MiB), 1: two kernels (dK/dV, then dQ;
+    bitwise repeatable), 2: one kernel (d = 128; dQ summed by reductions in L2, repeatable up to the order of fp32
+    additions).  Returns the previous setting."""
     return int(lib().tlin_set_backward_impl(int(impl)))
+
+
+def tlin_backward_arrangement(B, H, N, W, d) -> int:
+    """1 (two kernels) or 2 (one kernel): what a bf16 backward call of these sizes gets under the current setting."""
+    return int(lib().tlin_backward_arrangement(B, H, N, W, d))
 
 
 def tlin_last_launch_count() -> int:

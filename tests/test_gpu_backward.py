@@ -25,9 +25,10 @@ REL_L2, REL_MAX, ABS_FLOOR = 2e-2, 2e-2, 1e-5
 IMPLS = [0, 1]      # 0: tensor-core kernels, 1: CUDA-core kernels (the same switch as the forward's)
 
 
-def grads(q, k, v, dout, causal, impl=0, guarded=False, arrangement=0):
+def grads(q, k, v, dout, causal, impl=0, guarded=False, arrangement=1):
     """Gradients through the C-ABI.  guarded: dq, dk, dv and the workspace sit inside buffers of exactly the documented
-    sizes with filled guard regions on both sides, which must come back untouched.  arrangement: tlin_set_backward_impl."""
+    sizes with filled guard regions on both sides, which must come back untouched.  arrangement: tlin_set_backward_impl
+    (1, the two kernels, unless a test asks for the one kernel or for the library's own choice)."""
     out, lse = tl.tlin_attn_forward(q, k, v, causal_window=causal)
     prev = tl.tlin_set_forward_impl(impl)
     prev_arr = tl.tlin_set_backward_impl(arrangement)
@@ -69,7 +70,7 @@ def compare(got, ref, what):
     return e
 
 
-def run_case(B, H, N, W, d, causal, seed, peaky=False, impl=0, guarded=False, arrangement=0):
+def run_case(B, H, N, W, d, causal, seed, peaky=False, impl=0, guarded=False, arrangement=1):
     wl = synth.Workload("bwd", B, H, d, N, W, seed=seed, causal_window=causal)
     q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
     if peaky:
@@ -128,6 +129,22 @@ def test_backward_one_kernel_arrangement_repeats_dk_dv_bitwise_and_dq_within_fp3
     assert float(diff.max()) <= 2.0 ** -7 * float(a[0].float().abs().max())
     two = grads(q, k, v, dout, 1, 0, arrangement=1)
     assert torch.equal(a[1], two[1]) and torch.equal(a[2], two[2])      # dK, dV: the same products in the same order
+
+
+@pytest.mark.parametrize("B,H,N,W,d,causal", [(1, 2, 4000, 300, 128, 1), (2, 2, 515, 130, 128, 0), (1, 3, 1000, 77, 64, 1)])
+def test_backward_with_the_arrangement_the_library_chooses(B, H, N, W, d, causal):
+    # setting 0: small fp32 dQ buffers (<= 16 MiB) take the one kernel at d = 128, everything else the two kernels
+    prev = tl.tlin_set_backward_impl(0)
+    try:
+        assert tl.tlin_backward_arrangement(B, H, N, W, d) == (2 if d == 128 else 1)
+        assert tl.tlin_backward_arrangement(4, 32, 8192, 1024, 128) == 1        # 64 MiB of fp32 dQ
+        assert tl.tlin_backward_arrangement(1, 32, 32768, 512, 128) == 2        # 8 MiB
+        assert tl.tlin_backward_arrangement(1, 1, 1, 1, 36) < 0 and tl.tlin_backward_arrangement(0, 1, 1, 1, 128) < 0
+        tl.tlin_set_backward_impl(1)
+        assert tl.tlin_backward_arrangement(B, H, N, W, d) == 1
+    finally:
+        tl.tlin_set_backward_impl(prev)
+    run_case(B, H, N, W, d, causal, seed=650 + N + W, impl=0, guarded=True, arrangement=0)
 
 
 def test_backward_arrangement_switch_rejects_other_values_and_other_head_sizes_keep_two_kernels():
