@@ -318,7 +318,7 @@ int tlin_plan_decode(int B, int H, int L, int d, int num_sms, tlin_decode_plan* 
  * towards the end of a (b,h).  -1 on bad arguments. */
 int64_t tlin_plan_backward_share_start(int B, int H, int N, int W, int causal_window, int share, int n_shares);
 /* First unit of group g.  floor(g * total_units / n_groups), except under schedule 1 with the window rule: there a
- * (b,h,query tile) problem costs the key tiles its rows may use (+2 for starting and finishing it), which grows with the
+ * (b,h,query tile) problem costs the key tiles its rows may use (+3 for starting and finishing it and for its masked steps), which grows with the
  * query tile, and when there are at least three problems per group the groups take contiguous runs of problems whose
  * costliest run is as cheap as contiguous runs allow (long problems) and which stay close to equal shares of the cost. */
 int64_t tlin_plan_group_start(const tlin_fwd_plan* plan, int g);

@@ -43,7 +43,8 @@ inline cudaError_t allow_dynamic_smem(Kernel kernel, int bytes, bool (&done)[64]
 // table to the kernel as a launch parameter (the CTAs only index it).
 // Schedule 0 (units = (b,h,key tile)) and unmasked schedule 1 (units = (b,h,256-row query tile pair) problems, all of one
 // cost): equal counts, group g starts at floor(g * units / groups).  Schedule 1 with the window rule: problem qt may use
-// ceil((N-W+min(W,256(qt+1)))/128) key tiles; its cost is that number plus 2 (starting and finishing a problem), and, when there
+// ceil((N-W+min(W,256(qt+1)))/128) key tiles; its cost is that number plus 3 (starting and finishing a problem, the masked steps on the diagonal and the step the
+// pair's second tile runs alone: measured 2.6 key-tile times), and, when there
 // are at least three problems per group, the groups take contiguous runs of problems by cost: every group starting where the
 // cost before it reaches its share of the total, and, for problems of 10 key-tile times or more on average, moved as little
 // as needed to make the costliest run as cheap as contiguous runs allow (with fewer than three problems per group the
@@ -55,7 +56,7 @@ inline long long fwd_problem_cost(int N, int W, int key_tiles, int qt) {
     if (rows_end > W) rows_end = W;
     long long tiles = ((long long)N - W + rows_end + 127) / 128;
     if (tiles > key_tiles) tiles = key_tiles;
-    return tiles + 2;
+    return tiles + 3;
 }
 // fills starts->u[0 .. plan.n_groups]; plan.n_groups <= kMaxGroups
 void fwd_group_starts(const tlin_fwd_plan& plan, GroupStarts* starts);
@@ -96,7 +97,7 @@ __host__ __device__ inline long long bwd_first_unit_of_share(int N, int W, int c
 }
 
 // Batched forward (a table of small problems in one launch).  Units are whole (problem, b*h, 256-row query tile pair)
-// problems in table order; a CTA takes a contiguous run of them, the runs balanced by cost (allowed key tiles + 2) with
+// problems in table order; a CTA takes a contiguous run of them, the runs balanced by cost (allowed key tiles + 3 under the window rule, + 2 without) with
 // the costliest run as cheap as contiguous runs allow.  prefix[x] = cost of the first x units (prefix.size() = units + 1);
 // fills starts[0 .. n_ctas], every CTA non-empty (n_ctas <= units).
 constexpr int kMaxBatch = 24;          // problems per launch of the batched kernel (its table travels as a launch parameter)

@@ -105,9 +105,9 @@ def _check_plan(p, B, H, N, W, d, causal):
     by_cost = p.schedule == 1 and causal and p.q_tiles > 1 and p.total_units >= 3 * p.n_groups
     if by_cost:
         # window rule, whole problems per CTA: problem qt may use ceil((N-W+min(W,256(qt+1)))/128) key tiles; the groups take
-        # contiguous runs of problems, and the costliest run (cost = tiles + 2 per problem) must be the optimum over all ways
+        # contiguous runs of problems, and the costliest run (cost = tiles + 3 per problem) must be the optimum over all ways
         # of cutting the list into n_groups runs, found here by bisection over a plain greedy pass
-        cost = [min(p.key_tiles, -(-(N - W + min(W, 256 * (qt + 1))) // 128)) + 2 for qt in range(p.q_tiles)]
+        cost = [min(p.key_tiles, -(-(N - W + min(W, 256 * (qt + 1))) // 128)) + 3 for qt in range(p.q_tiles)]
         all_costs = cost * (p.total_units // p.q_tiles)
         loads = [sum(all_costs[a:b]) for a, b in zip(starts, starts[1:])]
 
@@ -287,7 +287,7 @@ def _unit_costs(specs):
         for qt in range(q_tiles):
             if causal:
                 rows_end = min(w, (qt + 1) * 256)
-                per_qt.append(min(key_tiles, -(-(n - w + rows_end) // 128)) + 2)
+                per_qt.append(min(key_tiles, -(-(n - w + rows_end) // 128)) + 3)
             else:
                 per_qt.append(key_tiles + 2)
         costs.extend(per_qt * bh)
