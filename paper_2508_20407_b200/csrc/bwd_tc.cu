@@ -465,6 +465,7 @@ bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 // The dK/dV kernel with a third accumulating product per chain step: dQ^T_x = K^T dS^T_x goes into the chain's dead dP^T_x
 // columns (dS^T_x now sits beside P^T_x over S^T_x), is read back by the chain's threads and added to an fp32 dQ buffer in the
 // workspace with reductions in L2.  Scores are computed once: five matrix products per (query, key) pair instead of seven.
+// Columns of a chain: [P^T q0-31 | dS^T q0-31 | P^T q32-63 | dS^T q32-63] (16 each, written over S^T_x half by half) and dQ^T_x (64).
 template <int D>
 __global__ void __launch_bounds__(ACfg<D>::kThreads, 1)
 bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -633,10 +634,10 @@ bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             commit_elected(&dqt_full[x]);
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-                if (elect_one()) mma_ts_parts(tDV, a + kk * 8, mnmaj_lo + do_off + kk * (2048 >> 4), desc_hi, idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+                if (elect_one()) mma_ts_parts(tDV, a + (kk >> 1) * 32 + (kk & 1) * 8, mnmaj_lo + do_off + kk * (2048 >> 4), desc_hi, idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-                if (elect_one()) mma_ts_parts(tDK, a + 32 + kk * 8, mnmaj_lo + q_off + kk * (2048 >> 4), desc_hi, idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+                if (elect_one()) mma_ts_parts(tDK, a + (kk >> 1) * 32 + 16 + (kk & 1) * 8, mnmaj_lo + q_off + kk * (2048 >> 4), desc_hi, idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
             commit_elected(&slot_empty[slot]);
         };
         bool ok = base_ok;
@@ -696,6 +697,9 @@ bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const uint32_t tS = tmem_base + lane_addr + C::kColR + wg * 128;
         const uint32_t tDP = tS + 64;
         bool ok = base_ok;
+        // the second half of a step's dQ^T_x values waits in registers and is handed to L2 while the next step's products run
+        uint32_t held[32];
+        float* held_row = nullptr;
         uint32_t g = 0, n = 0;
         int bh = (int)(u_begin / p.key_tiles), t = (int)(u_begin - (long long)bh * p.key_tiles);
         for (long long u = u_begin; u < u_end && ok; ++u, ++n, ++t) {
@@ -720,17 +724,15 @@ bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 if (!ok) break;
                 tc_fence_after();
                 const bool masked = q0 < q_min_warp;              // warp-uniform: some element of some lane is masked
-                // all of S^T_x comes into registers first: dS^T_x goes into the second half of its columns
-                uint32_t sv[2][32];
-                tmem_ld32_async(tS, sv[0]);
-                tmem_ld32_async(tS + 32, sv[1]);
-                tmem_wait_ld(sv[0]);
-                tmem_wait_ld(sv[1]);
+                // 32 queries at a time: P^T and dS^T of a half go over the 32 columns of S^T_x that have just been read
                 uint8_t* ds_row = smem + C::kOffStage + wg * 16384 + r * 128;       // this key's row of the dS^T_x tile
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    uint32_t dv_[32];
-                    tmem_ld32(tDP + h * 32, dv_);
+                    uint32_t sv[32], dv_[32];
+                    tmem_ld32_async(tS + h * 32, sv);
+                    tmem_ld32_async(tDP + h * 32, dv_);
+                    tmem_wait_ld(sv);
+                    tmem_wait_ld(dv_);
                     uint32_t pk[16], dk_[16];
 #pragma unroll
                     for (int c = 0; c < 32; c += 4) {
@@ -740,7 +742,7 @@ bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                         float pe[4], de[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            pe[e] = ex2(fmaf(__uint_as_float(sv[h][c + e]), p.scale_log2e, -lv[e]));
+                            pe[e] = ex2(fmaf(__uint_as_float(sv[c + e]), p.scale_log2e, -lv[e]));
                             if (masked && q0 + h * 32 + c + e < q_min) pe[e] = 0.f;
                             de[e] = pe[e] * (__uint_as_float(dv_[c + e]) - dlv[e]);
                         }
@@ -749,9 +751,8 @@ bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                         dk_[c / 2] = pack_bf16x2(de[0], de[1]);
                         dk_[c / 2 + 1] = pack_bf16x2(de[2], de[3]);
                     }
-                    // bf16 P^T_x over the first 32 columns of S^T_x, dS^T_x over the next 32 (all of S^T_x is in registers)
-                    tmem_st16(tS + h * 16, pk);
-                    tmem_st16(tS + 32 + h * 16, dk_);
+                    tmem_st16(tS + h * 32, pk);
+                    tmem_st16(tS + h * 32 + 16, dk_);
                     // and dS^T_x once more as the B operand of the dQ^T product: row = key, 64 queries = 128 bytes, 16-byte
                     // pieces at (piece xor row mod 8), the layout the 128-byte swizzle of the descriptors expects
 #pragma unroll
@@ -763,28 +764,30 @@ bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 fence_proxy_async_smem();             // the tile was written with ordinary stores and is read by the MMA
                 tc_fence_before();
                 mbar_arrive(&pds_full[wg]);
-                // ------------------------------------------------------------ dQ^T_x of this step -> fp32 dQ (L2 reductions)
+                // ------------------------------------------------------------ dQ^T_x -> fp32 dQ (reductions in L2)
+                // For one query the 32 lanes of a warp hold 32 consecutive floats of its row of the fp32 dQ buffer: one
+                // reduction instruction adds 128 consecutive bytes.  The half kept from the previous step goes first, while
+                // this step's products are in the pipe.
+                if (held_row != nullptr) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) atomicAdd(held_row + (long long)e * D, __uint_as_float(held[e]));
+                }
                 ok = __all_sync(0xffffffffu, mbar_wait(&dqt_full[wg], g & 1, abort_p));
                 if (!ok) break;
                 tc_fence_after();
                 // TMEM lane = column of dQ (this thread: r), TMEM column = query.  Once the values are in registers the columns
                 // are free for the chain's next score products.
-                uint32_t o[2][32];
-                tmem_ld32_async(tDP, o[0]);
-                tmem_ld32_async(tDP + 32, o[1]);
-                tmem_wait_ld(o[0]);
-                tmem_wait_ld(o[1]);
+                uint32_t o[32];
+                tmem_ld32_async(tDP, o);
+                tmem_ld32_async(tDP + 32, held);
+                tmem_wait_ld(o);
+                tmem_wait_ld(held);
                 tc_fence_before();
                 mbar_arrive(&dq_drained[wg]);
-                // for one query the 32 lanes of a warp hold 32 consecutive floats of its row of the fp32 dQ buffer: one
-                // reduction instruction adds 128 consecutive bytes in L2
-                {
-                    float* drow = p.ws + ((long long)bh * p.Wpad + q0) * D + r;
+                float* drow = p.ws + ((long long)bh * p.Wpad + q0) * D + r;
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) atomicAdd(drow + (long long)(h * 32 + e) * D, __uint_as_float(o[h][e]));
-                }
+                for (int e = 0; e < 32; ++e) atomicAdd(drow + (long long)e * D, __uint_as_float(o[e]));
+                held_row = drow + 32LL * D;
             }
             if (!ok) break;
             // ---------------------------------------------------------------- dK, dV of this key tile
@@ -830,6 +833,10 @@ bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             }
             tc_fence_before();
             mbar_arrive(acc_empty);
+        }
+        if (held_row != nullptr) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) atomicAdd(held_row + (long long)e * D, __uint_as_float(held[e]));
         }
     }
 
