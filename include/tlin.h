@@ -359,9 +359,9 @@ int tlin_set_forward_impl(int impl);
  *       contribution of every (128-key, 64-query) block is added to an fp32 buffer in the workspace by reductions in L2 and
  *       rounded to bf16 at the end, so dQ repeats only up to the order of those fp32 additions (dK, dV stay bitwise
  *       repeatable); needs B*H*ceil(W/128)*128*(d+2)*4 bytes of workspace, which tlin_workspace_bytes_backward includes;
- *   0 (the default) = the library chooses: arrangement 2 at d = 128 while that fp32 dQ buffer is at most 16 MiB (it then
- *       stays in L2 beside the streaming inputs and the call is 2 to 13 % faster on B200), arrangement 1 otherwise (the
- *       reductions, not the matrix products, bound arrangement 2, and with a larger buffer it is up to 15 % slower).
+ *   0 (the default) = the library chooses: arrangement 2 at d = 128 while that fp32 dQ buffer is at most 64 MiB (2 to 13 %
+ *       faster on B200), arrangement 1 otherwise (beyond that size the two are level: the reductions, not the matrix
+ *       products, bound arrangement 2).
  * Set 1 where bitwise repeatable gradients are needed.  Returns the old value; TLIN_ERR_INVALID_ARG for another argument.
  * tlin_backward_arrangement: the arrangement (1 or 2) a call with these sizes gets under the current setting; host-only. */
 int tlin_set_backward_impl(int impl);

@@ -498,7 +498,7 @@ def tlin_set_forward_impl(impl: int) -> int:
 
 
 def tlin_set_backward_impl(impl: int) -> int:
-    """0: the library chooses (one kernel while the fp32 dQ buffer is at most 16 MiB), 1: two kernels (dK/dV, then dQ;
+    """0: the library chooses (one kernel while the fp32 dQ buffer is at most 64 MiB), 1: two kernels (dK/dV, then dQ;
     bitwise repeatable), 2: one kernel (d = 128; dQ summed by reductions in L2, repeatable up to the order of fp32
     additions).  Returns the previous setting."""
     return int(lib().tlin_set_backward_impl(int(impl)))

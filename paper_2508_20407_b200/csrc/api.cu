@@ -232,8 +232,9 @@ extern "C" int tlin_attn_forward_host(const void* q_h, const void* k_h, const vo
 }
 
 // Which arrangement of the tensor-core backward a bf16 call with these sizes gets.  The one-kernel arrangement pays for its
-// two saved matrix products with fp32 reductions into a B*H*ceil(W/128)*128*d*4-byte dQ buffer: while that buffer stays in
-// L2 beside the streaming inputs (measured: up to 16 MiB) it is 2 to 13 % faster than the two kernels, beyond that slower.
+// two saved matrix products with fp32 reductions into a B*H*ceil(W/128)*128*d*4-byte dQ buffer.  Measured against the two
+// kernels it is 2 to 13 % faster while that buffer is at most 64 MiB and level with them beyond (its CTAs take the key
+// tiles in turn, so the rows being added to stay in L2 at any size); beyond 64 MiB the bitwise repeatable two kernels run.
 extern "C" int tlin_backward_arrangement(int B, int H, int N, int W, int d) {
     if (B <= 0 || H <= 0 || N <= 0 || W <= 0) return TLIN_ERR_INVALID_ARG;
     if (d != 64 && d != 128) return TLIN_ERR_UNSUPPORTED;
@@ -242,7 +243,7 @@ extern "C" int tlin_backward_arrangement(int B, int H, int N, int W, int d) {
     if (mode != 0) return mode;
     const long long wpad = ((long long)W + 127) / 128 * 128;
     const long long dq32 = (long long)B * H * wpad * d * 4;
-    return dq32 <= (16LL << 20) ? 2 : 1;
+    return dq32 <= (64LL << 20) ? 2 : 1;
 }
 
 static int backward_common(const void* q, const void* k, const void* v, const void* out, const float* lse,

@@ -527,10 +527,11 @@ bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const uint32_t tmem_base = *tmem_slot;
     volatile int* abort_p = abort_flag;
 
-    // The CTAs share the (b,h,key tile) units by cost (query tiles a key tile has to visit), not by count: with the
-    // window rule the last key tiles of a (b,h) are cheaper, down to one step.
-    const long long u_begin = bwd_first_unit_of_share(p.N, p.W, p.causal, p.total_units, p.key_tiles, blockIdx.x, gridDim.x);
-    const long long u_end = bwd_first_unit_of_share(p.N, p.W, p.causal, p.total_units, p.key_tiles, blockIdx.x + 1, gridDim.x);
+    // The CTAs take the (b,h,key tile) units in turn (CTA c: units c, c + CTAs, ...), so that at any time all of them work on
+    // the key tiles of two or three (b,h): the rows of the fp32 dQ buffer they add to, and the Q / dout tiles they read, then
+    // stay in L2 whatever the size of the call.  With the window rule the last key tiles of a (b,h) are cheaper; taking units in
+    // turn spreads those evenly.
+    const long long u_begin = blockIdx.x, u_end = p.total_units, u_step = gridDim.x;
 
     if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ TMA producer: Q / dout / row statistics ring
@@ -539,7 +540,7 @@ bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (lane == 0) {
             bool ok = base_ok;
             uint32_t hh = 0;                // chain steps (64 queries each) issued
-            for (long long u = u_begin; u < u_end && ok; ++u) {
+            for (long long u = u_begin; u < u_end && ok; u += u_step) {
                 const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
                 const int row_first = first_q_tile(p, t) * kQTile, row_end = p.q_tiles128 * kQTile;
                 for (int row = row_first; row < row_end && ok; row += 64, ++hh) {
@@ -569,10 +570,10 @@ bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (lane == 0) {
             bool ok = base_ok;
             uint32_t n = 0;
-            for (long long u = u_begin; u < u_end && ok; ++u, ++n) {
+            for (long long u = u_begin; u < u_end && ok; u += u_step, ++n) {
                 const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
-                if (u + 1 < u_end) {        // K, V have one buffer: the next tile's rows come as far as L2 meanwhile
-                    const int bh_n = (int)((u + 1) / p.key_tiles), t_n = (int)(u + 1 - (long long)bh_n * p.key_tiles);
+                if (u + u_step < u_end) {   // K, V have one buffer: the next tile's rows come as far as L2 meanwhile
+                    const int bh_n = (int)((u + u_step) / p.key_tiles), t_n = (int)(u + u_step - (long long)bh_n * p.key_tiles);
                     for (int x = 0; x < C::kBoxes; ++x) {
                         tma_prefetch_l2_3d(&map_k, x * 64, t_n * kTileN, bh_n);
                         tma_prefetch_l2_3d(&map_v, x * 64, t_n * kTileN, bh_n);
@@ -642,8 +643,8 @@ bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         };
         bool ok = base_ok;
         uint32_t g = 0, n = 0;              // 128-query steps done, key tiles done; chain x of step g uses ring entry 2g + x
-        int t = (int)(u_begin % p.key_tiles);
-        for (long long u = u_begin; u < u_end && ok; ++u, ++n, t = t + 1 == p.key_tiles ? 0 : t + 1) {
+        for (long long u = u_begin; u < u_end && ok; u += u_step, ++n) {
+            const int t = (int)(u % p.key_tiles);
             const int steps = p.q_tiles128 - first_q_tile(p, t);
             ok = __all_sync(0xffffffffu, mbar_wait(kv_full, n & 1, abort_p));
             if (!ok) break;
@@ -701,12 +702,8 @@ bwd_fused_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         uint32_t held[32];
         float* held_row = nullptr;
         uint32_t g = 0, n = 0;
-        int bh = (int)(u_begin / p.key_tiles), t = (int)(u_begin - (long long)bh * p.key_tiles);
-        for (long long u = u_begin; u < u_end && ok; ++u, ++n, ++t) {
-            if (t == p.key_tiles) {
-                t = 0;
-                ++bh;
-            }
+        for (long long u = u_begin; u < u_end && ok; u += u_step, ++n) {
+            const int bh = (int)(u / p.key_tiles), t = (int)(u - (long long)bh * p.key_tiles);
             const int key = t * kTileN + r;
             const int i_first = first_q_tile(p, t);
             const long long shift = (long long)p.N - p.W;       // query q may use key k iff q >= k - shift

@@ -133,11 +133,12 @@ def test_backward_one_kernel_arrangement_repeats_dk_dv_bitwise_and_dq_within_fp3
 
 @pytest.mark.parametrize("B,H,N,W,d,causal", [(1, 2, 4000, 300, 128, 1), (2, 2, 515, 130, 128, 0), (1, 3, 1000, 77, 64, 1)])
 def test_backward_with_the_arrangement_the_library_chooses(B, H, N, W, d, causal):
-    # setting 0: small fp32 dQ buffers (<= 16 MiB) take the one kernel at d = 128, everything else the two kernels
+    # setting 0: fp32 dQ buffers up to 64 MiB take the one kernel at d = 128, everything else the two kernels
     prev = tl.tlin_set_backward_impl(0)
     try:
         assert tl.tlin_backward_arrangement(B, H, N, W, d) == (2 if d == 128 else 1)
-        assert tl.tlin_backward_arrangement(4, 32, 8192, 1024, 128) == 1        # 64 MiB of fp32 dQ
+        assert tl.tlin_backward_arrangement(4, 32, 4096, 4096, 128) == 1        # 256 MiB of fp32 dQ
+        assert tl.tlin_backward_arrangement(4, 32, 8192, 1024, 128) == 2        # 64 MiB
         assert tl.tlin_backward_arrangement(1, 32, 32768, 512, 128) == 2        # 8 MiB
         assert tl.tlin_backward_arrangement(1, 1, 1, 1, 36) < 0 and tl.tlin_backward_arrangement(0, 1, 1, 1, 128) < 0
         tl.tlin_set_backward_impl(1)
