@@ -300,8 +300,9 @@ def test_backward_f32(B, H, N, W, d, causal):
             assert e["rel_l2"] <= 1e-4, f"{name}: rel L2 {e['rel_l2']:.3e}"
 
 
-@pytest.mark.parametrize("name,heads", [("train_chunk", ((0, 0), (1, 16), (3, 31))), ("train_seq", ((2, 9),))])
-def test_backward_at_the_benchmarked_training_shapes_on_sampled_heads(name, heads):
+@pytest.mark.parametrize("name,heads,arrangement", [("train_chunk", ((0, 0), (1, 16), (3, 31)), 1), ("train_seq", ((2, 9),), 1),
+                                                    ("train_chunk", ((0, 5), (2, 0), (3, 30)), 0)])
+def test_backward_at_the_benchmarked_training_shapes_on_sampled_heads(name, heads, arrangement):
     # the full workloads bench.py times (train_chunk: B4 H32 N8192 W1024, the last window of a sliding-window pass;
     # train_seq: B4 H32 N=W=4096, a whole sequence over itself, where the CTAs share whole problems by cost); the
     # oracle recomputes whole (b,h) pairs, which are independent problems: the first, a middle and the last one
@@ -309,7 +310,7 @@ def test_backward_at_the_benchmarked_training_shapes_on_sampled_heads(name, head
     q, k, v = synth.forward_inputs(wl, device=DEV, dtype=torch.bfloat16)
     g = torch.Generator(device="cpu").manual_seed(wl.seed + 99)
     dout = torch.randn(q.shape, generator=g, dtype=torch.float32).to(torch.bfloat16).to(DEV)
-    dq, dk, dv = grads(q, k, v, dout, wl.causal_window, 0)
+    dq, dk, dv = grads(q, k, v, dout, wl.causal_window, 0, arrangement=arrangement)   # 0: what bench.py times (the library's choice)
     for b, h in heads:
         sl = (slice(b, b + 1), slice(h, h + 1))
         rq, rk, rv = oracle.attn_backward(q[sl].cpu(), k[sl].cpu(), v[sl].cpu(), dout[sl].cpu(), wl.causal_window)
